@@ -1,0 +1,316 @@
+"""Counter-based generator of scheduling-round inputs (see package docstring).
+
+Record layout (structure of arrays, scenario-major, row stride = max_actions):
+
+  pool        u8   index into the workload's pool list
+  unit        u8   low 7 bits: unit multiplier g (units per multiplicity step);
+                   bit 7 (GANG): on a GPU pool the g*r units of a level form ONE
+                   contiguous aligned chunk; without it a level is r chunks of g
+  level_mask  u32  bit (r-1) set  <=>  multiplicity r (1..32) is allowed
+  s_us, p_us  i64  runtime parameters in microseconds (invariant / scalable part)
+  arrival_us  i64  arrival time (replay workloads only, non-decreasing per row)
+  n_actions   i32  per scenario
+  gpu_busy    u8   per scenario x node (all GPU pools' nodes concatenated in pool
+                   order): bit b set <=> GPU b of that node is occupied beforehand
+
+Actions of one scenario are stored in queue (first-come first-served) order.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, Optional, Tuple
+
+import numpy as np
+
+POOL_CPU, POOL_GPU, POOL_API = 0, 1, 2
+GANG = 0x80
+
+_U = np.uint64
+
+
+@dataclass(frozen=True)
+class Pool:
+    type: int          # POOL_CPU | POOL_GPU | POOL_API
+    capacity: int      # cores | GPUs | tokens per window (or concurrent calls)
+    group: int         # CPU: cores per NUMA domain; GPU: GPUs per node; API: 0
+    window_us: int = 0  # API quota period; 0 = concurrency limited
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    n_scenarios: int
+    max_actions: int
+    pools: Tuple[Pool, ...]
+    recipe: str
+    base_seed: int = 0
+    depth: int = 2
+    round_us: int = 10_000
+    replay: bool = False
+    max_rounds: int = 0
+    params: Dict[str, float] = field(default_factory=dict)
+
+    @property
+    def n_nodes(self) -> int:
+        return sum(p.capacity // p.group for p in self.pools if p.type == POOL_GPU)
+
+
+# --------------------------------------------------------------------------- RNG
+def _splitmix64(x: np.ndarray) -> np.ndarray:
+    with np.errstate(over="ignore"):
+        z = x + _U(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> _U(30))) * _U(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> _U(27))) * _U(0x94D049BB133111EB)
+        return z ^ (z >> _U(31))
+
+
+class _Draws:
+    """Random fields of a [scenario, action] grid; field ids select independent streams."""
+
+    def __init__(self, base_seed: int, lo: int, hi: int, n_cols: int, salt: int = 0):
+        sc = (np.arange(lo, hi, dtype=np.uint64) + _U(base_seed % (1 << 63)))[:, None]
+        col = np.arange(n_cols, dtype=np.uint64)[None, :]
+        with np.errstate(over="ignore"):
+            h0 = _splitmix64(sc ^ (_U(salt) * _U(0x632BE59BD9B4E019)))
+            self._h1 = _splitmix64(h0 ^ (col * _U(0xD1342543DE82EF95)))
+
+    def bits(self, fid: int) -> np.ndarray:
+        with np.errstate(over="ignore"):
+            return _splitmix64(self._h1 + _U(fid) * _U(0xA24BAED4963EE407))
+
+    def uniform(self, fid: int) -> np.ndarray:
+        return ((self.bits(fid) >> _U(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
+
+    def normal(self, fid: int) -> np.ndarray:
+        u1, u2 = self.uniform(fid), self.uniform(fid + 1)
+        return np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+
+    def lognormal_us(self, fid: int, median: float, sigma: float) -> np.ndarray:
+        v = np.exp(np.log(median) + sigma * self.normal(fid))
+        return np.minimum(np.floor(v), float(1 << 40)).astype(np.int64)
+
+
+# fixed field ids (two consecutive ids are consumed by a normal draw)
+_F_POOL, _F_INEL, _F_LEVEL, _F_S, _F_P, _F_OUT, _F_SIZE, _F_ARR, _F_DUR, _F_BUSY = (
+    1, 2, 3, 4, 6, 8, 9, 10, 11, 12)
+
+
+def _pow2_mask(max_level: int) -> int:
+    m, r = 0, 1
+    while r <= max_level:
+        m |= 1 << (r - 1)
+        r *= 2
+    return m
+
+
+def _choose(u: np.ndarray, probs) -> np.ndarray:
+    edges = np.cumsum(np.asarray(probs, dtype=np.float64))
+    edges[-1] = 1.0 + 1e-9
+    return np.searchsorted(edges, u, side="right").astype(np.uint8)
+
+
+def _single_pow2_level(u: np.ndarray, n_levels: np.ndarray) -> np.ndarray:
+    """mask with exactly one power-of-two multiplicity, index uniform in [0, n_levels)."""
+    idx = np.minimum((u * n_levels).astype(np.int64), n_levels - 1)
+    r = np.left_shift(np.int64(1), idx)
+    return np.left_shift(np.uint32(1), (r - 1).astype(np.uint32)).astype(np.uint32)
+
+
+# --------------------------------------------------------------------- recipes
+def _mixed_round(w: Workload, d: _Draws, S: int, N: int):
+    """Configs 0, 1, 4: independent single rounds over CPU / GPU(gang) / API pools."""
+    P = w.params
+    pool = _choose(d.uniform(_F_POOL), P["mix"])
+    ptype = np.array([p.type for p in w.pools], dtype=np.int64)[pool]
+    # highest power-of-two multiplicity per pool ("capped by pool")
+    cap_level = np.array(
+        [min(P["max_level"], 8 if p.type == POOL_GPU else P["max_level"]) if p.type != POOL_API else 1
+         for p in w.pools], dtype=np.int64)[pool]
+    n_levels = np.floor(np.log2(cap_level)).astype(np.int64) + 1
+    full_mask = np.array([_pow2_mask(int(c)) for c in range(0, 33)], dtype=np.uint32)[cap_level]
+    inelastic = (d.uniform(_F_INEL) < P["inelastic"]) | (ptype == POOL_API)
+    one = _single_pow2_level(d.uniform(_F_LEVEL), n_levels)
+    mask = np.where(inelastic, one, full_mask).astype(np.uint32)
+    unit = np.where(ptype == POOL_GPU, 1 | GANG, 1).astype(np.uint8)
+    s = d.lognormal_us(_F_S, 20_000.0, P["sigma_s"])
+    p = d.lognormal_us(_F_P, 200_000.0, P["sigma_p"])
+    if P.get("outliers", 0.0) > 0.0:
+        big = d.uniform(_F_OUT) < P["outliers"]
+        s = np.where(big, np.minimum(s * 100, 1 << 40), s)
+        p = np.where(big, np.minimum(p * 100, 1 << 40), p)
+    return dict(pool=pool, unit=unit, level_mask=mask, s_us=s, p_us=p, arrival_us=None)
+
+
+def _topology_round(w: Workload, d: _Draws, S: int, N: int):
+    """Config 3: one GPU pool, chunk size 1/2/4/8, elastic replica count 1..4."""
+    P = w.params
+    size_idx = _choose(d.uniform(_F_SIZE), P["size_probs"]).astype(np.int64)
+    unit = np.left_shift(np.int64(1), size_idx).astype(np.uint8)            # g = chunk size, no GANG
+    mask = np.full((S, N), (1 << int(P["max_replicas"])) - 1, dtype=np.uint32)
+    s = d.lognormal_us(_F_S, 20_000.0, P["sigma_s"])
+    p = d.lognormal_us(_F_P, 200_000.0, P["sigma_p"])
+    return dict(pool=np.zeros((S, N), np.uint8), unit=unit, level_mask=mask, s_us=s, p_us=p,
+                arrival_us=None)
+
+
+def _replay_trace(w: Workload, d: _Draws, S: int, N: int):
+    """Config 2: Poisson arrivals; CPU code execution (Pareto) and GPU reward model (uniform)."""
+    P = w.params
+    gap = np.floor(-np.log(d.uniform(_F_ARR)) * (1e6 / P["rate_per_s"])).astype(np.int64)
+    arrival = np.cumsum(gap, axis=1)
+    is_gpu = d.uniform(_F_POOL) >= P["cpu_fraction"]
+    u = d.uniform(_F_DUR)
+    t_cpu = np.minimum(np.floor(P["pareto_min_us"] * u ** (-1.0 / P["pareto_alpha"])), float(1 << 40))
+    t_gpu = np.floor(P["gpu_lo_us"] + u * (P["gpu_hi_us"] - P["gpu_lo_us"]))
+    t_cpu, t_gpu = t_cpu.astype(np.int64), t_gpu.astype(np.int64)
+    s_gpu = t_gpu // 5
+    s = np.where(is_gpu, s_gpu, t_cpu)
+    p = np.where(is_gpu, t_gpu - s_gpu, 0)
+    pool = is_gpu.astype(np.uint8)                                            # pool 0 CPU, 1 GPU
+    unit = np.where(is_gpu, 1 | GANG, 1).astype(np.uint8)
+    mask = np.where(is_gpu, _pow2_mask(8), 1).astype(np.uint32)
+    return dict(pool=pool, unit=unit, level_mask=mask, s_us=s, p_us=p, arrival_us=arrival)
+
+
+_RECIPES = {"mixed": _mixed_round, "topology": _topology_round, "replay": _replay_trace}
+
+
+def _busy_masks(w: Workload, lo: int, hi: int) -> Optional[np.ndarray]:
+    """Pre-occupied GPUs as aligned chunks: every aligned block of 8, 4, 2, 1 GPUs is
+    independently occupied with the same probability q, (1-q)^4 = 1 - busy_fraction."""
+    frac = w.params.get("busy_fraction", 0.0)
+    nodes = w.n_nodes
+    if nodes == 0:
+        return None
+    out = np.zeros((hi - lo, nodes), dtype=np.uint8)
+    if frac <= 0.0:
+        return out
+    q = 1.0 - (1.0 - frac) ** 0.25
+    d = _Draws(w.base_seed, lo, hi, nodes * 15, salt=7)
+    u = d.uniform(_F_BUSY).reshape(hi - lo, nodes, 15) < q
+    k = 0
+    for size in (8, 4, 2, 1):
+        for start in range(0, 8, size):
+            bits = np.uint8(((1 << size) - 1) << start)
+            out |= np.where(u[:, :, k], bits, np.uint8(0))
+            k += 1
+    # nodes narrower than 8 GPUs: drop bits beyond the group
+    col = 0
+    for p in w.pools:
+        if p.type == POOL_GPU:
+            n = p.capacity // p.group
+            out[:, col:col + n] &= np.uint8((1 << p.group) - 1)
+            col += n
+    return out
+
+
+# ------------------------------------------------------------------- configs
+_CPU_NUMA = 64
+CONFIGS: Dict[str, Workload] = {
+    # single round, one scenario, 64 actions, levels {1,2,4,8}
+    "cfg0": Workload("cfg0", 1, 64, (Pool(POOL_CPU, 256, _CPU_NUMA), Pool(POOL_GPU, 8, 8)), "mixed",
+                     params=dict(mix=(0.5, 0.5), max_level=8, inelastic=0.0, sigma_s=1.0, sigma_p=1.2)),
+    # batched rounds, 4096 x 1024, CPU / GPU 8x8 / API 512 per second
+    "cfg1": Workload("cfg1", 4096, 1024,
+                     (Pool(POOL_CPU, 4096, _CPU_NUMA), Pool(POOL_GPU, 64, 8), Pool(POOL_API, 512, 0, 1_000_000)),
+                     "mixed", params=dict(mix=(0.60, 0.25, 0.15), max_level=16, inelastic=0.20,
+                                          sigma_s=1.5, sigma_p=1.5)),
+    # trace replay, 256 x 20000, Poisson 50/s, 10 ms rounds
+    "cfg2": Workload("cfg2", 256, 20000, (Pool(POOL_CPU, 256, _CPU_NUMA), Pool(POOL_GPU, 8, 8)), "replay",
+                     replay=True, max_rounds=60_000,
+                     params=dict(rate_per_s=50.0, cpu_fraction=0.70, pareto_alpha=1.3, pareto_min_us=5_000.0,
+                                 gpu_lo_us=50_000.0, gpu_hi_us=800_000.0)),
+    # topology constrained GPU pool, 1024 x 2048, 64 nodes x 8, 30 % pre-occupied
+    "cfg3": Workload("cfg3", 1024, 2048, (Pool(POOL_GPU, 512, 8),), "topology",
+                     params=dict(size_probs=(0.4, 0.3, 0.2, 0.1), max_replicas=4, busy_fraction=0.30,
+                                 sigma_s=1.0, sigma_p=1.2)),
+    # large mixed, 16384 x 4096, four pools
+    "cfg4": Workload("cfg4", 16384, 4096,
+                     (Pool(POOL_CPU, 8192, _CPU_NUMA), Pool(POOL_GPU, 128, 8),
+                      Pool(POOL_API, 1000, 0, 1_000_000), Pool(POOL_API, 200, 0, 1_000_000)),
+                     "mixed", params=dict(mix=(0.50, 0.25, 0.15, 0.10), max_level=32, inelastic=0.35,
+                                          sigma_s=2.0, sigma_p=2.0, outliers=0.01)),
+}
+
+
+def make_workload(name: str, n_scenarios: Optional[int] = None, max_actions: Optional[int] = None,
+                  base_seed: Optional[int] = None) -> Workload:
+    """A named configuration, optionally shrunk (same recipe, fewer scenarios / actions)."""
+    w = CONFIGS[name]
+    kw = {}
+    if n_scenarios is not None:
+        kw["n_scenarios"] = int(n_scenarios)
+    if max_actions is not None:
+        kw["max_actions"] = int(max_actions)
+    if base_seed is not None:
+        kw["base_seed"] = int(base_seed)
+    if not kw:
+        return w
+    from dataclasses import replace
+    return replace(w, **kw)
+
+
+def generate(w: Workload, lo: int = 0, hi: Optional[int] = None) -> Dict[str, Optional[np.ndarray]]:
+    """Input arrays of scenarios [lo, hi) of workload `w` (host numpy arrays, C contiguous)."""
+    hi = w.n_scenarios if hi is None else hi
+    S, N = hi - lo, w.max_actions
+    d = _Draws(w.base_seed, lo, hi, N)
+    a = _RECIPES[w.recipe](w, d, S, N)
+    a["n_actions"] = np.full(S, N, dtype=np.int32)
+    a["gpu_busy"] = _busy_masks(w, lo, hi)
+    for k in ("pool", "unit", "level_mask", "s_us", "p_us", "arrival_us"):
+        if a[k] is not None:
+            a[k] = np.ascontiguousarray(a[k])
+    return a
+
+
+# ------------------------------------------------- randomized rounds for tests
+def random_round(seed: int, n_scenarios: int, max_actions: int, pools: Tuple[Pool, ...],
+                 *, contiguous_levels: float = 0.3, max_mult: int = 8, inelastic: float = 0.25,
+                 small_durations: float = 0.0, busy_fraction: float = 0.0, ragged: bool = True,
+                 replicas: float = 0.5) -> Tuple[Workload, Dict[str, Optional[np.ndarray]]]:
+    """Adversarial little rounds for parity and property tests: arbitrary level masks
+    (power-of-two sets, contiguous ranges, random subsets), mixed gang/replica GPU
+    requests, ragged action counts, optional tiny durations (forces ties) and
+    pre-occupied GPUs."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    S, N = n_scenarios, max_actions
+    w = Workload(f"random{seed}", S, N, tuple(pools), "random", base_seed=seed,
+                 params=dict(busy_fraction=busy_fraction))
+    pool = rng.integers(0, len(pools), size=(S, N)).astype(np.uint8)
+    ptype = np.array([p.type for p in pools])[pool]
+    kind = rng.random((S, N))
+    r_hi = rng.integers(1, max_mult + 1, size=(S, N))
+    r_lo = np.minimum(rng.integers(1, max_mult + 1, size=(S, N)), r_hi)
+    contiguous = ((np.int64(1) << r_hi) - 1) & ~((np.int64(1) << (r_lo - 1)) - 1)
+    pow2 = np.array([_pow2_mask(int(c)) for c in range(0, 33)], dtype=np.int64)[r_hi]
+    subset = rng.integers(1, 1 << max_mult, size=(S, N))
+    mask = np.where(kind < contiguous_levels, contiguous, np.where(kind < 0.8, pow2, subset))
+    single = np.int64(1) << (rng.integers(0, max_mult, size=(S, N)))
+    mask = np.where(rng.random((S, N)) < inelastic, single, mask)
+    unit = np.ones((S, N), dtype=np.int64)
+    is_gpu = ptype == POOL_GPU
+    rep = is_gpu & (rng.random((S, N)) < replicas)
+    grp = np.array([max(p.group, 1) for p in pools], dtype=np.int64)[pool]
+    unit = np.where(rep, np.minimum(np.int64(1) << rng.integers(0, 4, size=(S, N)), grp), unit)
+    unit = np.where(is_gpu & ~rep, 1 | GANG, unit)
+    # gang requests need power-of-two levels <= GPUs per node; replicas keep few multiplicities
+    gang_ok = np.array([_pow2_mask(int(c)) for c in range(0, 33)], dtype=np.int64)[np.minimum(grp, 32)]
+    mask = np.where(is_gpu & ~rep, mask & gang_ok, mask)
+    mask = np.where(is_gpu & ~rep & (mask == 0), 1, mask)
+    mask = np.where(rep, mask & 0xF, mask)
+    mask = np.where(rep & (mask == 0), 1, mask)
+    mask = np.where(ptype == POOL_API, 1, mask)
+    if small_durations > 0.0:
+        tiny = rng.random((S, N)) < small_durations
+    else:
+        tiny = np.zeros((S, N), dtype=bool)
+    s = np.where(tiny, rng.integers(0, 4, size=(S, N)), rng.integers(0, 50_000, size=(S, N)))
+    p = np.where(tiny, rng.integers(0, 12, size=(S, N)), rng.integers(0, 500_000, size=(S, N)))
+    n_act = rng.integers(0, N + 1, size=S).astype(np.int32) if ragged else np.full(S, N, np.int32)
+    a = dict(pool=pool, unit=unit.astype(np.uint8), level_mask=mask.astype(np.uint32),
+             s_us=s.astype(np.int64), p_us=p.astype(np.int64), arrival_us=None, n_actions=n_act)
+    a["gpu_busy"] = _busy_masks(w, 0, S)
+    for k in ("pool", "unit", "level_mask", "s_us", "p_us"):
+        a[k] = np.ascontiguousarray(a[k])
+    return w, a
