@@ -1,0 +1,150 @@
+/*
+ * tangram.h -- C ABI of the batched elastic scheduling round (ARL-Tangram, arxiv 2603.13019)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * One call schedules one round for many independent cluster scenarios at once.  Per
+ * scenario it does what the paper's scheduler does when it is invoked (Section 4.2):
+ *   - evaluates the action-duration model at every allowed allocation level (Eq. 1),
+ *   - takes the longest queue prefix whose least-required units fit every pool, chunk
+ *     topology included (Algorithm 1, line 2),
+ *   - per pool, either takes all candidates at their only level (Algorithm 1, lines 5-6) or
+ *     runs the greedy eviction loop (lines 8-14) whose objective is the optimal discrete
+ *     allocation of the kept candidates (DPArrange, Algorithm 3, with the GPU chunk
+ *     operator of Algorithm 4) plus the completion-heap estimate of everything that keeps
+ *     waiting (Algorithm 2),
+ *   - places what it selected: aligned power-of-two GPU chunks, smallest sufficient free
+ *     chunk first (Section 5.3); exclusive cores, same NUMA domain first (Section 5.2);
+ *     quota or concurrency accounting (Section 5.1),
+ *   - reports allocation, placement and predicted action completion time (Eq. 2).
+ * tangram_replay_trace repeats this round by round over an arrival trace entirely on the
+ * device (the workflow of Section 3: submit, queue, schedule, execute, return).
+ *
+ * All times are integer microseconds.  Every entry point returns 0 or a negative
+ * TANGRAM_E* code; data-dependent problems are reported per scenario in `status`, never
+ * by a device trap.  Nothing is allocated after tangram_round_create.
+ */
+#ifndef TANGRAM_H_
+#define TANGRAM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* pool types (Section 5: CPU manager, GPU manager, basic manager) */
+#define TANGRAM_POOL_CPU 0
+#define TANGRAM_POOL_GPU 1
+#define TANGRAM_POOL_API 2
+
+/* bit 7 of an action's `unit` byte: on a GPU pool the g*r GPUs of a level are ONE aligned
+ * chunk (a service instance of that degree of parallelism, Section 5.3); without it a
+ * level is r separate chunks of g GPUs (replicas). */
+#define TANGRAM_UNIT_GANG 0x80
+
+#define TANGRAM_MAX_POOLS 8
+
+/* return codes */
+#define TANGRAM_OK 0
+#define TANGRAM_EINVAL (-1)   /* null pointer, size out of range, bad pool description */
+#define TANGRAM_ENOMEM (-2)   /* device allocation failed in tangram_round_create        */
+#define TANGRAM_ECUDA (-3)    /* a CUDA runtime call failed; see tangram_last_cuda_error */
+
+/* per-scenario status words */
+#define TANGRAM_STATUS_OK 0
+#define TANGRAM_STATUS_BAD_ACTION 1   /* a record names no pool, has g = 0, no usable level, or
+                                         a GPU chunk size that is no power of two <= node size */
+#define TANGRAM_STATUS_UNSORTED 2     /* replay: arrivals not non-decreasing                   */
+#define TANGRAM_STATUS_WORKSPACE 4    /* a DP or heap did not fit the workspace; the scenario's
+                                         outputs are not valid                                 */
+
+typedef struct tangram_round tangram_round; /* opaque; owns only its device workspace */
+
+typedef struct {
+  int32_t type;      /* TANGRAM_POOL_*                                                    */
+  int32_t capacity;  /* cores | GPUs | tokens per window (or concurrent calls)            */
+  int32_t group;     /* CPU: cores per NUMA domain; GPU: GPUs per node (1,2,4,8);
+                        capacity must be a multiple of it; API: ignored                    */
+  int32_t window_us; /* API: quota period (usage refills at multiples of it); 0 = the limit
+                        is on concurrent usage.  Ignored for CPU and GPU pools.            */
+} tangram_pool_desc;
+
+typedef struct {
+  int32_t n_scenarios;  /* independent cluster scenarios per call, >= 1                    */
+  int32_t max_actions;  /* row stride of every per-action array, >= 1                      */
+  int32_t n_pools;      /* 1 .. TANGRAM_MAX_POOLS                                          */
+  int32_t depth;        /* levels tried for the first waiting action in the estimate
+                           (Algorithm 2); the paper evaluates with 2                       */
+  int64_t round_us;     /* replay: round period                                            */
+  int32_t max_rounds;   /* replay: rounds per call and rows of `occupancy`; 0 if unused    */
+  int32_t host_buffers; /* 0: tangram_actions / tangram_result hold DEVICE pointers;
+                           1: they hold HOST pointers and every call copies inputs in and
+                           results out on the given stream (pinned memory recommended)     */
+  int64_t workspace_bytes; /* scratch for large DP tables; 0 = default (1 GiB)             */
+  const tangram_pool_desc* pools; /* host array of n_pools entries, copied                 */
+} tangram_round_desc;
+
+/* Pending actions, structure of arrays, scenario-major: element (sc, i) of a per-action
+ * array is at [sc * max_actions + i]; the actions of a scenario are in queue (first-come
+ * first-served) order.  Caller-owned; read only. */
+typedef struct {
+  const uint8_t* pool;        /* index of the pool holding the action's key elastic resource */
+  const uint8_t* unit;        /* low 7 bits: g, units per multiplicity step; bit 7: GANG      */
+  const uint32_t* level_mask; /* bit r-1 set <=> the action may run with g*r units, r = 1..32 */
+  const int64_t* s_us;        /* duration model: T(r) = s + floor(p / r); both clamped to     */
+  const int64_t* p_us;        /*   [0, 2^40]                                                  */
+  const int64_t* arrival_us;  /* may be null (all 0).  Replay needs it, non-decreasing.       */
+  const int32_t* n_actions;   /* per scenario, 0 .. max_actions                               */
+  const uint8_t* gpu_busy;    /* may be null.  Per scenario, one byte per node of every GPU
+                                 pool (pools in index order, row stride = total nodes): bit b
+                                 set <=> GPU b of the node is occupied before the round       */
+} tangram_actions;
+
+/* Results, caller-owned, fully overwritten by a call (rows up to max_actions). */
+typedef struct {
+  int32_t* alloc_units;   /* units granted; 0 = not scheduled                                 */
+  int32_t* place_node;    /* GPU: node of the (first) chunk; CPU: NUMA domain of the lowest
+                             core; API: 0; -1 if not scheduled                                */
+  int32_t* place_off;     /* GPU: first GPU of the (first) chunk within the node; CPU: lowest
+                             core id; API: units of the pool consumed before the grant; -1    */
+  int64_t* act_us;        /* predicted completion time (queueing so far + execution), -1 if
+                             not scheduled; replay: completion - arrival                      */
+  int64_t* total_act_us;  /* per scenario: sum of act_us over scheduled actions               */
+  int32_t* n_selected;    /* per scenario                                                     */
+  int32_t* status;        /* per scenario, TANGRAM_STATUS_* bits                              */
+  int32_t* occupancy;     /* replay only, may be null: [scenario][round][pool] units in use
+                             after the round's scheduling; zero once the scenario drained     */
+  int32_t* rounds_used;   /* replay only, may be null: rounds until drained, else max_rounds  */
+} tangram_result;
+
+/* Validates the description, copies it, allocates all device workspace on the current CUDA
+ * device.  *out is set only on success. */
+int tangram_round_create(const tangram_round_desc* desc, tangram_round** out);
+
+/* One scheduling round at time now_us for every scenario, all pools empty except for
+ * `gpu_busy`, nothing executing (Algorithm 1 with an empty executing queue).
+ * Asynchronous on `cuda_stream` (a cudaStream_t, may be null for the default stream). */
+int tangram_schedule_batch(tangram_round* round, const tangram_actions* actions, int64_t now_us,
+                           tangram_result* result, void* cuda_stream);
+
+/* Replays each scenario's arrival trace: rounds at r * round_us, r = 0 .. max_rounds-1; each
+ * round releases finished actions, admits arrived ones, schedules as above with the running
+ * actions in the completion heap, and starts what was selected.  The whole loop runs on the
+ * device.  Asynchronous on `cuda_stream`. */
+int tangram_replay_trace(tangram_round* round, const tangram_actions* actions,
+                         tangram_result* result, void* cuda_stream);
+
+/* Frees the workspace.  The caller must have synchronised the streams it used. */
+void tangram_round_destroy(tangram_round* round);
+
+/* Launches of this library's kernels since the round was created (for accounting). */
+int64_t tangram_kernel_launches(const tangram_round* round);
+
+const char* tangram_strerror(int code);
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char* tangram_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TANGRAM_H_ */

@@ -1,0 +1,224 @@
+"""ctypes binding of libtangram.so: the same calls as include/tangram.h, with torch tensors
+(device memory, or pinned host memory in host-buffer mode) marshalled to raw pointers.
+
+There is no fallback: without the compiled CUDA library every call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Dict, Optional, Sequence
+
+POOL_CPU, POOL_GPU, POOL_API = 0, 1, 2
+UNIT_GANG = 0x80
+STATUS_OK, STATUS_BAD_ACTION, STATUS_UNSORTED, STATUS_WORKSPACE = 0, 1, 2, 4
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libtangram.so")
+_lib = None
+
+
+class TangramError(RuntimeError):
+    pass
+
+
+class _PoolDesc(C.Structure):
+    _fields_ = [("type", C.c_int32), ("capacity", C.c_int32), ("group", C.c_int32), ("window_us", C.c_int32)]
+
+
+class _RoundDesc(C.Structure):
+    _fields_ = [("n_scenarios", C.c_int32), ("max_actions", C.c_int32), ("n_pools", C.c_int32),
+                ("depth", C.c_int32), ("round_us", C.c_int64), ("max_rounds", C.c_int32),
+                ("host_buffers", C.c_int32), ("workspace_bytes", C.c_int64), ("pools", C.POINTER(_PoolDesc))]
+
+
+class _Actions(C.Structure):
+    _fields_ = [("pool", C.c_void_p), ("unit", C.c_void_p), ("level_mask", C.c_void_p), ("s_us", C.c_void_p),
+                ("p_us", C.c_void_p), ("arrival_us", C.c_void_p), ("n_actions", C.c_void_p),
+                ("gpu_busy", C.c_void_p)]
+
+
+class _Result(C.Structure):
+    _fields_ = [("alloc_units", C.c_void_p), ("place_node", C.c_void_p), ("place_off", C.c_void_p),
+                ("act_us", C.c_void_p), ("total_act_us", C.c_void_p), ("n_selected", C.c_void_p),
+                ("status", C.c_void_p), ("occupancy", C.c_void_p), ("rounds_used", C.c_void_p)]
+
+
+EXPORTS = ("tangram_round_create", "tangram_schedule_batch", "tangram_replay_trace",
+           "tangram_round_destroy", "tangram_kernel_launches", "tangram_strerror",
+           "tangram_last_cuda_error")
+
+
+def load_library(path: Optional[str] = None):
+    """dlopen the CUDA library (built in-tree by paper_2603_13019_b200.build)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _LIB_PATH
+    if not os.path.exists(p):
+        raise TangramError(f"{p} is missing: build it with `python -m paper_2603_13019_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = C.CDLL(p)
+    lib.tangram_round_create.restype = C.c_int
+    lib.tangram_round_create.argtypes = [C.POINTER(_RoundDesc), C.POINTER(C.c_void_p)]
+    lib.tangram_schedule_batch.restype = C.c_int
+    lib.tangram_schedule_batch.argtypes = [C.c_void_p, C.POINTER(_Actions), C.c_int64, C.POINTER(_Result), C.c_void_p]
+    lib.tangram_replay_trace.restype = C.c_int
+    lib.tangram_replay_trace.argtypes = [C.c_void_p, C.POINTER(_Actions), C.POINTER(_Result), C.c_void_p]
+    lib.tangram_round_destroy.restype = None
+    lib.tangram_round_destroy.argtypes = [C.c_void_p]
+    lib.tangram_kernel_launches.restype = C.c_int64
+    lib.tangram_kernel_launches.argtypes = [C.c_void_p]
+    lib.tangram_strerror.restype = C.c_char_p
+    lib.tangram_strerror.argtypes = [C.c_int]
+    lib.tangram_last_cuda_error.restype = C.c_char_p
+    if path is None:
+        _lib = lib
+    return lib
+
+
+@dataclass(frozen=True)
+class PoolDesc:
+    type: int
+    capacity: int
+    group: int
+    window_us: int = 0
+
+
+def _dtypes():
+    import torch
+    ins = dict(pool=torch.uint8, unit=torch.uint8, level_mask=torch.int32, s_us=torch.int64,
+               p_us=torch.int64, arrival_us=torch.int64, n_actions=torch.int32, gpu_busy=torch.uint8)
+    outs = dict(alloc_units=torch.int32, place_node=torch.int32, place_off=torch.int32,
+                act_us=torch.int64, total_act_us=torch.int64, n_selected=torch.int32,
+                status=torch.int32, occupancy=torch.int32, rounds_used=torch.int32)
+    return ins, outs
+
+
+def _check(rc: int):
+    if rc != 0:
+        lib = load_library()
+        msg = lib.tangram_strerror(rc).decode()
+        detail = lib.tangram_last_cuda_error().decode()
+        raise TangramError(f"tangram call failed: {msg}" + (f" ({detail})" if detail else ""))
+
+
+class Round:
+    """Owner of a tangram_round handle (device workspace)."""
+
+    def __init__(self, n_scenarios: int, max_actions: int, pools: Sequence, *, depth: int = 2,
+                 round_us: int = 10_000, max_rounds: int = 0, host_buffers: bool = False,
+                 workspace_bytes: int = 0):
+        self._lib = load_library()
+        self._h = None
+        self.n_scenarios, self.max_actions, self.pools = int(n_scenarios), int(max_actions), tuple(pools)
+        self.max_rounds, self.host_buffers = int(max_rounds), bool(host_buffers)
+        arr = (_PoolDesc * len(pools))(*[_PoolDesc(p.type, p.capacity, p.group, p.window_us) for p in pools])
+        desc = _RoundDesc(n_scenarios, max_actions, len(pools), depth, round_us, max_rounds,
+                          1 if host_buffers else 0, workspace_bytes, arr)
+        h = C.c_void_p()
+        _check(self._lib.tangram_round_create(C.byref(desc), C.byref(h)))
+        self._h = h
+
+    # -- marshalling ---------------------------------------------------------------
+    def _ptr(self, name: str, t, dtype, numel: Optional[int]):
+        if t is None:
+            return None
+        if t.dtype != dtype:
+            raise TangramError(f"{name}: expected {dtype}, got {t.dtype}")
+        if not t.is_contiguous():
+            raise TangramError(f"{name}: tensor must be contiguous")
+        if self.host_buffers == t.is_cuda:
+            raise TangramError(f"{name}: tensor must be on the {'host' if self.host_buffers else 'device'}")
+        if numel is not None and t.numel() != numel:
+            raise TangramError(f"{name}: expected {numel} elements, got {t.numel()}")
+        return t.data_ptr()
+
+    def _actions(self, a: Dict) -> _Actions:
+        ins, _ = _dtypes()
+        SN = self.n_scenarios * self.max_actions
+        nodes = sum(p.capacity // p.group for p in self.pools if p.type == POOL_GPU)
+        sizes = dict(pool=SN, unit=SN, level_mask=SN, s_us=SN, p_us=SN, arrival_us=SN,
+                     n_actions=self.n_scenarios, gpu_busy=self.n_scenarios * nodes)
+        return _Actions(*[self._ptr(k, a.get(k), ins[k], sizes[k]) for k in
+                          ("pool", "unit", "level_mask", "s_us", "p_us", "arrival_us", "n_actions", "gpu_busy")])
+
+    def new_result(self, replay: bool = False) -> Dict:
+        """Output tensors of the right shapes (device, or pinned host in host-buffer mode)."""
+        import torch
+        _, outs = _dtypes()
+        S, N = self.n_scenarios, self.max_actions
+        kw = dict(pin_memory=True) if self.host_buffers else dict(device="cuda")
+        shapes = dict(alloc_units=(S, N), place_node=(S, N), place_off=(S, N), act_us=(S, N),
+                      total_act_us=(S,), n_selected=(S,), status=(S,))
+        if replay:
+            shapes.update(occupancy=(S, self.max_rounds, len(self.pools)), rounds_used=(S,))
+        return {k: torch.empty(shp, dtype=outs[k], **kw) for k, shp in shapes.items()}
+
+    def _result(self, r: Dict) -> _Result:
+        _, outs = _dtypes()
+        S, N = self.n_scenarios, self.max_actions
+        sizes = dict(alloc_units=S * N, place_node=S * N, place_off=S * N, act_us=S * N, total_act_us=S,
+                     n_selected=S, status=S, occupancy=S * self.max_rounds * len(self.pools), rounds_used=S)
+        return _Result(*[self._ptr(k, r.get(k), outs[k], sizes[k]) for k in
+                         ("alloc_units", "place_node", "place_off", "act_us", "total_act_us", "n_selected",
+                          "status", "occupancy", "rounds_used")])
+
+    @staticmethod
+    def _stream(stream) -> int:
+        import torch
+        if stream is None:
+            stream = torch.cuda.current_stream()
+        return int(stream.cuda_stream)
+
+    # -- the calls --------------------------------------------------------------------
+    def schedule_batch(self, actions: Dict, now_us: int = 0, result: Optional[Dict] = None, stream=None) -> Dict:
+        """tangram_schedule_batch: one round for every scenario, asynchronous on `stream`."""
+        result = self.new_result() if result is None else result
+        a, r = self._actions(actions), self._result(result)
+        _check(self._lib.tangram_schedule_batch(self._h, C.byref(a), int(now_us), C.byref(r), self._stream(stream)))
+        return result
+
+    def replay_trace(self, actions: Dict, result: Optional[Dict] = None, stream=None) -> Dict:
+        """tangram_replay_trace: device-resident replay of every scenario's arrival trace."""
+        result = self.new_result(replay=True) if result is None else result
+        a, r = self._actions(actions), self._result(result)
+        _check(self._lib.tangram_replay_trace(self._h, C.byref(a), C.byref(r), self._stream(stream)))
+        return result
+
+    @property
+    def kernel_launches(self) -> int:
+        return int(self._lib.tangram_kernel_launches(self._h))
+
+    def destroy(self):
+        if getattr(self, "_h", None):
+            self._lib.tangram_round_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def round_create(n_scenarios: int, max_actions: int, pools: Sequence, **kw) -> Round:
+    """tangram_round_create."""
+    return Round(n_scenarios, max_actions, pools, **kw)
+
+
+def to_device(arrays: Dict, device: str = "cuda", pin: bool = False) -> Dict:
+    """numpy input arrays -> torch tensors (device memory, or pinned host memory)."""
+    import numpy as np
+    import torch
+    out = {}
+    for k, v in arrays.items():
+        if v is None:
+            out[k] = None
+            continue
+        if v.dtype == np.uint32:
+            v = v.view(np.int32)
+        t = torch.from_numpy(np.ascontiguousarray(v))
+        out[k] = t.pin_memory() if pin else t.to(device)
+    return out

@@ -1,0 +1,143 @@
+// Shared device-side definitions of the scheduling-round kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef long long i64;
+typedef unsigned long long u64;
+typedef unsigned int u32;
+typedef unsigned char u8;
+
+#define TG_INF 0x7fffffffffffffffLL
+#define TG_PARAM_MAX (1LL << 40)
+#define TG_MAX_POOLS 8
+#define TG_POOL_CPU 0
+#define TG_POOL_GPU 1
+#define TG_POOL_API 2
+#define TG_ST_BAD_ACTION 1
+#define TG_ST_UNSORTED 2
+#define TG_ST_WORKSPACE 4
+#define TG_FULL 0xffffffffu
+
+struct PoolDev {
+  int type, capacity, group, window_us;
+  int node0, n_nodes;   // GPU pools: first node in a gpu_busy row, node count
+  int slot0, n_slots;   // demand slots in the prefix scan (GPU: 4 nested levels, else 1)
+};
+
+// per (scenario, pool) facts produced by the prefix kernel
+struct PoolMeta {
+  int base;       // first position of the pool in the scenario's partitioned arrays
+  int count;      // actions of the pool in the queue
+  int m;          // candidates of the pool (they occupy positions base .. base+m-1)
+  int elastic;    // some candidate has more than one level
+};
+
+struct Params {
+  int S, N, P, depth, n_nodes_total, V;
+  PoolDev pool[TG_MAX_POOLS];
+  i64 now;
+  // inputs (device)
+  const u8* a_pool; const u8* a_unit; const u32* a_mask;
+  const i64* a_s; const i64* a_p; const i64* a_arrival;
+  const int* n_actions; const u8* gpu_busy;
+  // outputs (device)
+  int* o_alloc; int* o_node; int* o_off; i64* o_act; i64* o_total; int* o_nsel; int* o_status;
+  // workspace
+  int* order;        // [S][N] action index at each partitioned position
+  i64* tmin;         // [S][N] duration at the least level, partitioned order
+  PoolMeta* meta;    // [S][P]
+  char* slabs; u64 slab_bytes; int n_workers;
+  char* arena; u64 arena_bytes; u64* arena_top;
+};
+
+// ceil(2^64 / r) for r = 2..32: floor(p / r) == umul64hi(p, c_recip[r]) for 0 <= p <= 2^40,
+// because the rounding excess p * (r - 2^64 mod r) / (r * 2^64) stays below 2^-24 < 1/r.
+__constant__ u64 c_recip[33];
+// maximal free aligned blocks of a node, indexed by its busy mask: byte l = blocks of size 2^l
+__constant__ u32 c_fblocks[256];
+
+__device__ __forceinline__ i64 div_small(i64 p, int r) {
+  return r == 1 ? p : (i64)__umul64hi((u64)p, c_recip[r]);
+}
+__device__ __forceinline__ i64 clamp_param(i64 v) { return v < 0 ? 0 : (v > TG_PARAM_MAX ? TG_PARAM_MAX : v); }
+__device__ __forceinline__ i64 sat_add(i64 a, i64 b) {   // a, b >= 0
+  u64 c = (u64)a + (u64)b;
+  return c > (u64)TG_INF ? TG_INF : (i64)c;
+}
+__device__ __forceinline__ int ilog2(int v) { return 31 - __clz(v); }
+
+struct Act {
+  i64 s, p;
+  u32 mask;   // usable multiplicities: bit r-1
+  int g, gang;
+};
+
+// Usable levels of a record on its pool.  Returns false for records no pool can serve.
+__device__ __forceinline__ bool decode_levels(const PoolDev& pd, u8 unit, u32 mask, int& g, int& gang, u32& eff) {
+  g = unit & 0x7f;
+  gang = (unit >> 7) && pd.type == TG_POOL_GPU;
+  eff = 0;
+  if (g == 0) return false;
+  if (pd.type == TG_POOL_GPU) {
+    bool p2 = (g & (g - 1)) == 0;
+    if (gang) {
+      u32 ok = 0;
+      if (p2) {
+        if (g <= pd.group) ok |= 1u;
+        if (2 * g <= pd.group) ok |= 2u;
+        if (4 * g <= pd.group) ok |= 8u;
+        if (8 * g <= pd.group) ok |= 128u;
+      }
+      mask &= ok;
+    } else if (!(p2 && g <= pd.group)) return false;
+  }
+  eff = mask;
+  return mask != 0;
+}
+
+// Duration at multiplicity r (Eq. 1 in integer microseconds): s + floor(p / r)
+__device__ __forceinline__ i64 duration(i64 s, i64 p, int r) { return s + div_small(p, r); }
+
+// Chunk-size level that a grant of multiplicity r asks for
+__device__ __forceinline__ int level_of(int g, int gang, int r) { return ilog2(gang ? g * r : g); }
+
+__device__ __forceinline__ i64 warp_min64(i64 v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) { i64 t = __shfl_xor_sync(TG_FULL, v, o); v = t < v ? t : v; }
+  return v;
+}
+__device__ __forceinline__ i64 warp_sum64(i64 v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(TG_FULL, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_sum32(int v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(TG_FULL, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_min32(int v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v = min(v, __shfl_xor_sync(TG_FULL, v, o));
+  return v;
+}
+__device__ __forceinline__ int warp_max32(int v) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) v = max(v, __shfl_xor_sync(TG_FULL, v, o));
+  return v;
+}
+
+// Free capacity per chunk level of a GPU pool: cap[l] = GPUs held in maximal free aligned
+// blocks of size >= 2^l.  `busy` may be null (all free).  Warp-cooperative.
+__device__ __forceinline__ void gpu_caps(const PoolDev& pd, const u8* busy, int lane, int cap[4]) {
+  int F0 = 0, F1 = 0, F2 = 0, F3 = 0;
+  u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;   // GPUs beyond the node size count as busy
+  for (int v = lane; v < pd.n_nodes; v += 32) {
+    u32 b = (busy ? busy[pd.node0 + v] : 0u) | pad;
+    u32 f = c_fblocks[b & 0xffu];
+    F0 += f & 0xff; F1 += (f >> 8) & 0xff; F2 += (f >> 16) & 0xff; F3 += f >> 24;
+  }
+  F0 = warp_sum32(F0); F1 = warp_sum32(F1); F2 = warp_sum32(F2); F3 = warp_sum32(F3);
+  cap[3] = F3 * 8; cap[2] = cap[3] + F2 * 4; cap[1] = cap[2] + F1 * 2; cap[0] = cap[1] + F0;
+}

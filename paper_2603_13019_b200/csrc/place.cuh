@@ -1,0 +1,89 @@
+// Placement of what a pool's selection granted, one warp per (scenario, pool).
+//   GPU pools (Section 5.3): chunks are aligned power-of-two intervals inside a node; requests
+//     are served by size descending, then queue position; each takes the smallest sufficient
+//     maximal free block, lowest (node, start) first, and the low end of a split block.
+//   CPU pools (Section 5.2): cores are exclusive; an action's cores come from one NUMA domain
+//     when one fits (fewest free cores that still fit, lowest index), lowest core ids first;
+//     otherwise domains are filled in ascending order.
+//   API pools (Section 5.1): the grant is accounted against the quota / concurrency limit.
+#pragma once
+#include "common.cuh"
+
+// lowest start of a maximal free aligned block of size 2^bl in a node mask, or -1
+__device__ __forceinline__ int find_block(u32 busy, int bl, int group) {
+  const int bs = 1 << bl;
+  const u32 ones = (1u << bs) - 1u;
+  for (int st = 0; st < group; st += bs) {
+    if (busy & (ones << st)) continue;
+    if (bs < 8) {                                       // maximal: the enclosing block is not free
+      int ps = st & ~(2 * bs - 1);
+      u32 pones = ((1u << (2 * bs)) - 1u) << ps;
+      if (!(busy & pones)) continue;
+    }
+    return st;
+  }
+  return -1;
+}
+
+// nm: node busy masks of the pool (updated).  keep candidates, multiplicities r[].
+__device__ void place_gpu(const PoolDev& pd, u8* nm, int keep, const u8* cg, const u8* r,
+                          int* pnode, int* poff, int lane) {
+  const int top = ilog2(pd.group);
+  const u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;
+  for (int lz = top; lz >= 0; --lz) {
+    const int z = 1 << lz;
+    for (int i = 0; i < keep; ++i) {
+      const int g = cg[i] & 0x7f, gang = cg[i] >> 7, ri = r[i];
+      const int nreq = gang ? (g * ri == z ? 1 : 0) : (g == z ? ri : 0);
+      for (int rep = 0; rep < nreq; ++rep) {
+        int node = -1, start = -1;
+        for (int bl = lz; bl <= top && node < 0; ++bl) {
+          for (int v0 = 0; v0 < pd.n_nodes; v0 += 32) {
+            int v = v0 + lane;
+            bool has = v < pd.n_nodes && ((c_fblocks[nm[v] | pad] >> (8 * bl)) & 0xffu) != 0;
+            u32 b = __ballot_sync(TG_FULL, has);
+            if (b) { node = v0 + __ffs(b) - 1; start = find_block(nm[node] | pad, bl, pd.group); break; }
+          }
+        }
+        if (node < 0 || start < 0) continue;            // cannot happen: the selection fits
+        __syncwarp();
+        if (lane == 0) {
+          nm[node] |= (u8)(((1u << z) - 1u) << start);
+          if (rep == 0) { pnode[i] = node; poff[i] = start; }
+        }
+        __syncwarp();
+      }
+    }
+  }
+}
+
+// busy: one bit per core (word array); dfree: free cores per domain.  Both updated.
+__device__ void place_cpu(const PoolDev& pd, u32* busy, int* dfree, int keep, const u8* cg,
+                          const u8* r, int* pnode, int* poff, int lane) {
+  const int D = pd.capacity / pd.group;
+  for (int i = 0; i < keep; ++i) {
+    const int k = (cg[i] & 0x7f) * r[i];
+    i64 key = TG_INF;
+    for (int d = lane; d < D; d += 32) {
+      int f = dfree[d];
+      if (f >= k) key = min(key, ((i64)f << 32) | d);
+    }
+    key = warp_min64(key);
+    if (lane == 0) {
+      int lo = 0, hi = pd.capacity;
+      if (key != TG_INF) { int d = (int)(key & 0xffffffff); lo = d * pd.group; hi = lo + pd.group; }
+      int need = k, first = -1;
+      for (int c = lo; c < hi && need > 0; ++c) {
+        u32 w = busy[c >> 5];
+        if (w == 0xffffffffu && (c & 31) == 0 && c + 32 <= hi) { c += 31; continue; }
+        if (w >> (c & 31) & 1u) continue;
+        busy[c >> 5] = w | (1u << (c & 31));
+        dfree[c / pd.group] -= 1;
+        if (first < 0) first = c;
+        --need;
+      }
+      pnode[i] = first >= 0 ? first / pd.group : -1; poff[i] = first;
+    }
+    __syncwarp();
+  }
+}

@@ -1,0 +1,347 @@
+// Per-pool selection of a round, executed by one warp per (scenario, pool):
+//   optimal discrete allocation of a candidate prefix (DPArrange, Algorithms 3 and 4),
+//   completion-heap estimate of what keeps waiting (Algorithm 2), greedy eviction
+//   (Algorithm 1, lines 8-14).
+//
+// The DP runs in "extra demand over everybody's least level" coordinates: a cell is the
+// vector e = (e_1, e_2, e_4, e_8) of GPUs requested at chunk sizes >= 1, 2, 4, 8 beyond the
+// least-level requests (for core / quota pools only e_1 = extra units exists).  A cell is
+// feasible iff e_l <= free capacity at that level minus the least-level demand, so the
+// feasible cells form a box; a level whose capacity equals the next smaller level's is
+// implied by it and dropped from the box.  Two certificates skip the DP altogether:
+// every candidate's best level fits (then each takes the smallest level reaching its lowest
+// duration), or no spare unit exists (then everybody keeps the least level).
+// Ties follow the canonical order: lowest duration sum, then fewest units, then
+// (k_m, ..., k_1) lexicographically smallest.
+#pragma once
+#include "common.cuh"
+
+struct Slab {
+  char* base; u64 cap; u64 used;
+  __device__ __forceinline__ void* take(u64 bytes) {
+    bytes = (bytes + 15) & ~(u64)15;
+    if (used + bytes > cap) return nullptr;
+    void* p = base + used; used += bytes; return p;
+  }
+};
+
+// warp-uniform bump allocation from the shared arena (large DP tables only)
+__device__ __forceinline__ void* arena_take(const Params& P, u64 bytes, int lane) {
+  bytes = (bytes + 255) & ~(u64)255;
+  u64 off = 0;
+  if (lane == 0) off = atomicAdd(P.arena_top, bytes);
+  off = __shfl_sync(TG_FULL, off, 0);
+  if (off + bytes > P.arena_bytes) return nullptr;
+  return P.arena + off;
+}
+
+struct PoolTask {
+  // the pool
+  int type, group;
+  int cap[4];             // free capacity per chunk level (core / quota pools: cap[0] only)
+  // candidates of the pool in queue order
+  int m;
+  const i64* cs; const i64* cp; const u32* cmask; const u8* cg;
+  // what waits behind them on this pool: durations at the least level, and the first record
+  const i64* ac_tmin; int n_ac;
+  Act ac_first;
+  // completion times (relative to now) of what is running on the pool
+  const i64* seeds; int n_seeds;
+  int depth;
+  // results: multiplicity per candidate of the prefix under evaluation / of the accepted one
+  u8* rsel; u8* rkeep;
+  int* rowcand;           // scratch, m ints
+};
+
+// extra demand, per chunk level, of multiplicity r over the least multiplicity r0
+__device__ __forceinline__ void extra_demand(int type, int g, int gang, int r0, int r, int d[4]) {
+  d[0] = d[1] = d[2] = d[3] = 0;
+  if (type != TG_POOL_GPU) { d[0] = g * (r - r0); return; }
+  if (gang) {
+    int z = g * r, z0 = g * r0, lz = ilog2(z), lz0 = ilog2(z0);
+#pragma unroll
+    for (int l = 0; l < 4; ++l) if (l <= lz) d[l] = z - (l <= lz0 ? z0 : 0);
+  } else {
+    int lz = ilog2(g);
+#pragma unroll
+    for (int l = 0; l < 4; ++l) if (l <= lz) d[l] = g * (r - r0);
+  }
+}
+
+// smallest multiplicity that already reaches the duration of the largest one
+__device__ __forceinline__ int best_level(i64 p, u32 mask) {
+  int rmax = 32 - __clz(mask);
+  i64 tb = div_small(p, rmax);
+  u32 mm = mask;
+  while (mm) {
+    int r = __ffs(mm); mm &= mm - 1;
+    if (div_small(p, r) == tb) return r;
+  }
+  return rmax;
+}
+
+// Optimal allocation of candidates [0, q) -> T.rsel[0..q), duration sum -> *opt.
+// Returns false if the workspace is too small.
+__device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab slab, int lane, i64* opt) {
+  const bool gpu = T.type == TG_POOL_GPU;
+  int dmin[4] = {0, 0, 0, 0}, dbest[4] = {0, 0, 0, 0};
+  i64 tmin_sum = 0, tbest_sum = 0;
+  for (int i = lane; i < q; i += 32) {
+    int g = T.cg[i] & 0x7f, gang = T.cg[i] >> 7;
+    u32 mk = T.cmask[i];
+    int r0 = __ffs(mk), rb = best_level(T.cp[i], mk);
+    int lz0 = gpu ? level_of(g, gang, r0) : 0, lzb = gpu ? level_of(g, gang, rb) : 0;
+#pragma unroll
+    for (int l = 0; l < 4; ++l) {
+      if (l <= lz0) dmin[l] += g * r0;
+      if (l <= lzb) dbest[l] += g * rb;
+    }
+    tmin_sum += duration(T.cs[i], T.cp[i], r0);
+    tbest_sum += duration(T.cs[i], T.cp[i], rb);
+  }
+  bool fits_best = true;
+  int Y[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    dmin[l] = warp_sum32(dmin[l]); dbest[l] = warp_sum32(dbest[l]);
+    Y[l] = T.cap[l] - dmin[l];
+    if (l == 0 || gpu) fits_best &= dbest[l] <= T.cap[l];
+  }
+  tmin_sum = warp_sum64(tmin_sum); tbest_sum = warp_sum64(tbest_sum);
+  if (fits_best) {
+    for (int i = lane; i < q; i += 32) T.rsel[i] = (u8)best_level(T.cp[i], T.cmask[i]);
+    __syncwarp();
+    *opt = tbest_sum;
+    return true;
+  }
+  if (Y[0] <= 0) {
+    for (int i = lane; i < q; i += 32) T.rsel[i] = (u8)__ffs(T.cmask[i]);
+    __syncwarp();
+    *opt = tmin_sum;
+    return true;
+  }
+
+  // ---- DP over the box of feasible extra-demand vectors
+  int nrows = 0;
+  int maxex[4] = {0, 0, 0, 0};
+  for (int i0 = 0; i0 < q; i0 += 32) {
+    int i = i0 + lane;
+    bool el = false;
+    if (i < q) {
+      u32 mk = T.cmask[i];
+      el = (mk & (mk - 1)) != 0;
+      T.rsel[i] = (u8)__ffs(mk);
+      if (el) {
+        int d[4];
+        extra_demand(T.type, T.cg[i] & 0x7f, T.cg[i] >> 7, __ffs(mk), 32 - __clz(mk), d);
+#pragma unroll
+        for (int l = 0; l < 4; ++l) maxex[l] += d[l];
+      }
+    }
+    u32 b = __ballot_sync(TG_FULL, el);
+    if (el) T.rowcand[nrows + __popc(b & ((1u << lane) - 1u))] = i;
+    nrows += __popc(b);
+  }
+  int ext[4], stride[4];
+  bool kept[4];
+  u64 cells = 1;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    maxex[l] = warp_sum32(maxex[l]);
+    kept[l] = l == 0 || (gpu && T.cap[l] < T.cap[l - 1]);
+    int bound = min(Y[l], maxex[l]);
+    ext[l] = kept[l] ? (max(bound, 0) >> l) + 1 : 1;
+    stride[l] = (int)cells;
+    cells *= (u64)ext[l];
+    if (cells > (1ull << 30)) return false;
+  }
+  const int ncell = (int)cells;
+  i64* val = (i64*)slab.take(2 * cells * sizeof(i64));
+  u8* choice = val ? (u8*)slab.take((u64)nrows * cells) : nullptr;
+  if (!choice) {
+    char* big = (char*)arena_take(P, 2 * cells * sizeof(i64) + (u64)nrows * cells, lane);
+    if (!big) return false;
+    val = (i64*)big; choice = (u8*)(big + 2 * cells * sizeof(i64));
+  }
+  i64* prev = val; i64* cur = val + cells;
+  for (int c = lane; c < ncell; c += 32) prev[c] = c == 0 ? 0 : TG_INF;
+  __syncwarp();
+  for (int t = 0; t < nrows; ++t) {
+    const int i = T.rowcand[t];
+    const int g = T.cg[i] & 0x7f, gang = T.cg[i] >> 7;
+    const u32 mk = T.cmask[i];
+    const int r0 = __ffs(mk);
+    const i64 s = T.cs[i], p = T.cp[i];
+    u8* ch = choice + (u64)t * cells;
+    for (int c = lane; c < ncell; c += 32) {
+      int e[4];
+#pragma unroll
+      for (int l = 0; l < 4; ++l) e[l] = (c / stride[l]) % ext[l];
+      i64 best = TG_INF; int bestr = 0;
+      u32 mm = mk;
+      while (mm) {
+        int r = __ffs(mm); mm &= mm - 1;
+        int d[4];
+        extra_demand(T.type, g, gang, r0, r, d);
+        int off = 0; bool ok = true;
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+          if (kept[l]) { int dl = d[l] >> l; ok &= dl <= e[l]; off += dl * stride[l]; }
+        if (!ok) continue;
+        i64 pv = prev[c - off];
+        if (pv == TG_INF) continue;
+        i64 cand = pv + duration(s, p, r);
+        if (cand < best) { best = cand; bestr = r; }
+      }
+      cur[c] = best; ch[c] = (u8)bestr;
+    }
+    __syncwarp();
+    i64* tmp = prev; prev = cur; cur = tmp;
+  }
+  // best cell of the last row: lowest value, then fewest extra units (e_1 = index along dim 0)
+  i64 bv = TG_INF;
+  for (int c = lane; c < ncell; c += 32) bv = min(bv, prev[c]);
+  bv = warp_min64(bv);
+  if (bv == TG_INF) return false;                    // cannot happen for an accommodated prefix
+  int be = INT_MAX;
+  for (int c = lane; c < ncell; c += 32) if (prev[c] == bv) be = min(be, c % ext[0]);
+  be = warp_min32(be);
+  int cnt = 0, bc = -1;
+  for (int c = lane; c < ncell; c += 32) if (prev[c] == bv && c % ext[0] == be) { ++cnt; bc = max(bc, c); }
+  cnt = warp_sum32(cnt); bc = warp_max32(bc);
+  int fail = 0;
+  if (lane == 0) {
+    if (cnt == 1) {
+      int c = bc;
+      for (int t = nrows - 1; t >= 0; --t) {
+        int i = T.rowcand[t];
+        int r = choice[(u64)t * cells + c];
+        T.rsel[i] = (u8)r;
+        int d[4];
+        extra_demand(T.type, T.cg[i] & 0x7f, T.cg[i] >> 7, __ffs(T.cmask[i]), r, d);
+#pragma unroll
+        for (int l = 0; l < 4; ++l) if (kept[l]) c -= (d[l] >> l) * stride[l];
+      }
+    } else {
+      // several end cells tie on value and units: walk back all of them at once, keeping at
+      // each task (latest first) the cells whose choice is the smallest
+      const int TIE_CAP = 64;
+      int lst[TIE_CAP], nl = 0;
+      for (int c = 0; c < ncell; ++c)
+        if (prev[c] == bv && c % ext[0] == be) { if (nl < TIE_CAP) lst[nl++] = c; else fail = 1; }
+      for (int t = nrows - 1; t >= 0; --t) {
+        int i = T.rowcand[t];
+        const u8* ch = choice + (u64)t * cells;
+        int rm = 255;
+        for (int x = 0; x < nl; ++x) rm = min(rm, (int)ch[lst[x]]);
+        T.rsel[i] = (u8)rm;
+        int d[4];
+        extra_demand(T.type, T.cg[i] & 0x7f, T.cg[i] >> 7, __ffs(T.cmask[i]), rm, d);
+        int off = 0;
+#pragma unroll
+        for (int l = 0; l < 4; ++l) if (kept[l]) off += (d[l] >> l) * stride[l];
+        int nn = 0;
+        for (int x = 0; x < nl; ++x) {
+          if (ch[lst[x]] != rm) continue;
+          int c = lst[x] - off;
+          bool dup = false;
+          for (int y = 0; y < nn; ++y) dup |= lst[y] == c;
+          if (!dup) lst[nn++] = c;
+        }
+        nl = nn;
+      }
+    }
+  }
+  fail = __shfl_sync(TG_FULL, fail, 0);
+  if (fail) return false;
+  __syncwarp();
+  i64 sum = 0;
+  for (int i = lane; i < q; i += 32) sum += duration(T.cs[i], T.cp[i], T.rsel[i]);
+  *opt = warp_sum64(sum);
+  return true;
+}
+
+// d-th smallest set bit (d = 0 is the lowest) as a multiplicity
+__device__ __forceinline__ int nth_level(u32 mask, int d) {
+  for (int k = 0; k < d; ++k) mask &= mask - 1;
+  return __ffs(mask);
+}
+
+// Completion-heap estimate (Algorithm 2, estimate) of everything that is not in the prefix
+// [0, q): evicted candidates first, then the pool's waiting actions.  Lane d simulates depth d+1.
+__device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab slab, int lane, i64* est) {
+  const int n_ev = T.m - q;
+  const int n_rest = n_ev + T.n_ac;
+  if (n_rest == 0) { *est = 0; return true; }
+  i64 fs, fp; u32 fm;
+  if (n_ev > 0) { fs = T.cs[q]; fp = T.cp[q]; fm = T.cmask[q]; }
+  else { fs = T.ac_first.s; fp = T.ac_first.p; fm = T.ac_first.mask; }
+  const int dmax = min(min(T.depth, __popc(fm)), 32);
+  const int H = T.n_seeds + q;
+  i64* heaps = (i64*)slab.take((u64)dmax * H * sizeof(i64));
+  if (!heaps) heaps = (i64*)arena_take(P, (u64)dmax * H * sizeof(i64), lane);
+  if (!heaps) return false;
+  for (int d = 0; d < dmax; ++d)
+    for (int i = lane; i < H; i += 32)
+      heaps[(u64)d * H + i] = i < T.n_seeds ? T.seeds[i]
+                                            : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], T.rsel[i - T.n_seeds]);
+  __syncwarp();
+  i64 tmp = TG_INF;
+  if (lane < dmax) {
+    i64* h = heaps + (u64)lane * H;
+    for (int st = H / 2 - 1; st >= 0; --st) {           // heapify
+      i64 v = h[st]; int pos = st;
+      for (;;) {
+        int c = 2 * pos + 1;
+        if (c >= H) break;
+        if (c + 1 < H && h[c + 1] < h[c]) ++c;
+        if (h[c] < v) { h[pos] = h[c]; pos = c; } else break;
+      }
+      h[pos] = v;
+    }
+    tmp = 0;
+    for (int e = 0; e < n_rest; ++e) {
+      i64 dur;
+      if (e == 0) dur = duration(fs, fp, nth_level(fm, lane));
+      else if (e < n_ev) dur = duration(T.cs[q + e], T.cp[q + e], __ffs(T.cmask[q + e]));
+      else dur = T.ac_tmin[e - n_ev];
+      i64 v = h[0] + dur;                                // pop the earliest completion, push ts + T
+      tmp = sat_add(tmp, v);
+      int pos = 0;
+      for (;;) {
+        int c = 2 * pos + 1;
+        if (c >= H) break;
+        i64 hc = h[c];
+        if (c + 1 < H) { i64 h2 = h[c + 1]; if (h2 < hc) { hc = h2; ++c; } }
+        if (hc < v) { h[pos] = hc; pos = c; } else break;
+      }
+      h[pos] = v;
+    }
+  }
+  __syncwarp();
+  *est = warp_min64(tmp);
+  return true;
+}
+
+// Greedy eviction (Algorithm 1, lines 8-14).  Returns the number of candidates kept (their
+// multiplicities in T.rkeep), or -1 if the workspace is too small.
+__device__ int evict_loop(const Params& P, const PoolTask& T, Slab slab, int lane) {
+  i64 opt, est;
+  if (!solve_prefix(P, T, T.m, slab, lane, &opt)) return -1;
+  if (!estimate_rest(P, T, T.m, slab, lane, &est)) return -1;
+  i64 obj = sat_add(opt, est);
+  int keep = T.m;
+  for (int i = lane; i < T.m; i += 32) T.rkeep[i] = T.rsel[i];
+  __syncwarp();
+  for (int t = 1; t <= T.m - 1; ++t) {
+    const int q = T.m - t;
+    if (!solve_prefix(P, T, q, slab, lane, &opt)) return -1;
+    if (!estimate_rest(P, T, q, slab, lane, &est)) return -1;
+    i64 nobj = sat_add(opt, est);
+    if (nobj >= obj) break;
+    obj = nobj; keep = q;
+    for (int i = lane; i < q; i += 32) T.rkeep[i] = T.rsel[i];
+    __syncwarp();
+  }
+  return keep;
+}

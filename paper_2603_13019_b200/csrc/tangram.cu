@@ -1,0 +1,350 @@
+// Host side of the C ABI declared in include/tangram.h, and the per-pool round kernel.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+#include <new>
+
+#include "../../include/tangram.h"
+#include "common.cuh"
+#include "prefix_kernel.cuh"
+#include "select.cuh"
+#include "place.cuh"
+
+#define K2_THREADS 256
+
+// ---------------------------------------------------------------------------------------
+// Kernel 2 of a round: one warp per (scenario, pool).  Loads the pool's candidates, runs the
+// all-inelastic shortcut (Algorithm 1, lines 5-6) or the eviction loop, places the grants
+// and writes the candidates' outputs (Eq. 2 for the predicted completion time).
+// ---------------------------------------------------------------------------------------
+__device__ void run_pool_task(const Params& P, int sc, int j, Slab slab, int lane) {
+  const PoolMeta mt = P.meta[(size_t)sc * P.P + j];
+  const int m = mt.m;
+  if (m == 0) return;
+  const PoolDev& pd = P.pool[j];
+  const size_t row = (size_t)sc * P.N;
+
+  i64* cs = (i64*)slab.take((u64)m * 8);
+  i64* cp = (i64*)slab.take((u64)m * 8);
+  u32* cmask = (u32*)slab.take((u64)m * 4);
+  int* cidx = (int*)slab.take((u64)m * 4);
+  int* pnode = (int*)slab.take((u64)m * 4);
+  int* poff = (int*)slab.take((u64)m * 4);
+  int* rowcand = (int*)slab.take((u64)m * 4);
+  u8* cg = (u8*)slab.take(m);
+  u8* rsel = (u8*)slab.take(m);
+  u8* rkeep = (u8*)slab.take(m);
+  if (!rkeep) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); return; }
+
+  for (int i = lane; i < m; i += 32) {
+    int idx = P.order[row + mt.base + i];
+    int g, gang; u32 eff;
+    decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], g, gang, eff);
+    cidx[i] = idx; cmask[i] = eff; cg[i] = (u8)(g | (gang << 7));
+    cs[i] = clamp_param(P.a_s[row + idx]); cp[i] = clamp_param(P.a_p[row + idx]);
+    rkeep[i] = (u8)__ffs(eff);
+    pnode[i] = -1; poff[i] = -1;
+  }
+  __syncwarp();
+
+  const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr;
+  int keep = m;
+  if (mt.elastic) {
+    PoolTask T;
+    T.type = pd.type; T.group = pd.group;
+    T.cap[0] = pd.capacity; T.cap[1] = T.cap[2] = T.cap[3] = 0;
+    if (pd.type == TG_POOL_GPU) gpu_caps(pd, busy_row, lane, T.cap);
+    T.m = m; T.cs = cs; T.cp = cp; T.cmask = cmask; T.cg = cg;
+    T.n_ac = mt.count - m;
+    T.ac_tmin = P.tmin + row + mt.base + m;
+    T.ac_first.s = T.ac_first.p = 0; T.ac_first.mask = 1; T.ac_first.g = 1; T.ac_first.gang = 0;
+    if (T.n_ac > 0) {
+      int idx = P.order[row + mt.base + m];
+      decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], T.ac_first.g, T.ac_first.gang, T.ac_first.mask);
+      T.ac_first.s = clamp_param(P.a_s[row + idx]); T.ac_first.p = clamp_param(P.a_p[row + idx]);
+    }
+    T.seeds = nullptr; T.n_seeds = 0;
+    T.depth = P.depth;
+    T.rsel = rsel; T.rkeep = rkeep; T.rowcand = rowcand;
+    keep = evict_loop(P, T, slab, lane);
+    if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+  }
+
+  // placement on a fresh copy of the pool's topology state
+  if (pd.type == TG_POOL_GPU) {
+    u8* nm = (u8*)slab.take(pd.n_nodes);
+    if (!nm) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+    else {
+      for (int v = lane; v < pd.n_nodes; v += 32) nm[v] = busy_row ? busy_row[pd.node0 + v] : 0;
+      __syncwarp();
+      place_gpu(pd, nm, keep, cg, rkeep, pnode, poff, lane);
+    }
+  } else if (pd.type == TG_POOL_CPU) {
+    const int D = pd.capacity / pd.group, W = (pd.capacity + 31) / 32;
+    u32* busy = (u32*)slab.take((u64)W * 4);
+    int* dfree = (int*)slab.take((u64)D * 4);
+    if (!dfree) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+    else {
+      for (int w = lane; w < W; w += 32) busy[w] = 0;
+      for (int d = lane; d < D; d += 32) dfree[d] = pd.group;
+      __syncwarp();
+      place_cpu(pd, busy, dfree, keep, cg, rkeep, pnode, poff, lane);
+    }
+  } else {
+    if (lane == 0) {
+      int used = 0;
+      for (int i = 0; i < keep; ++i) { pnode[i] = 0; poff[i] = used; used += (cg[i] & 0x7f) * rkeep[i]; }
+    }
+    __syncwarp();
+  }
+
+  i64 tot = 0; int cnt = 0;
+  for (int i = lane; i < m; i += 32) {
+    const size_t o = row + cidx[i];
+    if (i < keep) {
+      int r = rkeep[i];
+      i64 arr = P.a_arrival ? P.a_arrival[o] : 0;
+      i64 act = (P.now - arr) + duration(cs[i], cp[i], r);
+      P.o_alloc[o] = (cg[i] & 0x7f) * r; P.o_node[o] = pnode[i]; P.o_off[o] = poff[i]; P.o_act[o] = act;
+      tot += act; ++cnt;
+    } else {
+      P.o_alloc[o] = 0; P.o_node[o] = -1; P.o_off[o] = -1; P.o_act[o] = -1;
+    }
+  }
+  tot = warp_sum64(tot); cnt = warp_sum32(cnt);
+  if (lane == 0 && cnt) {
+    atomicAdd((u64*)&P.o_total[sc], (u64)tot);
+    atomicAdd(&P.o_nsel[sc], cnt);
+  }
+}
+
+__global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ Params P) {
+  const int lane = threadIdx.x & 31;
+  const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
+  const int nw = (gridDim.x * K2_THREADS) >> 5;
+  Slab slab;
+  slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
+  const int n_tasks = P.S * P.P;
+  for (int task = gw; task < n_tasks; task += nw) run_pool_task(P, task / P.P, task % P.P, slab, lane);
+}
+
+// ---------------------------------------------------------------------------------------
+// host
+// ---------------------------------------------------------------------------------------
+static thread_local char g_cuda_err[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+  return TANGRAM_ECUDA;
+}
+#define CK(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail(e_, #call); } while (0)
+
+struct tangram_round {
+  tangram_round_desc desc;
+  tangram_pool_desc pools[TANGRAM_MAX_POOLS];
+  Params P;                 // template: pools, sizes, workspace pointers
+  int device;
+  int64_t launches;
+  // workspace
+  void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
+  // staging for host-buffer mode
+  char* d_stage; size_t stage_bytes;
+  size_t in_off[8], out_off[9];
+};
+
+static cudaError_t fill_tables() {
+  u64 recip[33];
+  recip[0] = recip[1] = 0;
+  // ceil(2^64 / r) = floor((2^64 - 1) / r) + 1 for every r >= 2
+  for (int r = 2; r <= 32; ++r) recip[r] = 0xffffffffffffffffull / (u64)r + 1ull;
+  u32 fb[256];
+  for (int b = 0; b < 256; ++b) {
+    int F[4] = {0, 0, 0, 0};
+    // maximal free aligned blocks of an 8-GPU node with busy mask b
+    if (b == 0) F[3] = 1;
+    else
+      for (int h = 0; h < 8; h += 4) {
+        if (((b >> h) & 0xf) == 0) { F[2]++; continue; }
+        for (int q = h; q < h + 4; q += 2) {
+          if (((b >> q) & 0x3) == 0) { F[1]++; continue; }
+          for (int s = q; s < q + 2; ++s) if (!((b >> s) & 1)) F[0]++;
+        }
+      }
+    fb[b] = (u32)F[0] | ((u32)F[1] << 8) | ((u32)F[2] << 16) | ((u32)F[3] << 24);
+  }
+  cudaError_t e = cudaMemcpyToSymbol(c_recip, recip, sizeof(recip));
+  if (e == cudaSuccess) e = cudaMemcpyToSymbol(c_fblocks, fb, sizeof(fb));
+  return e;
+}
+
+extern "C" const char* tangram_strerror(int code) {
+  switch (code) {
+    case TANGRAM_OK: return "ok";
+    case TANGRAM_EINVAL: return "invalid argument";
+    case TANGRAM_ENOMEM: return "out of device memory";
+    case TANGRAM_ECUDA: return "CUDA runtime error";
+    default: return "unknown error";
+  }
+}
+
+extern "C" const char* tangram_last_cuda_error(void) { return g_cuda_err; }
+
+extern "C" int64_t tangram_kernel_launches(const tangram_round* r) { return r ? r->launches : 0; }
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_round** out) {
+  if (!desc || !out || !desc->pools) return TANGRAM_EINVAL;
+  if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
+      desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->max_rounds < 0 ||
+      desc->round_us < 0 || desc->workspace_bytes < 0)
+    return TANGRAM_EINVAL;
+  if ((int64_t)desc->n_scenarios * desc->max_actions > (int64_t)1 << 31) return TANGRAM_EINVAL;
+  tangram_round* r = new (std::nothrow) tangram_round();
+  if (!r) return TANGRAM_ENOMEM;
+  memset(r, 0, sizeof(*r));
+  r->desc = *desc;
+  Params& P = r->P;
+  P.S = desc->n_scenarios; P.N = desc->max_actions; P.P = desc->n_pools; P.depth = desc->depth;
+  int node0 = 0, slot0 = 0;
+  for (int j = 0; j < desc->n_pools; ++j) {
+    const tangram_pool_desc& pd = desc->pools[j];
+    r->pools[j] = pd;
+    bool ok = pd.capacity >= 1 && pd.capacity <= (1 << 20) && pd.window_us >= 0;
+    if (pd.type == TANGRAM_POOL_GPU)
+      ok = ok && (pd.group == 1 || pd.group == 2 || pd.group == 4 || pd.group == 8) && pd.capacity % pd.group == 0;
+    else if (pd.type == TANGRAM_POOL_CPU) ok = ok && pd.group >= 1 && pd.capacity % pd.group == 0;
+    else if (pd.type != TANGRAM_POOL_API) ok = false;
+    if (!ok) { delete r; return TANGRAM_EINVAL; }
+    PoolDev& d = P.pool[j];
+    d.type = pd.type; d.capacity = pd.capacity; d.group = pd.type == TANGRAM_POOL_API ? 1 : pd.group;
+    d.window_us = pd.type == TANGRAM_POOL_API ? pd.window_us : 0;
+    d.node0 = node0; d.n_nodes = pd.type == TANGRAM_POOL_GPU ? pd.capacity / pd.group : 0;
+    node0 += d.n_nodes;
+    d.slot0 = slot0; d.n_slots = pd.type == TANGRAM_POOL_GPU ? 4 : 1;
+    slot0 += d.n_slots;
+  }
+  r->desc.pools = r->pools;
+  P.n_nodes_total = node0;
+  P.V = slot0 + desc->n_pools;
+
+  cudaError_t e = cudaGetDevice(&r->device);
+  cudaDeviceProp prop;
+  if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, r->device);
+  if (e == cudaSuccess) e = fill_tables();
+  if (e != cudaSuccess) { delete r; return cuda_fail(e, "device set-up"); }
+
+  const size_t SN = (size_t)P.S * P.N;
+  P.n_workers = prop.multiProcessorCount * 4 * (K2_THREADS / 32);
+  if ((int64_t)P.n_workers > (int64_t)P.S * P.P) P.n_workers = (int)align_up((size_t)P.S * P.P, K2_THREADS / 32);
+  // every worker warp owns a slab that holds the candidate arrays, heaps and small DP tables of
+  // the pool it is working on; larger DP tables come from the shared arena
+  size_t per_cand = 8 + 8 + 4 + 4 + 4 + 4 + 4 + 3 + 16 * (size_t)desc->depth;
+  size_t slab = align_up((size_t)P.N * per_cand + 64 * 1024 + (1 << 20) / 4 + 4096, 256);
+  P.slab_bytes = slab;
+  P.arena_bytes = desc->workspace_bytes ? (u64)desc->workspace_bytes : (1ull << 30);
+  bool bad = false;
+  bad |= cudaMalloc(&r->d_order, SN * sizeof(int)) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_tmin, SN * sizeof(i64)) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_meta, (size_t)P.S * P.P * sizeof(PoolMeta)) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_slabs, (size_t)P.n_workers * slab) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_arena, P.arena_bytes) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_arena_top, 256) != cudaSuccess;
+  if (!bad && desc->host_buffers) {
+    size_t off = 0;
+    size_t in_sz[8] = {SN, SN, SN * 4, SN * 8, SN * 8, SN * 8, (size_t)P.S * 4, (size_t)P.S * (node0 ? node0 : 1)};
+    for (int k = 0; k < 8; ++k) { r->in_off[k] = off; off = align_up(off + in_sz[k], 256); }
+    size_t occ = (size_t)P.S * (desc->max_rounds > 0 ? desc->max_rounds : 0) * P.P * 4;
+    size_t out_sz[9] = {SN * 4, SN * 4, SN * 4, SN * 8, (size_t)P.S * 8, (size_t)P.S * 4, (size_t)P.S * 4,
+                        occ ? occ : 4, (size_t)P.S * 4};
+    for (int k = 0; k < 9; ++k) { r->out_off[k] = off; off = align_up(off + out_sz[k], 256); }
+    r->stage_bytes = off;
+    bad |= cudaMalloc((void**)&r->d_stage, off) != cudaSuccess;
+  }
+  if (bad) { cudaGetLastError(); tangram_round_destroy(r); return TANGRAM_ENOMEM; }
+  P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
+  P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
+  e = cudaFuncSetAttribute(k_prefix, cudaFuncAttributeMaxDynamicSharedMemorySize, P.V * K1_THREADS * 4);
+  if (e != cudaSuccess) { tangram_round_destroy(r); return cuda_fail(e, "cudaFuncSetAttribute"); }
+  *out = r;
+  return TANGRAM_OK;
+}
+
+extern "C" void tangram_round_destroy(tangram_round* r) {
+  if (!r) return;
+  cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
+  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage);
+  delete r;
+}
+
+// In host-buffer mode: copy the caller's arrays into the staging area and point P at it.
+static int stage_inputs(tangram_round* r, const tangram_actions* a, Params& P, cudaStream_t st) {
+  const size_t SN = (size_t)P.S * P.N;
+  char* d = r->d_stage;
+  const void* src[8] = {a->pool, a->unit, a->level_mask, a->s_us, a->p_us, a->arrival_us, a->n_actions, a->gpu_busy};
+  size_t sz[8] = {SN, SN, SN * 4, SN * 8, SN * 8, SN * 8, (size_t)P.S * 4, (size_t)P.S * P.n_nodes_total};
+  for (int k = 0; k < 8; ++k)
+    if (src[k] && sz[k]) CK(cudaMemcpyAsync(d + r->in_off[k], src[k], sz[k], cudaMemcpyHostToDevice, st));
+  P.a_pool = (const u8*)(d + r->in_off[0]); P.a_unit = (const u8*)(d + r->in_off[1]);
+  P.a_mask = (const u32*)(d + r->in_off[2]); P.a_s = (const i64*)(d + r->in_off[3]);
+  P.a_p = (const i64*)(d + r->in_off[4]);
+  P.a_arrival = a->arrival_us ? (const i64*)(d + r->in_off[5]) : nullptr;
+  P.n_actions = (const int*)(d + r->in_off[6]);
+  P.gpu_busy = (a->gpu_busy && P.n_nodes_total) ? (const u8*)(d + r->in_off[7]) : nullptr;
+  P.o_alloc = (int*)(d + r->out_off[0]); P.o_node = (int*)(d + r->out_off[1]); P.o_off = (int*)(d + r->out_off[2]);
+  P.o_act = (i64*)(d + r->out_off[3]); P.o_total = (i64*)(d + r->out_off[4]); P.o_nsel = (int*)(d + r->out_off[5]);
+  P.o_status = (int*)(d + r->out_off[6]);
+  return TANGRAM_OK;
+}
+
+static int unstage_outputs(tangram_round* r, const tangram_result* res, const Params& P, cudaStream_t st) {
+  const size_t SN = (size_t)P.S * P.N;
+  char* d = r->d_stage;
+  void* dst[7] = {res->alloc_units, res->place_node, res->place_off, res->act_us, res->total_act_us,
+                  res->n_selected, res->status};
+  size_t sz[7] = {SN * 4, SN * 4, SN * 4, SN * 8, (size_t)P.S * 8, (size_t)P.S * 4, (size_t)P.S * 4};
+  for (int k = 0; k < 7; ++k) CK(cudaMemcpyAsync(dst[k], d + r->out_off[k], sz[k], cudaMemcpyDeviceToHost, st));
+  return TANGRAM_OK;
+}
+
+static bool check_io(const tangram_actions* a, const tangram_result* res) {
+  return a && res && a->pool && a->unit && a->level_mask && a->s_us && a->p_us && a->n_actions &&
+         res->alloc_units && res->place_node && res->place_off && res->act_us && res->total_act_us &&
+         res->n_selected && res->status;
+}
+
+static void bind_device_io(Params& P, const tangram_actions* a, const tangram_result* res) {
+  P.a_pool = a->pool; P.a_unit = a->unit; P.a_mask = a->level_mask;
+  P.a_s = (const i64*)a->s_us; P.a_p = (const i64*)a->p_us; P.a_arrival = (const i64*)a->arrival_us;
+  P.n_actions = a->n_actions;
+  P.gpu_busy = P.n_nodes_total ? a->gpu_busy : nullptr;
+  P.o_alloc = res->alloc_units; P.o_node = res->place_node; P.o_off = res->place_off;
+  P.o_act = (i64*)res->act_us; P.o_total = (i64*)res->total_act_us;
+  P.o_nsel = res->n_selected; P.o_status = res->status;
+}
+
+extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a, int64_t now_us,
+                                      tangram_result* res, void* cuda_stream) {
+  if (!r || !check_io(a, res)) return TANGRAM_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Params P = r->P;
+  P.now = now_us;
+  if (r->desc.host_buffers) {
+    int rc = stage_inputs(r, a, P, st);
+    if (rc) return rc;
+  } else bind_device_io(P, a, res);
+  CK(cudaMemsetAsync(P.arena_top, 0, sizeof(u64), st));
+  k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
+  k_select<<<P.n_workers / (K2_THREADS / 32), K2_THREADS, 0, st>>>(P);
+  r->launches += 2;
+  CK(cudaGetLastError());
+  if (r->desc.host_buffers) return unstage_outputs(r, res, P, st);
+  return TANGRAM_OK;
+}
+
+extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, tangram_result* res,
+                                    void* cuda_stream) {
+  (void)r; (void)a; (void)res; (void)cuda_stream;
+  return TANGRAM_EINVAL;
+}

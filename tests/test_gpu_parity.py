@@ -1,0 +1,107 @@
+"""Parity of the CUDA path with the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+from workloads import POOL_API, POOL_CPU, POOL_GPU, Pool, generate, make_workload, random_round
+
+pytestmark = pytest.mark.gpu
+
+OUT_KEYS = ("status", "n_selected", "total_act_us", "alloc_units", "place_node", "place_off", "act_us")
+
+
+def gpu_round(pools, a, depth=2, now_us=0, host_buffers=False):
+    import torch
+    from paper_2603_13019_b200 import binding
+    S, N = a["pool"].shape
+    rnd = binding.Round(S, N, pools, depth=depth, host_buffers=host_buffers)
+    t = binding.to_device(a, pin=host_buffers)
+    out = rnd.schedule_batch(t, now_us=now_us)
+    torch.cuda.synchronize()
+    res = {k: v.cpu().numpy() for k, v in out.items()}
+    rnd.destroy()
+    return res
+
+
+def assert_same(o, g):
+    for k in OUT_KEYS:
+        if not np.array_equal(o[k], g[k]):
+            bad = np.argwhere(o[k] != g[k])
+            first = tuple(bad[0])
+            raise AssertionError(
+                f"{k} differs at {first}: oracle {o[k][first]} cuda {g[k][first]} ({len(bad)} mismatches)")
+
+
+@pytest.mark.parametrize("name,S", [("cfg0", 1), ("cfg1", 96), ("cfg3", 48), ("cfg4", 24)])
+def test_named_configs_match_oracle(oracle, name, S):
+    w = make_workload(name, n_scenarios=S)
+    a = generate(w)
+    o = oracle.schedule_batch(w.pools, a, depth=w.depth)
+    g = gpu_round(w.pools, a, depth=w.depth)
+    assert_same(o, g)
+    assert np.all(g["status"] == 0)
+
+
+POOLSETS = [
+    (Pool(POOL_CPU, 16, 4), Pool(POOL_GPU, 16, 8), Pool(POOL_API, 5, 0, 1_000_000)),
+    (Pool(POOL_GPU, 24, 8),),
+    (Pool(POOL_CPU, 40, 8), Pool(POOL_GPU, 8, 4)),
+    (Pool(POOL_CPU, 6, 2), Pool(POOL_API, 3, 0, 0)),
+    (Pool(POOL_CPU, 300, 64), Pool(POOL_GPU, 64, 8), Pool(POOL_GPU, 6, 2), Pool(POOL_API, 40, 0, 1000)),
+]
+
+
+@pytest.mark.parametrize("seed", range(15))
+def test_random_rounds_match_oracle(oracle, seed):
+    pools = POOLSETS[seed % len(POOLSETS)]
+    N = [40, 77, 300][seed % 3]
+    w, a = random_round(500 + seed, 64, N, pools, small_durations=0.4 if seed % 2 else 0.0,
+                        busy_fraction=0.3 if seed % 3 == 0 else 0.0, max_mult=[8, 4, 12][seed % 3])
+    for depth, now in ((2, 12345), (1, 0), (3, 7)):
+        o = oracle.schedule_batch(pools, a, depth=depth, now_us=now)
+        g = gpu_round(pools, a, depth=depth, now_us=now)
+        assert_same(o, g)
+
+
+def test_ties_everywhere_match_oracle(oracle):
+    # durations so small that many allocations tie on the duration sum
+    pools = (Pool(POOL_CPU, 12, 4), Pool(POOL_GPU, 16, 8))
+    w, a = random_round(901, 128, 24, pools, small_durations=1.0, busy_fraction=0.25, inelastic=0.1)
+    o = oracle.schedule_batch(pools, a)
+    g = gpu_round(pools, a)
+    assert_same(o, g)
+
+
+def test_edge_cases_match_oracle(oracle):
+    pools = (Pool(POOL_CPU, 8, 4), Pool(POOL_GPU, 8, 8))
+    w, a = random_round(77, 8, 16, pools)
+    a["n_actions"][:] = [0, 1, 16, 16, 3, 16, 16, 2]
+    a["level_mask"][3, 5] = 0                      # no usable level -> bad scenario
+    a["pool"][5, 0] = 7                            # unknown pool -> bad scenario
+    a["unit"][6, :] = 1                            # GPU actions become single-GPU replicas
+    a["s_us"][2, :] = -5                           # clamped to 0
+    a["p_us"][2, 0] = 1 << 50                      # clamped to 2^40
+    o = oracle.schedule_batch(pools, a)
+    g = gpu_round(pools, a)
+    assert_same(o, g)
+    assert list(g["status"][[3, 5]]) == [1, 1] and g["n_selected"][0] == 0
+
+
+def test_arrivals_and_host_buffers_match_oracle(oracle):
+    w = make_workload("cfg1", n_scenarios=16)
+    a = generate(w)
+    rng = np.random.default_rng(5)
+    a["arrival_us"] = np.sort(rng.integers(0, 50_000, a["pool"].shape), axis=1).astype(np.int64)
+    o = oracle.schedule_batch(w.pools, a, now_us=60_000)
+    assert_same(o, gpu_round(w.pools, a, now_us=60_000))
+    assert_same(o, gpu_round(w.pools, a, now_us=60_000, host_buffers=True))
+
+
+def test_long_queue_spans_several_tiles(oracle):
+    # 9000 actions per scenario: the prefix kernel walks three tiles with carried prefix sums
+    pools = (Pool(POOL_CPU, 3000, 64), Pool(POOL_GPU, 512, 8), Pool(POOL_API, 2000, 0, 1_000_000))
+    w, a = random_round(31, 6, 9000, pools, max_mult=4, ragged=False)
+    a["n_actions"][:] = [9000, 8191, 4097, 4096, 100, 9000]
+    o = oracle.schedule_batch(pools, a)
+    g = gpu_round(pools, a)
+    assert_same(o, g)
+    assert o["n_selected"].max() > 300
