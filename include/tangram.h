@@ -140,6 +140,16 @@ void tangram_round_destroy(tangram_round* round);
 /* Launches of this library's kernels since the round was created (for accounting). */
 int64_t tangram_kernel_launches(const tangram_round* round);
 
+/* Measurement aid (no counterpart in the paper).  tangram_set_profiling(round, 1) creates CUDA
+ * events once; from then on every call records events around each of its kernels on the
+ * call's stream (up to 256 calls between two switches).  After the caller has synchronised,
+ * tangram_kernel_time_ms sums device time and launches of kernel index `kernel`
+ * (0 .. 2, named by tangram_kernel_name) since profiling was last switched on;
+ * tangram_set_profiling(round, 0) destroys the events. */
+int tangram_set_profiling(tangram_round* round, int enable);
+int tangram_kernel_time_ms(tangram_round* round, int kernel, double* total_ms, int64_t* launches);
+const char* tangram_kernel_name(int kernel);
+
 const char* tangram_strerror(int code);
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char* tangram_last_cuda_error(void);

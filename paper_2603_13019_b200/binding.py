@@ -47,7 +47,8 @@ class _Result(C.Structure):
 
 EXPORTS = ("tangram_round_create", "tangram_schedule_batch", "tangram_replay_trace",
            "tangram_round_destroy", "tangram_kernel_launches", "tangram_strerror",
-           "tangram_last_cuda_error")
+           "tangram_last_cuda_error", "tangram_set_profiling", "tangram_kernel_time_ms",
+           "tangram_kernel_name")
 
 
 def load_library(path: Optional[str] = None):
@@ -73,6 +74,12 @@ def load_library(path: Optional[str] = None):
     lib.tangram_strerror.restype = C.c_char_p
     lib.tangram_strerror.argtypes = [C.c_int]
     lib.tangram_last_cuda_error.restype = C.c_char_p
+    lib.tangram_set_profiling.restype = C.c_int
+    lib.tangram_set_profiling.argtypes = [C.c_void_p, C.c_int]
+    lib.tangram_kernel_time_ms.restype = C.c_int
+    lib.tangram_kernel_time_ms.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.tangram_kernel_name.restype = C.c_char_p
+    lib.tangram_kernel_name.argtypes = [C.c_int]
     if path is None:
         _lib = lib
     return lib
@@ -186,6 +193,19 @@ class Round:
         a, r = self._actions(actions), self._result(result)
         _check(self._lib.tangram_replay_trace(self._h, C.byref(a), C.byref(r), self._stream(stream)))
         return result
+
+    def set_profiling(self, enable: bool):
+        """tangram_set_profiling: record CUDA events around every kernel of the following calls."""
+        _check(self._lib.tangram_set_profiling(self._h, 1 if enable else 0))
+
+    def kernel_times(self) -> Dict[str, tuple]:
+        """tangram_kernel_time_ms for every kernel: name -> (total ms, launches).  Synchronise first."""
+        out = {}
+        for k in range(3):
+            ms, n = C.c_double(0.0), C.c_int64(0)
+            _check(self._lib.tangram_kernel_time_ms(self._h, k, C.byref(ms), C.byref(n)))
+            out[self._lib.tangram_kernel_name(k).decode()] = (ms.value, n.value)
+        return out
 
     @property
     def kernel_launches(self) -> int:

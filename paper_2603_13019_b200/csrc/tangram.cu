@@ -12,6 +12,9 @@
 #include "place.cuh"
 
 #define K2_THREADS 256
+#define TG_PROF_CALLS 256   // calls whose kernels can be timed between two queries
+#define TG_PROF_K 2         // kernels per call at most
+#define TG_N_KERNELS 3
 
 // ---------------------------------------------------------------------------------------
 // Kernel 2 of a round: one warp per (scenario, pool).  Loads the pool's candidates, runs the
@@ -151,7 +154,11 @@ struct tangram_round {
   // staging for host-buffer mode
   char* d_stage; size_t stage_bytes;
   size_t in_off[8], out_off[9];
+  // optional per-kernel timing: events recorded around every kernel of a call
+  cudaEvent_t* ev; int ev_calls, ev_used; int ev_kernel[TG_PROF_CALLS][TG_PROF_K];
 };
+
+static const char* const g_kernel_names[TG_N_KERNELS] = {"k_prefix", "k_select", "k_replay"};
 
 static cudaError_t fill_tables() {
   u64 recip[33];
@@ -271,8 +278,59 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   return TANGRAM_OK;
 }
 
+extern "C" int tangram_set_profiling(tangram_round* r, int enable) {
+  if (!r) return TANGRAM_EINVAL;
+  if (enable && !r->ev) {
+    const int n = TG_PROF_CALLS * (TG_PROF_K + 1);
+    r->ev = new (std::nothrow) cudaEvent_t[n];
+    if (!r->ev) return TANGRAM_ENOMEM;
+    for (int i = 0; i < n; ++i) {
+      cudaError_t e = cudaEventCreate(&r->ev[i]);
+      if (e != cudaSuccess) {
+        for (int k = 0; k < i; ++k) cudaEventDestroy(r->ev[k]);
+        delete[] r->ev; r->ev = nullptr;
+        return cuda_fail(e, "cudaEventCreate");
+      }
+    }
+  }
+  if (!enable && r->ev) {
+    for (int i = 0; i < TG_PROF_CALLS * (TG_PROF_K + 1); ++i) cudaEventDestroy(r->ev[i]);
+    delete[] r->ev; r->ev = nullptr;
+  }
+  r->ev_used = 0;
+  return TANGRAM_OK;
+}
+
+extern "C" const char* tangram_kernel_name(int kernel) {
+  return kernel >= 0 && kernel < TG_N_KERNELS ? g_kernel_names[kernel] : "";
+}
+
+extern "C" int tangram_kernel_time_ms(tangram_round* r, int kernel, double* total_ms, int64_t* launches) {
+  if (!r || !total_ms || !launches || kernel < 0 || kernel >= TG_N_KERNELS) return TANGRAM_EINVAL;
+  *total_ms = 0.0; *launches = 0;
+  if (!r->ev) return TANGRAM_OK;
+  for (int c = 0; c < r->ev_used; ++c)
+    for (int k = 0; k < TG_PROF_K; ++k) {
+      if (r->ev_kernel[c][k] != kernel) continue;
+      float ms = 0.f;
+      cudaEvent_t* e = r->ev + c * (TG_PROF_K + 1);
+      CK(cudaEventElapsedTime(&ms, e[k], e[k + 1]));
+      *total_ms += ms; *launches += 1;
+    }
+  return TANGRAM_OK;
+}
+
+// events of the current call, or null when timing is off or the event pool is used up
+static cudaEvent_t* prof_begin(tangram_round* r, int k0, int k1) {
+  if (!r->ev || r->ev_used >= TG_PROF_CALLS) return nullptr;
+  int c = r->ev_used++;
+  r->ev_kernel[c][0] = k0; r->ev_kernel[c][1] = k1;
+  return r->ev + c * (TG_PROF_K + 1);
+}
+
 extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
+  if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
   cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage);
   delete r;
@@ -335,8 +393,12 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
     if (rc) return rc;
   } else bind_device_io(P, a, res);
   CK(cudaMemsetAsync(P.arena_top, 0, sizeof(u64), st));
+  cudaEvent_t* ev = prof_begin(r, 0, 1);
+  if (ev) CK(cudaEventRecord(ev[0], st));
   k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
+  if (ev) CK(cudaEventRecord(ev[1], st));
   k_select<<<P.n_workers / (K2_THREADS / 32), K2_THREADS, 0, st>>>(P);
+  if (ev) CK(cudaEventRecord(ev[2], st));
   r->launches += 2;
   CK(cudaGetLastError());
   if (r->desc.host_buffers) return unstage_outputs(r, res, P, st);

@@ -46,7 +46,7 @@ POOLSETS = [
     (Pool(POOL_GPU, 24, 8),),
     (Pool(POOL_CPU, 40, 8), Pool(POOL_GPU, 8, 4)),
     (Pool(POOL_CPU, 6, 2), Pool(POOL_API, 3, 0, 0)),
-    (Pool(POOL_CPU, 300, 64), Pool(POOL_GPU, 64, 8), Pool(POOL_GPU, 6, 2), Pool(POOL_API, 40, 0, 1000)),
+    (Pool(POOL_CPU, 320, 64), Pool(POOL_GPU, 64, 8), Pool(POOL_GPU, 6, 2), Pool(POOL_API, 40, 0, 1000)),
 ]
 
 
