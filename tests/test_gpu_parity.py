@@ -98,7 +98,7 @@ def test_arrivals_and_host_buffers_match_oracle(oracle):
 
 def test_long_queue_spans_several_tiles(oracle):
     # 9000 actions per scenario: the prefix kernel walks three tiles with carried prefix sums
-    pools = (Pool(POOL_CPU, 3000, 64), Pool(POOL_GPU, 512, 8), Pool(POOL_API, 2000, 0, 1_000_000))
+    pools = (Pool(POOL_CPU, 3008, 64), Pool(POOL_GPU, 512, 8), Pool(POOL_API, 2000, 0, 1_000_000))
     w, a = random_round(31, 6, 9000, pools, max_mult=4, ragged=False)
     a["n_actions"][:] = [9000, 8191, 4097, 4096, 100, 9000]
     o = oracle.schedule_batch(pools, a)
