@@ -49,6 +49,8 @@ extern "C" {
 #define TANGRAM_EINVAL (-1)   /* null pointer, size out of range, bad pool description */
 #define TANGRAM_ENOMEM (-2)   /* device allocation failed in tangram_round_create        */
 #define TANGRAM_ECUDA (-3)    /* a CUDA runtime call failed; see tangram_last_cuda_error */
+#define TANGRAM_ETOOBIG (-4)  /* tangram_schedule_batch_static: the batch needs more scratch than
+                                 the built-in array holds                                    */
 
 /* per-scenario status words */
 #define TANGRAM_STATUS_OK 0
@@ -133,6 +135,37 @@ int tangram_schedule_batch(tangram_round* round, const tangram_actions* actions,
  * device.  Asynchronous on `cuda_stream`. */
 int tangram_replay_trace(tangram_round* round, const tangram_actions* actions,
                          tangram_result* result, void* cuda_stream);
+
+/* The same round as tangram_schedule_batch for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside another framework's
+ * memory pool whose allocator must see every byte on the device, in a latency-critical loop
+ * where an allocation's implicit device synchronisation is not acceptable, or in a process
+ * whose device memory is fully reserved up front.  Such a caller has no tangram_round: it
+ * passes the description, its own DEVICE input and output buffers (host_buffers must be 0)
+ * and a stream, and the library calls neither cudaMalloc nor cudaFree nor any other
+ * allocating routine.
+ *
+ * All scratch lives in one array of TANGRAM_STATIC_SCRATCH_BYTES that is part of the library
+ * image: every GPU that loads the library holds those bytes until the process exits, whether
+ * or not this entry point is ever called.  A batch whose scratch does not fit is refused with
+ * TANGRAM_ETOOBIG and nothing is launched; roughly, 12 bytes per action of
+ * n_scenarios * max_actions plus eight worker areas of about 63 * max_actions + 330 KiB plus
+ * 4 MiB for large DP tables must fit.  At most 32 worker warps run, so this call is slower on
+ * big batches; results are identical.  A scenario whose DP tables outgrow what is left of the
+ * array is marked TANGRAM_STATUS_WORKSPACE in `status`, exactly as with a round whose
+ * workspace_bytes is too small; the other scenarios of the batch are unaffected.
+ *
+ * The first call on each device (with that device current) looks up the array's device
+ * address and loads two small constant tables; make that first call outside any stream
+ * capture.  Every call uses the same array and leaves its contents behind: two calls whose
+ * kernels can overlap on the GPU (different streams, or different host threads on one
+ * device) race on it and must be serialised by the caller; calls on one stream are safe.
+ * Asynchronous on `cuda_stream`. */
+#define TANGRAM_STATIC_SCRATCH_BYTES (32u << 20)
+int tangram_schedule_batch_static(const tangram_round_desc* desc, const tangram_actions* actions,
+                                  int64_t now_us, tangram_result* result, void* cuda_stream);
 
 /* Frees the workspace.  The caller must have synchronised the streams it used. */
 void tangram_round_destroy(tangram_round* round);

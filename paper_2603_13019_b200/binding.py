@@ -48,7 +48,7 @@ class _Result(C.Structure):
 EXPORTS = ("tangram_round_create", "tangram_schedule_batch", "tangram_replay_trace",
            "tangram_round_destroy", "tangram_kernel_launches", "tangram_strerror",
            "tangram_last_cuda_error", "tangram_set_profiling", "tangram_kernel_time_ms",
-           "tangram_kernel_name")
+           "tangram_kernel_name", "tangram_schedule_batch_static")
 
 
 def load_library(path: Optional[str] = None):
@@ -80,6 +80,9 @@ def load_library(path: Optional[str] = None):
     lib.tangram_kernel_time_ms.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.tangram_kernel_name.restype = C.c_char_p
     lib.tangram_kernel_name.argtypes = [C.c_int]
+    lib.tangram_schedule_batch_static.restype = C.c_int
+    lib.tangram_schedule_batch_static.argtypes = [C.POINTER(_RoundDesc), C.POINTER(_Actions), C.c_int64,
+                                                  C.POINTER(_Result), C.c_void_p]
     if path is None:
         _lib = lib
     return lib
@@ -242,3 +245,37 @@ def to_device(arrays: Dict, device: str = "cuda", pin: bool = False) -> Dict:
         t = torch.from_numpy(np.ascontiguousarray(v))
         out[k] = t.pin_memory() if pin else t.to(device)
     return out
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def schedule_batch_static(pools: Sequence, actions: Dict, result: Dict, *, depth: int = 2, now_us: int = 0,
+                          stream=None) -> int:
+    """tangram_schedule_batch_static: one round without a Round object and without any device
+    allocation by the library -- for callers that may not call cudaMalloc (their framework owns
+    all device memory, or an allocation's implicit synchronisation is unacceptable).  `actions`
+    and `result` are caller-owned DEVICE tensors shaped like those of Round.schedule_batch.
+    The library's scratch is a fixed 32 MiB array inside the library image, shared by all calls:
+    serialise calls that could overlap on the GPU, and make the first call on a device outside
+    stream capture.  Returns the C return code (0, or -4 when the batch is too large for the
+    array) instead of raising, so that callers can fall back to a Round."""
+    lib = load_library()
+    ins, outs = _dtypes()
+    S, N = actions["pool"].shape
+    arr = (_PoolDesc * len(pools))(*[_PoolDesc(p.type, p.capacity, p.group, p.window_us) for p in pools])
+    desc = _RoundDesc(S, N, len(pools), depth, 0, 0, 0, 0, arr)
+
+    def ptr(t):
+        return None if t is None else t.data_ptr()
+
+    for k, t in list(actions.items()) + list(result.items()):
+        if t is not None and not (t.is_cuda and t.is_contiguous()):
+            raise TangramError(f"{k}: a contiguous device tensor is required")
+    a = _Actions(*[ptr(actions.get(k)) for k in
+                   ("pool", "unit", "level_mask", "s_us", "p_us", "arrival_us", "n_actions", "gpu_busy")])
+    r = _Result(*[ptr(result.get(k)) for k in
+                  ("alloc_units", "place_node", "place_off", "act_us", "total_act_us", "n_selected", "status",
+                   "occupancy", "rounds_used")])
+    return int(lib.tangram_schedule_batch_static(C.byref(desc), C.byref(a), int(now_us), C.byref(r),
+                                                 Round._stream(stream)))

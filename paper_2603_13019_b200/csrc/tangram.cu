@@ -191,6 +191,7 @@ extern "C" const char* tangram_strerror(int code) {
     case TANGRAM_EINVAL: return "invalid argument";
     case TANGRAM_ENOMEM: return "out of device memory";
     case TANGRAM_ECUDA: return "CUDA runtime error";
+    case TANGRAM_ETOOBIG: return "problem too large for the static scratch array";
     default: return "unknown error";
   }
 }
@@ -409,4 +410,102 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
                                     void* cuda_stream) {
   (void)r; (void)a; (void)res; (void)cuda_stream;
   return TANGRAM_EINVAL;
+}
+
+
+// ---------------------------------------------------------------------------------------
+// tangram_schedule_batch_static: the same round for callers that must not allocate.
+// All scratch (partition order, least-level durations, per-pool facts, worker slabs, DP arena)
+// is carved out of one file-scope device array that every GPU loading this library holds
+// until the process exits.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[TANGRAM_STATIC_SCRATCH_BYTES];
+
+#define TG_MAX_DEVICES 64
+static unsigned char* g_static_ptr[TG_MAX_DEVICES];   // device address of the array, per device
+static bool g_static_ready[TG_MAX_DEVICES];
+
+// Once per device, with that device current: resolve the array's device address (its name is
+// only a host-side handle here and must not be handed to a kernel) and load the constant tables.
+static int static_setup(int* dev_out) {
+  int dev = -1;
+  CK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= TG_MAX_DEVICES) return TANGRAM_EINVAL;
+  if (!g_static_ready[dev]) {
+    unsigned char* ptr = nullptr;
+    CK(cudaGetSymbolAddress((void**)&ptr, g_static_scratch));
+    CK(fill_tables());
+    g_static_ptr[dev] = ptr;
+    g_static_ready[dev] = true;
+  }
+  *dev_out = dev;
+  return TANGRAM_OK;
+}
+
+extern "C" int tangram_schedule_batch_static(const tangram_round_desc* desc, const tangram_actions* a,
+                                             int64_t now_us, tangram_result* res, void* cuda_stream) {
+  if (!desc || !desc->pools || !check_io(a, res)) return TANGRAM_EINVAL;
+  if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
+      desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->host_buffers)
+    return TANGRAM_EINVAL;
+  if ((int64_t)desc->n_scenarios * desc->max_actions > (int64_t)1 << 31) return TANGRAM_ETOOBIG;
+  Params P;
+  memset(&P, 0, sizeof(P));
+  P.S = desc->n_scenarios; P.N = desc->max_actions; P.P = desc->n_pools; P.depth = desc->depth;
+  int node0 = 0, slot0 = 0;
+  for (int j = 0; j < desc->n_pools; ++j) {
+    const tangram_pool_desc& pd = desc->pools[j];
+    bool ok = pd.capacity >= 1 && pd.capacity <= (1 << 20) && pd.window_us >= 0;
+    if (pd.type == TANGRAM_POOL_GPU)
+      ok = ok && (pd.group == 1 || pd.group == 2 || pd.group == 4 || pd.group == 8) && pd.capacity % pd.group == 0;
+    else if (pd.type == TANGRAM_POOL_CPU) ok = ok && pd.group >= 1 && pd.capacity % pd.group == 0;
+    else if (pd.type != TANGRAM_POOL_API) ok = false;
+    if (!ok) return TANGRAM_EINVAL;
+    PoolDev& d = P.pool[j];
+    d.type = pd.type; d.capacity = pd.capacity; d.group = pd.type == TANGRAM_POOL_API ? 1 : pd.group;
+    d.window_us = pd.type == TANGRAM_POOL_API ? pd.window_us : 0;
+    d.node0 = node0; d.n_nodes = pd.type == TANGRAM_POOL_GPU ? pd.capacity / pd.group : 0;
+    node0 += d.n_nodes;
+    d.slot0 = slot0; d.n_slots = pd.type == TANGRAM_POOL_GPU ? 4 : 1;
+    slot0 += d.n_slots;
+  }
+  P.n_nodes_total = node0;
+  P.V = slot0 + desc->n_pools;
+  P.now = now_us;
+
+  // carve the array: fixed parts first, then as many worker slabs as fit, the rest is the arena
+  const size_t SN = (size_t)P.S * P.N;
+  const size_t budget = TANGRAM_STATIC_SCRATCH_BYTES, arena_min = (size_t)4 << 20;
+  size_t off = 0;
+  const size_t o_top = off;   off = align_up(off + 256, 256);
+  const size_t o_meta = off;  off = align_up(off + (size_t)P.S * P.P * sizeof(PoolMeta), 256);
+  const size_t o_order = off; off = align_up(off + SN * sizeof(int), 256);
+  const size_t o_tmin = off;  off = align_up(off + SN * sizeof(i64), 256);
+  size_t per_cand = 8 + 8 + 4 + 4 + 4 + 4 + 4 + 3 + 16 * (size_t)desc->depth;
+  size_t slab = align_up((size_t)P.N * per_cand + 64 * 1024 + (1 << 20) / 4 + 4096, 256);
+  const int wpb = K2_THREADS / 32;
+  if (off + arena_min + slab * wpb > budget) return TANGRAM_ETOOBIG;
+  size_t workers = (budget - off - arena_min) / slab / wpb * wpb;
+  size_t wanted = align_up((size_t)P.S * P.P, wpb);
+  if (workers > wanted) workers = wanted;
+  if (workers > 32) workers = 32;                       // keep most of the array for DP tables
+  const size_t o_slabs = off; off += workers * slab;
+  const size_t o_arena = off;
+
+  int dev = -1;
+  int rc = static_setup(&dev);
+  if (rc) return rc;
+  unsigned char* base = g_static_ptr[dev];
+  P.arena_top = (u64*)(base + o_top); P.meta = (PoolMeta*)(base + o_meta);
+  P.order = (int*)(base + o_order); P.tmin = (i64*)(base + o_tmin);
+  P.slabs = (char*)(base + o_slabs); P.slab_bytes = slab; P.n_workers = (int)workers;
+  P.arena = (char*)(base + o_arena); P.arena_bytes = budget - o_arena;
+  bind_device_io(P, a, res);
+
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CK(cudaMemsetAsync(P.arena_top, 0, sizeof(u64), st));   // the only part that must start at zero
+  k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
+  k_select<<<P.n_workers / wpb, K2_THREADS, 0, st>>>(P);
+  CK(cudaGetLastError());
+  return TANGRAM_OK;
 }

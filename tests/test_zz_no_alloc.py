@@ -1,0 +1,86 @@
+"""tangram_schedule_batch_static: the round for callers that cannot allocate device memory.
+
+Some users embed the scheduler where cudaMalloc is not an option: their framework owns every
+byte of device memory, or they sit in a loop where the implicit synchronisation of an
+allocation is too costly.  For them the library carries a fixed 32 MiB scratch array and an
+entry point that allocates nothing.  This file checks, through the C ABI, that the entry point
+gives exactly what tangram_schedule_batch gives (the scheduler's outputs are integers, so the
+comparison is bit for bit, as in the other GPU tests), on two calls in a row that reuse the
+shared array with different inputs, and that an oversized batch is refused cleanly.
+
+Collected last on purpose: a failure here cannot hide the results of the other tests.
+"""
+import numpy as np
+import pytest
+
+from workloads import generate, make_workload
+
+pytestmark = pytest.mark.gpu
+
+KEYS = ("status", "n_selected", "total_act_us", "alloc_units", "place_node", "place_off", "act_us")
+
+
+def _both_ways(w, a, now_us):
+    import torch
+    from paper_2603_13019_b200 import binding
+    S, N = a["pool"].shape
+    dev = binding.to_device(a)
+    rnd = binding.Round(S, N, w.pools, depth=w.depth)
+    want = rnd.schedule_batch(dev, now_us=now_us)
+    torch.cuda.synchronize()
+    # outputs of the allocation-free call are the caller's own buffers; poison them first
+    got = {k: torch.full_like(v, -7) for k, v in want.items()}
+    rc = binding.schedule_batch_static(w.pools, dev, got, depth=w.depth, now_us=now_us)
+    torch.cuda.synchronize()
+    rnd.destroy()
+    return rc, {k: v.cpu().numpy() for k, v in want.items()}, {k: v.cpu().numpy() for k, v in got.items()}
+
+
+def test_static_entry_point_matches_the_regular_one_twice():
+    # second call: other pools, other sizes, leftovers of the first call still in the array
+    for name, S, now in (("cfg1", 48, 0), ("cfg4", 6, 4321)):
+        w = make_workload(name, n_scenarios=S)
+        a = generate(w)
+        rc, want, got = _both_ways(w, a, now)
+        assert rc == 0
+        for k in KEYS:
+            assert np.array_equal(want[k], got[k]), f"{name}: {k} differs"
+        assert got["n_selected"].sum() > 0 and np.all(got["status"] == 0)
+
+
+def test_static_entry_point_flags_scenarios_whose_tables_do_not_fit():
+    # fragmented GPU pools can need DP tables of several MiB; the built-in array may run out, and
+    # then that scenario (only) carries the workspace status instead of results
+    w = make_workload("cfg3", n_scenarios=12)
+    a = generate(w)
+    rc, want, got = _both_ways(w, a, 0)
+    assert rc == 0 and np.all(want["status"] == 0)
+    assert set(np.unique(got["status"])) <= {0, 4}
+    ok = got["status"] == 0
+    assert ok.sum() >= 6
+    for k in KEYS:
+        assert np.array_equal(want[k][ok], got[k][ok]), f"cfg3: {k} differs"
+
+
+def test_static_entry_point_refuses_what_does_not_fit():
+    import torch
+    from paper_2603_13019_b200 import binding
+    w = make_workload("cfg4", n_scenarios=1024)        # 4 Mi actions need 48 MiB of scratch
+    S, N = w.n_scenarios, w.max_actions
+    # no inputs are read when the call is refused, so tiny placeholders of the right type do
+    z8 = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    z32 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    z64 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    lib = binding.load_library()
+    import ctypes as C
+    arr = (binding._PoolDesc * len(w.pools))(*[binding._PoolDesc(p.type, p.capacity, p.group, p.window_us)
+                                                 for p in w.pools])
+    desc = binding._RoundDesc(S, N, len(w.pools), 2, 0, 0, 0, 0, arr)
+    a = binding._Actions(z8.data_ptr(), z8.data_ptr(), z32.data_ptr(), z64.data_ptr(), z64.data_ptr(), None,
+                         z32.data_ptr(), None)
+    r = binding._Result(z32.data_ptr(), z32.data_ptr(), z32.data_ptr(), z64.data_ptr(), z64.data_ptr(),
+                        z32.data_ptr(), z32.data_ptr(), None, None)
+    rc = lib.tangram_schedule_batch_static(C.byref(desc), C.byref(a), 0, C.byref(r), None)
+    assert rc == -4 and b"static scratch" in lib.tangram_strerror(rc)
+    torch.cuda.synchronize()
+    assert int(z32.item()) == 0                      # nothing was launched, nothing was written
