@@ -323,17 +323,12 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab sl
   return true;
 }
 
-// Greedy eviction (Algorithm 1, lines 8-14).  Returns the number of candidates kept (their
-// multiplicities in T.rkeep), or -1 if the workspace is too small.
-__device__ int evict_loop(const Params& P, const PoolTask& T, Slab slab, int lane) {
+// Greedy eviction (Algorithm 1, lines 8-14), continued from a state in which the first `keep`
+// candidates are kept with objective `obj` and multiplicities T.rkeep.  Returns the number of
+// candidates finally kept, or -1 if the workspace is too small.
+__device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int lane, i64 obj, int keep) {
   i64 opt, est;
-  if (!solve_prefix(P, T, T.m, slab, lane, &opt)) return -1;
-  if (!estimate_rest(P, T, T.m, slab, lane, &est)) return -1;
-  i64 obj = sat_add(opt, est);
-  int keep = T.m;
-  for (int i = lane; i < T.m; i += 32) T.rkeep[i] = T.rsel[i];
-  __syncwarp();
-  for (int t = 1; t <= T.m - 1; ++t) {
+  for (int t = T.m - keep + 1; t <= T.m - 1; ++t) {
     const int q = T.m - t;
     if (!solve_prefix(P, T, q, slab, lane, &opt)) return -1;
     if (!estimate_rest(P, T, q, slab, lane, &est)) return -1;
@@ -344,4 +339,14 @@ __device__ int evict_loop(const Params& P, const PoolTask& T, Slab slab, int lan
     __syncwarp();
   }
   return keep;
+}
+
+// The whole loop, starting from the full candidate list.
+__device__ int evict_loop(const Params& P, const PoolTask& T, Slab slab, int lane) {
+  i64 opt, est;
+  if (!solve_prefix(P, T, T.m, slab, lane, &opt)) return -1;
+  if (!estimate_rest(P, T, T.m, slab, lane, &est)) return -1;
+  for (int i = lane; i < T.m; i += 32) T.rkeep[i] = T.rsel[i];
+  __syncwarp();
+  return evict_resume(P, T, slab, lane, sat_add(opt, est), T.m);
 }

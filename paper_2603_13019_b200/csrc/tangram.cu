@@ -3,6 +3,7 @@
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
+#include <limits.h>
 #include <new>
 
 #include "../../include/tangram.h"
@@ -10,78 +11,94 @@
 #include "prefix_kernel.cuh"
 #include "select.cuh"
 #include "place.cuh"
+#include "sims.cuh"
 
 #define K2_THREADS 256
 #define TG_PROF_CALLS 256   // calls whose kernels can be timed between two queries
-#define TG_PROF_K 2         // kernels per call at most
-#define TG_N_KERNELS 3
+#define TG_PROF_K 4         // timed intervals per call at most
+#define TG_N_KERNELS 6
 
 // ---------------------------------------------------------------------------------------
-// Kernel 2 of a round: one warp per (scenario, pool).  Loads the pool's candidates, runs the
-// all-inelastic shortcut (Algorithm 1, lines 5-6) or the eviction loop, places the grants
-// and writes the candidates' outputs (Eq. 2 for the predicted completion time).
+// Per-(scenario, pool) work of a round, one warp per task.  The pieces are shared by
+//   k_select            everything in one kernel (general path: any number of evictions,
+//                       running actions in the heap; used by the allocation-free entry point),
+//   k_solve / k_finish  the batched path: k_solve computes the optimal allocations of the full
+//                       candidate list and of the list without its last candidate, k_sims
+//                       (sims.cuh) runs all completion-heap simulations one thread each,
+//                       k_finish compares the two objectives (Algorithm 1, lines 8-14), goes on
+//                       evicting in the rare case the first eviction pays, places the grants
+//                       and writes the candidates' outputs (Eq. 2).
 // ---------------------------------------------------------------------------------------
-__device__ void run_pool_task(const Params& P, int sc, int j, Slab slab, int lane) {
-  const PoolMeta mt = P.meta[(size_t)sc * P.P + j];
+struct CandArrays {
+  i64* cs; i64* cp; u32* cmask; int* cidx; int* pnode; int* poff; int* rowcand;
+  u8* cg; u8* rsel; u8* rkeep;
+};
+
+__device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta& mt, Slab& slab, int lane,
+                                  CandArrays& C) {
   const int m = mt.m;
-  if (m == 0) return;
   const PoolDev& pd = P.pool[j];
   const size_t row = (size_t)sc * P.N;
-
-  i64* cs = (i64*)slab.take((u64)m * 8);
-  i64* cp = (i64*)slab.take((u64)m * 8);
-  u32* cmask = (u32*)slab.take((u64)m * 4);
-  int* cidx = (int*)slab.take((u64)m * 4);
-  int* pnode = (int*)slab.take((u64)m * 4);
-  int* poff = (int*)slab.take((u64)m * 4);
-  int* rowcand = (int*)slab.take((u64)m * 4);
-  u8* cg = (u8*)slab.take(m);
-  u8* rsel = (u8*)slab.take(m);
-  u8* rkeep = (u8*)slab.take(m);
-  if (!rkeep) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); return; }
-
+  C.cs = (i64*)slab.take((u64)m * 8);
+  C.cp = (i64*)slab.take((u64)m * 8);
+  C.cmask = (u32*)slab.take((u64)m * 4);
+  C.cidx = (int*)slab.take((u64)m * 4);
+  C.pnode = (int*)slab.take((u64)m * 4);
+  C.poff = (int*)slab.take((u64)m * 4);
+  C.rowcand = (int*)slab.take((u64)m * 4);
+  C.cg = (u8*)slab.take(m);
+  C.rsel = (u8*)slab.take(m);
+  C.rkeep = (u8*)slab.take(m);
+  if (!C.rkeep) return false;
   for (int i = lane; i < m; i += 32) {
     int idx = P.order[row + mt.base + i];
     int g, gang; u32 eff;
     decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], g, gang, eff);
-    cidx[i] = idx; cmask[i] = eff; cg[i] = (u8)(g | (gang << 7));
-    cs[i] = clamp_param(P.a_s[row + idx]); cp[i] = clamp_param(P.a_p[row + idx]);
-    rkeep[i] = (u8)__ffs(eff);
-    pnode[i] = -1; poff[i] = -1;
+    C.cidx[i] = idx; C.cmask[i] = eff; C.cg[i] = (u8)(g | (gang << 7));
+    C.cs[i] = clamp_param(P.a_s[row + idx]); C.cp[i] = clamp_param(P.a_p[row + idx]);
+    C.rkeep[i] = (u8)__ffs(eff);
+    C.pnode[i] = -1; C.poff[i] = -1;
   }
   __syncwarp();
+  return true;
+}
 
+__device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, const CandArrays& C, int lane,
+                          PoolTask& T) {
+  const PoolDev& pd = P.pool[j];
+  const size_t row = (size_t)sc * P.N;
   const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr;
-  int keep = m;
-  if (mt.elastic) {
-    PoolTask T;
-    T.type = pd.type; T.group = pd.group;
-    T.cap[0] = pd.capacity; T.cap[1] = T.cap[2] = T.cap[3] = 0;
-    if (pd.type == TG_POOL_GPU) gpu_caps(pd, busy_row, lane, T.cap);
-    T.m = m; T.cs = cs; T.cp = cp; T.cmask = cmask; T.cg = cg;
-    T.n_ac = mt.count - m;
-    T.ac_tmin = P.tmin + row + mt.base + m;
-    T.ac_first.s = T.ac_first.p = 0; T.ac_first.mask = 1; T.ac_first.g = 1; T.ac_first.gang = 0;
-    if (T.n_ac > 0) {
-      int idx = P.order[row + mt.base + m];
-      decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], T.ac_first.g, T.ac_first.gang, T.ac_first.mask);
-      T.ac_first.s = clamp_param(P.a_s[row + idx]); T.ac_first.p = clamp_param(P.a_p[row + idx]);
-    }
-    T.seeds = nullptr; T.n_seeds = 0;
-    T.depth = P.depth;
-    T.rsel = rsel; T.rkeep = rkeep; T.rowcand = rowcand;
-    keep = evict_loop(P, T, slab, lane);
-    if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+  T.type = pd.type; T.group = pd.group;
+  T.cap[0] = pd.capacity; T.cap[1] = T.cap[2] = T.cap[3] = 0;
+  if (pd.type == TG_POOL_GPU) gpu_caps(pd, busy_row, lane, T.cap);
+  T.m = mt.m; T.cs = C.cs; T.cp = C.cp; T.cmask = C.cmask; T.cg = C.cg;
+  T.n_ac = mt.count - mt.m;
+  T.ac_tmin = P.tmin + row + mt.base + mt.m;
+  T.ac_first.s = T.ac_first.p = 0; T.ac_first.mask = 1; T.ac_first.g = 1; T.ac_first.gang = 0;
+  if (T.n_ac > 0) {
+    int idx = P.order[row + mt.base + mt.m];
+    decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], T.ac_first.g, T.ac_first.gang, T.ac_first.mask);
+    T.ac_first.s = clamp_param(P.a_s[row + idx]); T.ac_first.p = clamp_param(P.a_p[row + idx]);
   }
+  T.seeds = nullptr; T.n_seeds = 0;
+  T.depth = P.depth;
+  T.rsel = C.rsel; T.rkeep = C.rkeep; T.rowcand = C.rowcand;
+}
 
-  // placement on a fresh copy of the pool's topology state
+// placement on a fresh copy of the pool's topology state, then the candidates' outputs
+__device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& mt, const CandArrays& C,
+                                int keep, Slab slab, int lane) {
+  const int m = mt.m;
+  const PoolDev& pd = P.pool[j];
+  const size_t row = (size_t)sc * P.N;
+  const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr;
   if (pd.type == TG_POOL_GPU) {
     u8* nm = (u8*)slab.take(pd.n_nodes);
     if (!nm) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
     else {
       for (int v = lane; v < pd.n_nodes; v += 32) nm[v] = busy_row ? busy_row[pd.node0 + v] : 0;
       __syncwarp();
-      place_gpu(pd, nm, keep, cg, rkeep, pnode, poff, lane);
+      place_gpu(pd, nm, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
     }
   } else if (pd.type == TG_POOL_CPU) {
     const int D = pd.capacity / pd.group, W = (pd.capacity + 31) / 32;
@@ -92,24 +109,24 @@ __device__ void run_pool_task(const Params& P, int sc, int j, Slab slab, int lan
       for (int w = lane; w < W; w += 32) busy[w] = 0;
       for (int d = lane; d < D; d += 32) dfree[d] = pd.group;
       __syncwarp();
-      place_cpu(pd, busy, dfree, keep, cg, rkeep, pnode, poff, lane);
+      place_cpu(pd, busy, dfree, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
     }
   } else {
     if (lane == 0) {
       int used = 0;
-      for (int i = 0; i < keep; ++i) { pnode[i] = 0; poff[i] = used; used += (cg[i] & 0x7f) * rkeep[i]; }
+      for (int i = 0; i < keep; ++i) { C.pnode[i] = 0; C.poff[i] = used; used += (C.cg[i] & 0x7f) * C.rkeep[i]; }
     }
     __syncwarp();
   }
 
   i64 tot = 0; int cnt = 0;
   for (int i = lane; i < m; i += 32) {
-    const size_t o = row + cidx[i];
+    const size_t o = row + C.cidx[i];
     if (i < keep) {
-      int r = rkeep[i];
+      int r = C.rkeep[i];
       i64 arr = P.a_arrival ? P.a_arrival[o] : 0;
-      i64 act = (P.now - arr) + duration(cs[i], cp[i], r);
-      P.o_alloc[o] = (cg[i] & 0x7f) * r; P.o_node[o] = pnode[i]; P.o_off[o] = poff[i]; P.o_act[o] = act;
+      i64 act = (P.now - arr) + duration(C.cs[i], C.cp[i], r);
+      P.o_alloc[o] = (C.cg[i] & 0x7f) * r; P.o_node[o] = C.pnode[i]; P.o_off[o] = C.poff[i]; P.o_act[o] = act;
       tot += act; ++cnt;
     } else {
       P.o_alloc[o] = 0; P.o_node[o] = -1; P.o_off[o] = -1; P.o_act[o] = -1;
@@ -122,6 +139,24 @@ __device__ void run_pool_task(const Params& P, int sc, int j, Slab slab, int lan
   }
 }
 
+__device__ void run_pool_task(const Params& P, int sc, int j, Slab slab, int lane) {
+  const PoolMeta mt = P.meta[(size_t)sc * P.P + j];
+  if (mt.m == 0) return;
+  CandArrays C;
+  if (!gather_candidates(P, sc, j, mt, slab, lane, C)) {
+    if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE);
+    return;
+  }
+  int keep = mt.m;
+  if (mt.elastic) {
+    PoolTask T;
+    make_task(P, sc, j, mt, C, lane, T);
+    keep = evict_loop(P, T, slab, lane);
+    if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+  }
+  place_and_write(P, sc, j, mt, C, keep, slab, lane);
+}
+
 __global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ Params P) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
@@ -130,6 +165,101 @@ __global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ P
   slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
   const int n_tasks = P.S * P.P;
   for (int task = gw; task < n_tasks; task += nw) run_pool_task(P, task / P.P, task % P.P, slab, lane);
+}
+
+// workspace of the batched path, indexed like the partitioned arrays
+struct BatchWs {
+  TaskState* ts;   // [S][P]
+  i64* seed2;      // [S][N] durations of the first m-1 candidates under their optimal allocation
+  u8* rs1;         // [S][N] multiplicities of the optimal allocation of all m candidates
+  u8* rs2;         // [S][N] ... of the first m-1
+};
+
+__global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Params P, const BatchWs W) {
+  const int lane = threadIdx.x & 31;
+  const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
+  const int nw = (gridDim.x * K2_THREADS) >> 5;
+  const int n_tasks = P.S * P.P;
+  for (int task = gw; task < n_tasks; task += nw) {
+    const int sc = task / P.P, j = task % P.P;
+    const PoolMeta mt = P.meta[task];
+    TaskState* st = W.ts + task;
+    if (mt.m == 0 || !mt.elastic) { if (lane == 0) st->flags = 0; continue; }
+    Slab slab;
+    slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
+    CandArrays C;
+    bool ok = gather_candidates(P, sc, j, mt, slab, lane, C);
+    i64 opt0 = 0, opt1 = 0;
+    if (ok) {
+      PoolTask T;
+      make_task(P, sc, j, mt, C, lane, T);
+      const size_t pos = (size_t)sc * P.N + mt.base;
+      ok = solve_prefix(P, T, mt.m, slab, lane, &opt0);
+      if (ok) {
+        for (int i = lane; i < mt.m; i += 32) {
+          W.rs1[pos + i] = C.rsel[i];
+          P.tmin[pos + i] = duration(C.cs[i], C.cp[i], C.rsel[i]);   // heap seeds of the full list
+        }
+        __syncwarp();
+        if (mt.m >= 2) {
+          ok = solve_prefix(P, T, mt.m - 1, slab, lane, &opt1);
+          if (ok)
+            for (int i = lane; i < mt.m - 1; i += 32) {
+              W.rs2[pos + i] = C.rsel[i];
+              W.seed2[pos + i] = duration(C.cs[i], C.cp[i], C.rsel[i]);
+            }
+        }
+      }
+    }
+    if (lane == 0) {
+      st->opt[0] = opt0; st->opt[1] = opt1;
+      st->est[0] = (mt.count - mt.m) > 0 ? TG_INF : 0;
+      st->est[1] = TG_INF;
+      st->flags = ok ? TS_SOLVED : TS_FAILED;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ Params P, const BatchWs W) {
+  const int lane = threadIdx.x & 31;
+  const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
+  const int nw = (gridDim.x * K2_THREADS) >> 5;
+  const int n_tasks = P.S * P.P;
+  for (int task = gw; task < n_tasks; task += nw) {
+    const int sc = task / P.P, j = task % P.P;
+    const PoolMeta mt = P.meta[task];
+    if (mt.m == 0) continue;
+    Slab slab;
+    slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
+    CandArrays C;
+    if (!gather_candidates(P, sc, j, mt, slab, lane, C)) {
+      if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE);
+      continue;
+    }
+    int keep = mt.m;
+    if (mt.elastic) {
+      const TaskState st = W.ts[task];
+      if (!(st.flags & TS_SOLVED) || (st.flags & TS_FAILED)) keep = -1;
+      else {
+        const size_t pos = (size_t)sc * P.N + mt.base;
+        i64 obj = sat_add(st.opt[0], st.est[0]);
+        for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = W.rs1[pos + i];
+        if (mt.m >= 2) {
+          i64 nobj = sat_add(st.opt[1], st.est[1]);
+          if (nobj < obj) {                                  // the first eviction pays: go on (rare)
+            for (int i = lane; i < mt.m - 1; i += 32) C.rkeep[i] = W.rs2[pos + i];
+            __syncwarp();
+            PoolTask T;
+            make_task(P, sc, j, mt, C, lane, T);
+            keep = evict_resume(P, T, slab, lane, nobj, mt.m - 1);
+          }
+        }
+        __syncwarp();
+      }
+      if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+    }
+    place_and_write(P, sc, j, mt, C, keep, slab, lane);
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -151,6 +281,7 @@ struct tangram_round {
   int64_t launches;
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
+  BatchWs W; int sim_blocks;
   // staging for host-buffer mode
   char* d_stage; size_t stage_bytes;
   size_t in_off[8], out_off[9];
@@ -158,7 +289,11 @@ struct tangram_round {
   cudaEvent_t* ev; int ev_calls, ev_used; int ev_kernel[TG_PROF_CALLS][TG_PROF_K];
 };
 
-static const char* const g_kernel_names[TG_N_KERNELS] = {"k_prefix", "k_select", "k_replay"};
+static const char* const g_kernel_names[TG_N_KERNELS] = {"k_prefix", "k_select", "k_replay",
+                                                          "k_solve", "k_sims", "k_finish"};
+// heap-capacity classes of k_sims: (lo, hi] with heaps in shared memory; beyond the last, in the arena
+static const int g_sim_classes[] = {0, 32, 64, 96, 128, 160, 192, 256, 384};
+#define TG_N_SIM_CLASSES 8
 
 static cudaError_t fill_tables() {
   u64 recip[33];
@@ -259,6 +394,11 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc(&r->d_slabs, (size_t)P.n_workers * slab) != cudaSuccess;
   bad |= cudaMalloc(&r->d_arena, P.arena_bytes) != cudaSuccess;
   bad |= cudaMalloc(&r->d_arena_top, 256) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.ts, (size_t)P.S * P.P * sizeof(TaskState)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.seed2, SN * sizeof(i64)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.rs1, SN) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.rs2, SN) != cudaSuccess;
+  r->sim_blocks = (int)(((long long)P.P * P.S * 2 * P.depth + SIM_THREADS - 1) / SIM_THREADS);
   if (!bad && desc->host_buffers) {
     size_t off = 0;
     size_t in_sz[8] = {SN, SN, SN * 4, SN * 8, SN * 8, SN * 8, (size_t)P.S * 4, (size_t)P.S * (node0 ? node0 : 1)};
@@ -274,6 +414,9 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_prefix, cudaFuncAttributeMaxDynamicSharedMemorySize, P.V * K1_THREADS * 4);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_sims, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (g_sim_classes[TG_N_SIM_CLASSES] + 4) * SIM_THREADS * (int)sizeof(i64));
   if (e != cudaSuccess) { tangram_round_destroy(r); return cuda_fail(e, "cudaFuncSetAttribute"); }
   *out = r;
   return TANGRAM_OK;
@@ -322,10 +465,10 @@ extern "C" int tangram_kernel_time_ms(tangram_round* r, int kernel, double* tota
 }
 
 // events of the current call, or null when timing is off or the event pool is used up
-static cudaEvent_t* prof_begin(tangram_round* r, int k0, int k1) {
+static cudaEvent_t* prof_begin(tangram_round* r, int k0, int k1, int k2, int k3) {
   if (!r->ev || r->ev_used >= TG_PROF_CALLS) return nullptr;
   int c = r->ev_used++;
-  r->ev_kernel[c][0] = k0; r->ev_kernel[c][1] = k1;
+  r->ev_kernel[c][0] = k0; r->ev_kernel[c][1] = k1; r->ev_kernel[c][2] = k2; r->ev_kernel[c][3] = k3;
   return r->ev + c * (TG_PROF_K + 1);
 }
 
@@ -334,6 +477,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
   cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage);
+  cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   delete r;
 }
 
@@ -394,13 +538,22 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
     if (rc) return rc;
   } else bind_device_io(P, a, res);
   CK(cudaMemsetAsync(P.arena_top, 0, sizeof(u64), st));
-  cudaEvent_t* ev = prof_begin(r, 0, 1);
+  cudaEvent_t* ev = prof_begin(r, 0, 3, 4, 5);
+  const int wblocks = P.n_workers / (K2_THREADS / 32);
   if (ev) CK(cudaEventRecord(ev[0], st));
   k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
   if (ev) CK(cudaEventRecord(ev[1], st));
-  k_select<<<P.n_workers / (K2_THREADS / 32), K2_THREADS, 0, st>>>(P);
+  k_solve<<<wblocks, K2_THREADS, 0, st>>>(P, r->W);
   if (ev) CK(cudaEventRecord(ev[2], st));
-  r->launches += 2;
+  for (int c = 0; c < TG_N_SIM_CLASSES; ++c) {
+    const int lo = g_sim_classes[c], hi = g_sim_classes[c + 1];
+    k_sims<<<r->sim_blocks, SIM_THREADS, (hi + 4) * SIM_THREADS * sizeof(i64), st>>>(P, r->W.ts, r->W.seed2, lo, hi, 0);
+  }
+  k_sims<<<r->sim_blocks, SIM_THREADS, 0, st>>>(P, r->W.ts, r->W.seed2, g_sim_classes[TG_N_SIM_CLASSES], INT_MAX, 1);
+  if (ev) CK(cudaEventRecord(ev[3], st));
+  k_finish<<<wblocks, K2_THREADS, 0, st>>>(P, r->W);
+  if (ev) CK(cudaEventRecord(ev[4], st));
+  r->launches += 3 + TG_N_SIM_CLASSES + 1;
   CK(cudaGetLastError());
   if (r->desc.host_buffers) return unstage_outputs(r, res, P, st);
   return TANGRAM_OK;
