@@ -87,3 +87,46 @@ __device__ void place_cpu(const PoolDev& pd, u32* busy, int* dfree, int keep, co
     __syncwarp();
   }
 }
+
+// CPU placement on a pool nobody occupies yet (a single round).  Cores are only ever taken
+// lowest id first, so the used cores of a domain are always a prefix of it: the free count per
+// domain is the whole state and a grant's first core follows from it.  Same rule as place_cpu.
+__device__ void place_cpu_fresh(const PoolDev& pd, int* dfree, int keep, const u8* cg, const u8* r,
+                                int* pnode, int* poff, int lane) {
+  const int D = pd.capacity / pd.group;
+  for (int d = lane; d < D; d += 32) dfree[d] = pd.group;
+  __syncwarp();
+  for (int i0 = 0; i0 < keep; i0 += 32) {
+    // this lane's candidate of the block of 32; its units are broadcast when its turn comes
+    const int mine = i0 + lane < keep ? (cg[i0 + lane] & 0x7f) * r[i0 + lane] : 0;
+    const int nb = min(32, keep - i0);
+    for (int b = 0; b < nb; ++b) {
+      const int k = __shfl_sync(TG_FULL, mine, b);
+      i64 key = TG_INF;
+      for (int d = lane; d < D; d += 32) {
+        int f = dfree[d];
+        if (f >= k) key = min(key, ((i64)f << 32) | d);
+      }
+      key = warp_min64(key);
+      if (lane == 0) {
+        int first = -1;
+        if (key != TG_INF) {
+          int d = (int)(key & 0xffffffff);
+          first = d * pd.group + (pd.group - dfree[d]);
+          dfree[d] -= k;
+        } else {
+          int need = k;
+          for (int d = 0; d < D && need > 0; ++d) {
+            int f = dfree[d];
+            if (f == 0) continue;
+            if (first < 0) first = d * pd.group + (pd.group - f);
+            int take = min(f, need);
+            dfree[d] = f - take; need -= take;
+          }
+        }
+        pnode[i0 + b] = first >= 0 ? first / pd.group : -1; poff[i0 + b] = first;
+      }
+      __syncwarp();
+    }
+  }
+}

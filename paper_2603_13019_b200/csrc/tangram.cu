@@ -29,6 +29,13 @@
 //                       evicting in the rare case the first eviction pays, places the grants
 //                       and writes the candidates' outputs (Eq. 2).
 // ---------------------------------------------------------------------------------------
+// Tasks are handed out by a counter so that long tasks do not pile up on the same warps.
+__device__ __forceinline__ int next_task(u64* counter, int lane) {
+  u64 x = 0;
+  if (lane == 0) x = atomicAdd(counter, 1ull);
+  return (int)__shfl_sync(TG_FULL, x, 0);
+}
+
 struct CandArrays {
   i64* cs; i64* cp; u32* cmask; int* cidx; int* pnode; int* poff; int* rowcand;
   u8* cg; u8* rsel; u8* rkeep;
@@ -101,16 +108,10 @@ __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& 
       place_gpu(pd, nm, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
     }
   } else if (pd.type == TG_POOL_CPU) {
-    const int D = pd.capacity / pd.group, W = (pd.capacity + 31) / 32;
-    u32* busy = (u32*)slab.take((u64)W * 4);
+    const int D = pd.capacity / pd.group;
     int* dfree = (int*)slab.take((u64)D * 4);
     if (!dfree) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
-    else {
-      for (int w = lane; w < W; w += 32) busy[w] = 0;
-      for (int d = lane; d < D; d += 32) dfree[d] = pd.group;
-      __syncwarp();
-      place_cpu(pd, busy, dfree, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
-    }
+    else place_cpu_fresh(pd, dfree, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
   } else {
     if (lane == 0) {
       int used = 0;
@@ -164,7 +165,12 @@ __global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ P
   Slab slab;
   slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
   const int n_tasks = P.S * P.P;
-  for (int task = gw; task < n_tasks; task += nw) run_pool_task(P, task / P.P, task % P.P, slab, lane);
+  (void)nw;
+  for (;;) {
+    const int x = next_task(P.arena_top + 3, lane);
+    if (x >= n_tasks) break;
+    run_pool_task(P, x % P.S, x / P.S, slab, lane);       // pool-major: pool 0 of every scenario first
+  }
 }
 
 // workspace of the batched path, indexed like the partitioned arrays
@@ -180,8 +186,11 @@ __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Pa
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
   const int nw = (gridDim.x * K2_THREADS) >> 5;
   const int n_tasks = P.S * P.P;
-  for (int task = gw; task < n_tasks; task += nw) {
-    const int sc = task / P.P, j = task % P.P;
+  (void)nw;
+  for (;;) {
+    const int x = next_task(P.arena_top + 1, lane);
+    if (x >= n_tasks) break;
+    const int sc = x % P.S, j = x / P.S, task = sc * P.P + j;
     const PoolMeta mt = P.meta[task];
     TaskState* st = W.ts + task;
     if (mt.m == 0 || !mt.elastic) { if (lane == 0) st->flags = 0; continue; }
@@ -225,8 +234,11 @@ __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ P
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
   const int nw = (gridDim.x * K2_THREADS) >> 5;
   const int n_tasks = P.S * P.P;
-  for (int task = gw; task < n_tasks; task += nw) {
-    const int sc = task / P.P, j = task % P.P;
+  (void)nw;
+  for (;;) {
+    const int x = next_task(P.arena_top + 2, lane);
+    if (x >= n_tasks) break;
+    const int sc = x % P.S, j = x / P.S, task = sc * P.P + j;
     const PoolMeta mt = P.meta[task];
     if (mt.m == 0) continue;
     Slab slab;
@@ -537,7 +549,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
     int rc = stage_inputs(r, a, P, st);
     if (rc) return rc;
   } else bind_device_io(P, a, res);
-  CK(cudaMemsetAsync(P.arena_top, 0, sizeof(u64), st));
+  CK(cudaMemsetAsync(P.arena_top, 0, 256, st));          // arena top and the task counters
   cudaEvent_t* ev = prof_begin(r, 0, 3, 4, 5);
   const int wblocks = P.n_workers / (K2_THREADS / 32);
   if (ev) CK(cudaEventRecord(ev[0], st));
@@ -656,7 +668,7 @@ extern "C" int tangram_schedule_batch_static(const tangram_round_desc* desc, con
   bind_device_io(P, a, res);
 
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  CK(cudaMemsetAsync(P.arena_top, 0, sizeof(u64), st));   // the only part that must start at zero
+  CK(cudaMemsetAsync(P.arena_top, 0, 256, st));           // the only part that must start at zero
   k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
   k_select<<<P.n_workers / wpb, K2_THREADS, 0, st>>>(P);
   CK(cudaGetLastError());
