@@ -15,6 +15,7 @@
 
 #define K2_THREADS 256
 #define TG_PROF_CALLS 256   // calls whose kernels can be timed between two queries
+#define TG_N_SIM_CLASSES 22
 #define TG_PROF_K 4         // timed intervals per call at most
 #define TG_N_KERNELS 6
 
@@ -293,7 +294,11 @@ struct tangram_round {
   int64_t launches;
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
-  BatchWs W; int sim_blocks;
+  BatchWs W; int sim_blocks; SimLists L; int n_sm;
+  // the capacity classes of k_sims are independent: they run on side streams between a fork
+  // and a join event so that their partial waves overlap
+  cudaStream_t sim_stream[TG_N_SIM_CLASSES + 1];
+  cudaEvent_t sim_fork, sim_join[TG_N_SIM_CLASSES + 1];
   // staging for host-buffer mode
   char* d_stage; size_t stage_bytes;
   size_t in_off[8], out_off[9];
@@ -303,9 +308,11 @@ struct tangram_round {
 
 static const char* const g_kernel_names[TG_N_KERNELS] = {"k_prefix", "k_select", "k_replay",
                                                           "k_solve", "k_sims", "k_finish"};
-// heap-capacity classes of k_sims: (lo, hi] with heaps in shared memory; beyond the last, in the arena
-static const int g_sim_classes[] = {0, 32, 64, 96, 128, 160, 192, 256, 384};
-#define TG_N_SIM_CLASSES 8
+// capacity classes (slots per simulation) of the shared-memory simulation kernels
+static const int g_sim_caps[TG_N_SIM_CLASSES] = {16, 32, 48, 64, 80, 96, 112, 128, 144, 160, 176, 192, 224, 256,
+                                                 320, 384, 512, 768, 1024, 1536, 2048, 2816};
+#define TG_SMEM_PER_SM 233472   // shared memory an SM can split among resident blocks
+#define TG_SMEM_PER_BLOCK 232448
 
 static cudaError_t fill_tables() {
   u64 recip[33];
@@ -410,7 +417,20 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc((void**)&r->W.seed2, SN * sizeof(i64)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.rs1, SN) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.rs2, SN) != cudaSuccess;
-  r->sim_blocks = (int)(((long long)P.P * P.S * 2 * P.depth + SIM_THREADS - 1) / SIM_THREADS);
+  const long long n_sims = (long long)P.P * P.S * 2 * P.depth;
+  r->sim_blocks = (int)((n_sims + 31) / 32);
+  r->n_sm = prop.multiProcessorCount;
+  r->L.n_groups = (int)((n_sims + SIM_PER_WARP - 1) / SIM_PER_WARP);
+  r->L.n_classes = TG_N_SIM_CLASSES;
+  for (int c = 0; c < TG_N_SIM_CLASSES; ++c) r->L.cap[c] = g_sim_caps[c];
+  bad |= cudaMalloc((void**)&r->L.count, 2 * 64 * sizeof(int)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->L.list, (size_t)TG_N_SIM_CLASSES * r->L.n_groups * sizeof(int)) != cudaSuccess;
+  r->L.cursor = r->L.count ? r->L.count + 64 : nullptr;
+  bad |= cudaEventCreateWithFlags(&r->sim_fork, cudaEventDisableTiming) != cudaSuccess;
+  for (int c = 0; c <= TG_N_SIM_CLASSES; ++c) {
+    bad |= cudaStreamCreateWithFlags(&r->sim_stream[c], cudaStreamNonBlocking) != cudaSuccess;
+    bad |= cudaEventCreateWithFlags(&r->sim_join[c], cudaEventDisableTiming) != cudaSuccess;
+  }
   if (!bad && desc->host_buffers) {
     size_t off = 0;
     size_t in_sz[8] = {SN, SN, SN * 4, SN * 8, SN * 8, SN * 8, (size_t)P.S * 4, (size_t)P.S * (node0 ? node0 : 1)};
@@ -427,8 +447,9 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_prefix, cudaFuncAttributeMaxDynamicSharedMemorySize, P.V * K1_THREADS * 4);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_sims, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (g_sim_classes[TG_N_SIM_CLASSES] + 4) * SIM_THREADS * (int)sizeof(i64));
+    e = cudaFuncSetAttribute(k_sims4<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_PER_BLOCK - 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_sims4<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_PER_BLOCK - 1024);
   if (e != cudaSuccess) { tangram_round_destroy(r); return cuda_fail(e, "cudaFuncSetAttribute"); }
   *out = r;
   return TANGRAM_OK;
@@ -490,6 +511,12 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
   cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
+  cudaFree(r->L.count); cudaFree(r->L.list);
+  if (r->sim_fork) cudaEventDestroy(r->sim_fork);
+  for (int c = 0; c <= TG_N_SIM_CLASSES; ++c) {
+    if (r->sim_stream[c]) cudaStreamDestroy(r->sim_stream[c]);
+    if (r->sim_join[c]) cudaEventDestroy(r->sim_join[c]);
+  }
   delete r;
 }
 
@@ -557,15 +584,28 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   if (ev) CK(cudaEventRecord(ev[1], st));
   k_solve<<<wblocks, K2_THREADS, 0, st>>>(P, r->W);
   if (ev) CK(cudaEventRecord(ev[2], st));
+  CK(cudaMemsetAsync(r->L.count, 0, 2 * 64 * sizeof(int), st));
+  k_sim_classify<<<(r->L.n_groups + 255) / 256, 256, 0, st>>>(P, r->W.ts, r->L);
+  CK(cudaEventRecord(r->sim_fork, st));
   for (int c = 0; c < TG_N_SIM_CLASSES; ++c) {
-    const int lo = g_sim_classes[c], hi = g_sim_classes[c + 1];
-    k_sims<<<r->sim_blocks, SIM_THREADS, (hi + 4) * SIM_THREADS * sizeof(i64), st>>>(P, r->W.ts, r->W.seed2, lo, hi, 0);
+    cudaStream_t ss = r->sim_stream[c];
+    CK(cudaStreamWaitEvent(ss, r->sim_fork, 0));
+    const int smem = g_sim_caps[c] * SIM_PER_WARP * SIM_SLOT_BYTES;
+    int per_sm = TG_SMEM_PER_SM / (smem + 1024);
+    if (per_sm > 32) per_sm = 32;
+    if (per_sm < 1) per_sm = 1;
+    int grid = r->n_sm * per_sm;
+    if (grid > r->L.n_groups) grid = r->L.n_groups;
+    if (2 * g_sim_caps[c] <= 512) k_sims4<2><<<grid, 32, smem, ss>>>(P, r->W.ts, r->W.seed2, r->L, c);
+    else k_sims4<3><<<grid, 32, smem, ss>>>(P, r->W.ts, r->W.seed2, r->L, c);
+    CK(cudaEventRecord(r->sim_join[c], ss));
+    CK(cudaStreamWaitEvent(st, r->sim_join[c], 0));
   }
-  k_sims<<<r->sim_blocks, SIM_THREADS, 0, st>>>(P, r->W.ts, r->W.seed2, g_sim_classes[TG_N_SIM_CLASSES], INT_MAX, 1);
+  k_sims_big<<<r->sim_blocks, 32, 0, st>>>(P, r->W.ts, r->W.seed2, g_sim_caps[TG_N_SIM_CLASSES - 1], r->L.count + 63);
   if (ev) CK(cudaEventRecord(ev[3], st));
   k_finish<<<wblocks, K2_THREADS, 0, st>>>(P, r->W);
   if (ev) CK(cudaEventRecord(ev[4], st));
-  r->launches += 3 + TG_N_SIM_CLASSES + 1;
+  r->launches += 5 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
   if (r->desc.host_buffers) return unstage_outputs(r, res, P, st);
   return TANGRAM_OK;
