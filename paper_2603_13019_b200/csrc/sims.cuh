@@ -1,42 +1,52 @@
 // Completion-heap simulations of Algorithm 2 (estimate).
 //
 // A round needs, per elastic (scenario, pool), the objective of the full candidate list and of
-// the list without its last candidate (the first eviction step), each at `depth` levels of the
-// first waiting action: 2 * depth independent sequential simulations of |waiting| "pop the
-// earliest completion, push completion + duration" steps.
+// the list without its last candidate (the first eviction step).  Each is a sequential
+// simulation of |waiting| "pop the earliest completion ts, push ts + T" steps.
 //
-// The priority queue of a simulation is a winner tree over its H slots: slot values val[0..H)
-// and, for every internal node n = 1..H-1 of the implicit tree (leaf i = node H+i), the slot
-// holding the subtree's minimum.  Replacing the minimum only touches the path from its leaf to
-// the root, and the siblings on that path are known from the leaf alone.  FOUR LANES share one
-// simulation: each lane loads the siblings of its 2-3 levels, a two-step prefix-minimum over
-// the four lanes yields the winner entering every level, each lane stores its levels' winners.
-// A warp thus runs 8 simulations with a short dependent chain per step, and four times as
-// many warps are resident for the same shared memory as with one lane per simulation (the
-// trees' shared-memory footprint, not registers, limits residency).
+// One simulation per prefix is enough although Algorithm 2 tries `depth` levels of the first
+// waiting action and keeps the best: if one multiset of completion times is elementwise <=
+// another, it stays so after a step with the same T and every popped time is <=, so the
+// estimate is non-decreasing in the first action's duration; durations do not grow with the
+// level, hence the best depth is always the largest level tried.
 //
-// Work distribution: k_sim_classify sorts groups of 8 consecutive simulations (same pool,
+// The priority queue is a winner tree of packed keys: node n of the implicit tree over H slots
+// (leaf i = node H + i) holds the smallest key of its subtree, key = 2^62 | completion << 12 |
+// slot.  Replacing the minimum only touches the path from its leaf to the root, and the
+// siblings on that path are known from the leaf alone, so their loads are all issued at once
+// and only a chain of minima remains sequential.  With bit 62 set every key is the bit pattern
+// of a positive normal double, whose order is the integer order, so a key minimum is one fmin.
+// One lane runs one simulation; a warp's 32 trees live in shared memory interleaved by lane
+// (node n of lane t at n * 32 + t, conflict free).  Shared memory bounds how many simulations
+// are resident, so what matters is the latency of a step, not the number of warps.
+// A completion time that would not fit the 49 value bits sends the simulation to the exact
+// 64-bit kernel below.
+//
+// Work distribution: k_sim_classify sorts groups of 32 consecutive simulations (same pool,
 // neighbouring scenarios, hence similar H) into capacity classes; one persistent kernel per
 // class, sized to fill the GPU at that class's shared-memory footprint, pulls groups from its
-// list.  Classes run concurrently on side streams.  Trees too large for shared memory are
-// simulated one lane each in the arena (k_sims_big).
+// list.  Classes run concurrently on side streams.  k_sims_big (trees in the arena) takes what
+// is too large for shared memory or overflowed the packing.
 #pragma once
 #include "common.cuh"
 
-#define SIM_G 4                 // lanes per simulation
-#define SIM_PER_WARP 8          // simulations per warp (32 / SIM_G)
-#define SIM_SLOT_BYTES 10       // shared memory per slot: i64 value + u16 node
-typedef unsigned short u16;
+#define SIM_PER_WARP 32         // simulations per warp
+#define SIM_SLOT_BYTES 16       // shared memory per slot: two tree nodes of 8 bytes
+#define SIM_SLOT_BITS 12
+#define SIM_VALUE_LIMIT (1LL << 49)
+#define SIM_KEY_BIAS (1LL << 62)
+#define SIM_KEY_INF 0x7FE0000000000000LL
 
 // per (scenario, pool) state handed from the solve kernel to the simulations and the finish kernel
 struct TaskState {
   i64 opt[2];     // optimal duration sum of all m candidates / of the first m-1
-  i64 est[2];     // estimate of the rest for those two prefixes: min over depths (atomicMin)
+  i64 est[2];     // estimate of the rest for those two prefixes
   int flags;      // TS_* bits
   int pad;
 };
 #define TS_SOLVED 1   // both prefixes solved, heap seeds written
 #define TS_FAILED 2   // workspace too small
+#define TS_REDO0 4    // simulation of prefix e overflowed the packed keys: bit TS_REDO0 << e
 
 __device__ __forceinline__ int nth_level_of(u32 mask, int d) {
   for (int k = 0; k < d; ++k) mask &= mask - 1;
@@ -51,12 +61,11 @@ struct SimJob {
   TaskState* st;
 };
 
-// number of slots of simulation `sim` (0 if it does not exist); cheap, for classification
+// simulation index = (pool * S + scenario) * 2 + e
 __device__ __forceinline__ int sim_slots(const Params& P, const TaskState* ts, long long sim) {
-  const long long n_sims = (long long)P.P * P.S * 2 * P.depth;
-  if (sim >= n_sims) return 0;
-  long long x = sim / P.depth;
-  const int e = (int)(x & 1); x >>= 1;
+  if (sim >= (long long)P.P * P.S * 2) return 0;
+  const int e = (int)(sim & 1);
+  const long long x = sim >> 1;
   const int sc = (int)(x % P.S), j = (int)(x / P.S);
   const PoolMeta mt = P.meta[(size_t)sc * P.P + j];
   if (!(mt.elastic && mt.m >= 1 + e && (e + mt.count - mt.m) > 0)) return 0;
@@ -67,11 +76,9 @@ __device__ __forceinline__ int sim_slots(const Params& P, const TaskState* ts, l
 __device__ __forceinline__ SimJob sim_job(const Params& P, TaskState* ts, const i64* seed2, long long sim) {
   SimJob J;
   J.active = false; J.H = 0; J.n_list = 0; J.e = 0; J.seeds = nullptr; J.lst = nullptr; J.first_dur = 0; J.st = nullptr;
-  const long long n_sims = (long long)P.P * P.S * 2 * P.depth;
-  if (sim >= n_sims) return J;
-  const int d = (int)(sim % P.depth);
-  long long x = sim / P.depth;
-  const int e = (int)(x & 1); x >>= 1;
+  if (sim >= (long long)P.P * P.S * 2) return J;
+  const int e = (int)(sim & 1);
+  const long long x = sim >> 1;
   const int sc = (int)(x % P.S), j = (int)(x / P.S);
   const PoolMeta mt = P.meta[(size_t)sc * P.P + j];
   J.st = ts + (size_t)sc * P.P + j;
@@ -80,11 +87,12 @@ __device__ __forceinline__ SimJob sim_job(const Params& P, TaskState* ts, const 
   if (!(mt.elastic && mt.m >= 1 + e && (e + n_ac) > 0 && (J.st->flags & TS_SOLVED))) return J;
   const size_t row = (size_t)sc * P.N;
   const PoolDev& pd = P.pool[j];
-  // first remaining action: the evicted last candidate (e = 1) or the first waiting one
+  // first remaining action: the evicted last candidate (e = 1) or the first waiting one; it takes
+  // the largest of its first `depth` levels (see the header for why that depth is the best)
   const int idx = P.order[row + mt.base + mt.m - e];
   int g, gang; u32 fm;
   decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], g, gang, fm);
-  if (d >= min(P.depth, __popc(fm))) return J;
+  const int d = min(P.depth, __popc(fm)) - 1;
   J.active = true;
   J.first_dur = duration(clamp_param(P.a_s[row + idx]), clamp_param(P.a_p[row + idx]), nth_level_of(fm, d));
   J.H = mt.m - e;
@@ -96,7 +104,7 @@ __device__ __forceinline__ SimJob sim_job(const Params& P, TaskState* ts, const 
 
 // work lists of the capacity classes
 struct SimLists {
-  int* count;      // [n_classes] groups appended
+  int* count;      // [n_classes] groups appended; count[63]: something is left for k_sims_big
   int* cursor;     // [n_classes] groups taken
   int* list;       // [n_classes][n_groups]
   int n_groups, n_classes;
@@ -116,21 +124,30 @@ __global__ void k_sim_classify(const __grid_constant__ Params P, const TaskState
   L.list[(size_t)c * L.n_groups + pos] = g;
 }
 
-struct Key { i64 v; int i; };
-__device__ __forceinline__ Key key_min(Key a, Key b) { return b.v < a.v ? b : a; }
+// minimum of two keys (see the header: keys order like the doubles they spell)
+__device__ __forceinline__ i64 key_min(i64 a, i64 b) {
+  return __double_as_longlong(fmin(__longlong_as_double(a), __longlong_as_double(b)));
+}
 
-// position of element e of simulation s inside a warp's arrays (swizzled against bank conflicts)
-__device__ __forceinline__ int sim_at(int e, int s) { return e * SIM_PER_WARP + ((s + e) & (SIM_PER_WARP - 1)); }
+__device__ __forceinline__ i64 lds64(u32 addr) {
+  i64 v;
+  asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts64(u32 addr, i64 v) {
+  asm volatile("st.shared.b64 [%0], %1;" :: "r"(addr), "l"(v) : "memory");
+}
 
-// One persistent warp per block; LPL = tree levels per lane (4 * LPL >= path length of the class).
-template <int LPL>
-__global__ void __launch_bounds__(32) k_sims4(const __grid_constant__ Params P, TaskState* ts, const i64* seed2,
+// One persistent warp per block, one lane per simulation; MAXD bounds the path length of the
+// class (2 * capacity <= 2^(MAXD+1)).  Node n of lane t is at shared address base + n * 256 with
+// base = (512-aligned start) + t * 8, so that with o = n * 256 the sibling of a node is at
+// (base + o) ^ 256 and the node offsets of a leaf-to-root path are (leaf offset >> level) & ~255.
+template <int MAXD>
+__global__ void __launch_bounds__(32) k_sims1(const __grid_constant__ Params P, TaskState* ts, const i64* seed2,
                                               const SimLists L, int cls) {
   extern __shared__ __align__(16) unsigned char sim_smem[];
-  const int hcap = L.cap[cls];
-  i64* val = (i64*)sim_smem;
-  u16* tree = (u16*)(sim_smem + (size_t)hcap * SIM_PER_WARP * sizeof(i64));
-  const int lane = threadIdx.x, q = lane & (SIM_G - 1), s = lane >> 2;
+  const int lane = threadIdx.x;
+  const u32 base = (((u32)__cvta_generic_to_shared(sim_smem) + 511u) & ~511u) + (u32)lane * 8u;
   const int count = L.count[cls];
   for (;;) {
     int gi = 0;
@@ -138,100 +155,76 @@ __global__ void __launch_bounds__(32) k_sims4(const __grid_constant__ Params P, 
     gi = __shfl_sync(TG_FULL, gi, 0);
     if (gi >= count) break;
     const int grp = L.list[(size_t)cls * L.n_groups + gi];
-    const SimJob J = sim_job(P, ts, seed2, (long long)grp * SIM_PER_WARP + s);
+    const SimJob J = sim_job(P, ts, seed2, (long long)grp * SIM_PER_WARP + lane);
+    if (!J.active) continue;                           // lanes are independent: no warp-wide step below
     const int H = J.H;
-    __syncwarp();
-    if (J.active) {
-      for (int i = q; i < H; i += SIM_G) val[sim_at(i, s)] = J.seeds[i];
-    }
-    __syncwarp();
-    if (J.active && q == 0) {
-      for (int n = H - 1; n >= 1; --n) {
-        int ca = 2 * n, cb = 2 * n + 1;
-        int a = ca >= H ? ca - H : (int)tree[sim_at(ca, s)];
-        int b = cb >= H ? cb - H : (int)tree[sim_at(cb, s)];
-        tree[sim_at(n, s)] = (u16)(val[sim_at(b, s)] < val[sim_at(a, s)] ? b : a);
-      }
-    }
-    __syncwarp();
-    int w = 0; i64 wv = 0;
-    if (J.active) { w = H > 1 ? (int)tree[sim_at(1, s)] : 0; wv = val[sim_at(w, s)]; }
-    const int steps = J.active ? J.n_list + 1 : 0;
-    const int kmax = warp_max32(steps);
+    for (int i = 0; i < H; ++i) sts64(base + (u32)(H + i) * 256u, SIM_KEY_BIAS | (J.seeds[i] << SIM_SLOT_BITS) | i);
+    for (int n = H - 1; n >= 1; --n)
+      sts64(base + (u32)n * 256u, key_min(lds64(base + (u32)(2 * n) * 256u), lds64(base + (u32)(2 * n + 1) * 256u)));
+    i64 top = lds64(base + (u32)(H > 1 ? 1 : H) * 256u);   // key of the earliest completion
     i64 tmp = 0;
-    i64 d0 = J.first_dur;
-    i64 d1 = J.n_list > 0 ? J.lst[0] : 0, d2 = J.n_list > 1 ? J.lst[1] : 0;
-    for (int k = 0; k < kmax; ++k) {
-      const bool live = k < steps;
-      i64 d3 = (live && k + 2 < J.n_list) ? J.lst[k + 2] : 0;       // durations fetched three steps ahead
-      const i64 v = wv + d0;                                         // pop earliest completion, push ts + T
-      if (live) tmp = sat_add(tmp, v);
-      const int n0 = H + w;
-      if (live && q == 0) val[sim_at(w, s)] = v;
-      // siblings of this lane's levels
-      Key sk[LPL]; int par[LPL];
+    u32 ovf = 0;
+    // durations are fetched a chunk of four ahead (stream[0] = first action, then the list)
+    const int steps = J.n_list + 1;
+    i64 cur[4], nxt[4];
 #pragma unroll
-      for (int x = 0; x < LPL; ++x) {
-        const int n = n0 >> (q * LPL + x);
-        par[x] = (live && n >= 2) ? (n >> 1) : 0;
-        sk[x].v = TG_INF; sk[x].i = 0;
-        if (par[x]) {
-          const int sb = n ^ 1;
-          sk[x].i = sb >= H ? sb - H : (int)tree[sim_at(sb, s)];
+    for (int x = 0; x < 4; ++x) cur[x] = x == 0 ? J.first_dur : (x <= J.n_list ? J.lst[x - 1] : 0);
+    for (int k0 = 0; k0 < steps; k0 += 4) {
+#pragma unroll
+      for (int x = 0; x < 4; ++x) nxt[x] = (k0 + 4 + x <= J.n_list) ? J.lst[k0 + 3 + x] : 0;
+      i64 chunk = 0;                                   // four completions < 2^51: no overflow here
+#pragma unroll
+      for (int x4 = 0; x4 < 4; ++x4) {
+        if (k0 + x4 < steps) {
+          const u32 w = (u32)top & ((1u << SIM_SLOT_BITS) - 1u);
+          const i64 v = ((top >> SIM_SLOT_BITS) & ((1LL << 50) - 1)) + cur[x4];   // pop earliest, push ts + T
+          chunk += v;
+          ovf |= (u32)(v >> 32);
+          i64 c = SIM_KEY_BIAS | (v << SIM_SLOT_BITS) | (i64)w;
+          const u32 o0 = ((u32)H + w) << 8;            // byte offset of the leaf
+          sts64(base + o0, c);
+          i64 sk[MAXD]; u32 pa[MAXD];
+#pragma unroll
+          for (int x = 0; x < MAXD; ++x) {
+            pa[x] = base + ((o0 >> (x + 1)) & ~255u);  // parent of the level-x node
+            const u32 cu = base + ((o0 >> x) & ~255u); // the level-x node itself
+            sk[x] = lds64(cu ^ 256u);                  // its sibling (a harmless read beyond the root)
+          }
+#pragma unroll
+          for (int x = 0; x < MAXD; ++x) {
+            if ((o0 >> (x + 9)) != 0) {                // level-x node is not the root: n >= 2
+              c = key_min(c, sk[x]);
+              sts64(pa[x], c);
+            }
+          }
+          top = c;
         }
       }
+      tmp = sat_add(tmp, chunk);
 #pragma unroll
-      for (int x = 0; x < LPL; ++x) if (par[x]) sk[x].v = val[sim_at(sk[x].i, s)];
-      // minimum over this lane's levels, then exclusive prefix-minimum over the lanes below it
-      Key lm = sk[0];
-#pragma unroll
-      for (int x = 1; x < LPL; ++x) lm = key_min(lm, sk[x]);
-      Key pm = lm;
-#pragma unroll
-      for (int off = 1; off < SIM_G; off <<= 1) {
-        Key o;
-        o.v = __shfl_up_sync(TG_FULL, pm.v, off, SIM_G);
-        o.i = __shfl_up_sync(TG_FULL, pm.i, off, SIM_G);
-        if (q >= off) pm = key_min(pm, o);
-      }
-      Key ex;
-      ex.v = __shfl_up_sync(TG_FULL, pm.v, 1, SIM_G);
-      ex.i = __shfl_up_sync(TG_FULL, pm.i, 1, SIM_G);
-      Key c; c.v = v; c.i = w;
-      if (q > 0) c = key_min(c, ex);
-      // winners of this lane's levels, bottom up
-#pragma unroll
-      for (int x = 0; x < LPL; ++x) {
-        if (par[x]) {
-          c = key_min(c, sk[x]);
-          tree[sim_at(par[x], s)] = (u16)c.i;
-        }
-      }
-      // the top lane holds the new overall winner
-      const i64 nv = __shfl_sync(TG_FULL, c.v, SIM_G - 1, SIM_G);
-      const int ni = __shfl_sync(TG_FULL, c.i, SIM_G - 1, SIM_G);
-      if (live) { wv = nv; w = ni; }
-      d0 = d1; d1 = d2; d2 = d3;
-      __syncwarp();
+      for (int x = 0; x < 4; ++x) cur[x] = nxt[x];
     }
-    if (J.active && q == 0) atomicMin((u64*)&J.st->est[J.e], (u64)tmp);
+    if (ovf >> 17) { atomicOr(&J.st->flags, TS_REDO0 << J.e); L.count[63] = 1; }   // a completion >= 2^49
+    else J.st->est[J.e] = tmp;
   }
 }
 
-// One lane per simulation, trees in the arena: for H beyond the largest shared-memory class.
+// One lane per simulation, exact 64-bit values, trees in the arena: for H beyond the largest
+// shared-memory class and for simulations whose packed keys overflowed.
 __global__ void __launch_bounds__(32) k_sims_big(const __grid_constant__ Params P, TaskState* ts,
                                                  const i64* seed2, int hcap_lo, const int* any_big) {
   if (*any_big == 0) return;
   const int t = threadIdx.x;
-  const SimJob J = sim_job(P, ts, seed2, (long long)blockIdx.x * 32 + t);
+  SimJob J = sim_job(P, ts, seed2, (long long)blockIdx.x * 32 + t);
+  if (J.active && !(J.H > hcap_lo || (J.st->flags & (TS_REDO0 << J.e)))) J.active = false;
   const int hmax = warp_max32(J.active ? J.H : 0);
-  if (hmax <= hcap_lo) return;
+  if (hmax == 0) return;
   u64 off = 0;
   const u64 bytes = ((u64)hmax * 32 * (sizeof(i64) + 2 * sizeof(u32)) + 255) & ~(u64)255;
   if (t == 0) off = atomicAdd(P.arena_top, bytes);
   off = __shfl_sync(TG_FULL, off, 0);
   if (off + bytes > P.arena_bytes) { if (J.active) atomicOr(&J.st->flags, TS_FAILED); return; }
-  if (!J.active || J.H <= hcap_lo) return;
+  if (!J.active) return;
   i64* val = (i64*)(P.arena + off);
   u32* tree = (u32*)(P.arena + off + (u64)hmax * 32 * sizeof(i64));
   const int H = J.H;
@@ -262,5 +255,5 @@ __global__ void __launch_bounds__(32) k_sims_big(const __grid_constant__ Params 
     w = ci; wv = cv;
     dur = nxt;
   }
-  atomicMin((u64*)&J.st->est[J.e], (u64)tmp);
+  J.st->est[J.e] = tmp;
 }

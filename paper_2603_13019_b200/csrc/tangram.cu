@@ -310,9 +310,24 @@ static const char* const g_kernel_names[TG_N_KERNELS] = {"k_prefix", "k_select",
                                                           "k_solve", "k_sims", "k_finish"};
 // capacity classes (slots per simulation) of the shared-memory simulation kernels
 static const int g_sim_caps[TG_N_SIM_CLASSES] = {16, 32, 48, 64, 80, 96, 112, 128, 144, 160, 176, 192, 224, 256,
-                                                 320, 384, 512, 768, 1024, 1536, 2048, 2816};
+                                                 320, 352, 384, 400, 416, 432, 440, 448};
 #define TG_SMEM_PER_SM 233472   // shared memory an SM can split among resident blocks
 #define TG_SMEM_PER_BLOCK 232448
+
+typedef void (*sims_fn)(const Params, TaskState*, const i64*, const SimLists, int);
+// simulation kernel of a capacity class: path length bound = floor(log2(2 * cap - 1))
+static sims_fn sim_kernel(int cap) {
+  int d = 0;
+  while ((2 * cap - 1) >> (d + 1)) ++d;
+  switch (d) {
+    case 0: case 1: case 2: case 3: case 4: return k_sims1<4>;
+    case 5: return k_sims1<5>;
+    case 6: return k_sims1<6>;
+    case 7: return k_sims1<7>;
+    case 8: return k_sims1<8>;
+    default: return k_sims1<9>;
+  }
+}
 
 static cudaError_t fill_tables() {
   u64 recip[33];
@@ -417,7 +432,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc((void**)&r->W.seed2, SN * sizeof(i64)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.rs1, SN) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.rs2, SN) != cudaSuccess;
-  const long long n_sims = (long long)P.P * P.S * 2 * P.depth;
+  const long long n_sims = (long long)P.P * P.S * 2;
   r->sim_blocks = (int)((n_sims + 31) / 32);
   r->n_sm = prop.multiProcessorCount;
   r->L.n_groups = (int)((n_sims + SIM_PER_WARP - 1) / SIM_PER_WARP);
@@ -446,10 +461,9 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_prefix, cudaFuncAttributeMaxDynamicSharedMemorySize, P.V * K1_THREADS * 4);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_sims4<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_PER_BLOCK - 1024);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_sims4<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_PER_BLOCK - 1024);
+  for (int c = 0; c < TG_N_SIM_CLASSES && e == cudaSuccess; ++c)
+    e = cudaFuncSetAttribute(sim_kernel(g_sim_caps[c]), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             TG_SMEM_PER_BLOCK - 1024);
   if (e != cudaSuccess) { tangram_round_destroy(r); return cuda_fail(e, "cudaFuncSetAttribute"); }
   *out = r;
   return TANGRAM_OK;
@@ -590,14 +604,13 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   for (int c = 0; c < TG_N_SIM_CLASSES; ++c) {
     cudaStream_t ss = r->sim_stream[c];
     CK(cudaStreamWaitEvent(ss, r->sim_fork, 0));
-    const int smem = g_sim_caps[c] * SIM_PER_WARP * SIM_SLOT_BYTES;
+    const int smem = g_sim_caps[c] * SIM_PER_WARP * SIM_SLOT_BYTES + 512;
     int per_sm = TG_SMEM_PER_SM / (smem + 1024);
     if (per_sm > 32) per_sm = 32;
     if (per_sm < 1) per_sm = 1;
     int grid = r->n_sm * per_sm;
     if (grid > r->L.n_groups) grid = r->L.n_groups;
-    if (2 * g_sim_caps[c] <= 512) k_sims4<2><<<grid, 32, smem, ss>>>(P, r->W.ts, r->W.seed2, r->L, c);
-    else k_sims4<3><<<grid, 32, smem, ss>>>(P, r->W.ts, r->W.seed2, r->L, c);
+    sim_kernel(g_sim_caps[c])<<<grid, 32, smem, ss>>>(P, r->W.ts, r->W.seed2, r->L, c);
     CK(cudaEventRecord(r->sim_join[c], ss));
     CK(cudaStreamWaitEvent(st, r->sim_join[c], 0));
   }
