@@ -15,11 +15,16 @@
 // (k_m, ..., k_1) lexicographically smallest.
 #pragma once
 #include "common.cuh"
+#include "sims.cuh"
 
+// Scratch of one worker warp: a window of shared memory first (what is read over and over in
+// sequential loops belongs there), its slab in global memory once the window is full.
 struct Slab {
-  char* base; u64 cap; u64 used;
+  char* base; u64 cap; u64 used;          // global slab
+  char* fbase; u32 fcap; u32 fused;       // shared-memory window (generic address), may be empty
   __device__ __forceinline__ void* take(u64 bytes) {
     bytes = (bytes + 15) & ~(u64)15;
+    if (fused + bytes <= fcap) { void* p = fbase + fused; fused += (u32)bytes; return p; }
     if (used + bytes > cap) return nullptr;
     void* p = base + used; used += bytes; return p;
   }
@@ -51,6 +56,8 @@ struct PoolTask {
   // results: multiplicity per candidate of the prefix under evaluation / of the accepted one
   u8* rsel; u8* rkeep;
   int* rowcand;           // scratch, m ints
+  // shared memory of this warp for a winner tree (0 = none): address and capacity in slots
+  u32 sim_base; int sim_cap;
 };
 
 // extra demand, per chunk level, of multiplicity r over the least multiplicity r0
@@ -278,6 +285,25 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab sl
   else { fs = T.ac_first.s; fp = T.ac_first.p; fm = T.ac_first.mask; }
   const int dmax = min(min(T.depth, __popc(fm)), 32);
   const int H = T.n_seeds + q;
+  if (T.sim_base && H <= T.sim_cap) {
+    // one lane, one depth (the largest level tried is the best one), tree in shared memory
+    i64 val = 0; int bad = 0;
+    if (lane == 0) {
+      bool overflow;
+      const i64 fd = duration(fs, fp, nth_level_of(fm, dmax - 1));
+      val = tree_sim<9, 3>(
+          T.sim_base, H, n_rest,
+          [&](int i) { return i < T.n_seeds ? T.seeds[i]
+                                            : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], T.rsel[i - T.n_seeds]); },
+          [&](int k) { return k == 0 ? fd
+                            : (k < n_ev ? duration(T.cs[q + k], T.cp[q + k], __ffs(T.cmask[q + k])) : T.ac_tmin[k - n_ev]); },
+          &overflow);
+      bad = overflow;
+    }
+    __syncwarp();
+    bad = __shfl_sync(TG_FULL, bad, 0);
+    if (!bad) { *est = __shfl_sync(TG_FULL, val, 0); return true; }
+  }
   i64* heaps = (i64*)slab.take((u64)dmax * H * sizeof(i64));
   if (!heaps) heaps = (i64*)arena_take(P, (u64)dmax * H * sizeof(i64), lane);
   if (!heaps) return false;

@@ -138,10 +138,67 @@ __device__ __forceinline__ void sts64(u32 addr, i64 v) {
   asm volatile("st.shared.b64 [%0], %1;" :: "r"(addr), "l"(v) : "memory");
 }
 
-// One persistent warp per block, one lane per simulation; MAXD bounds the path length of the
-// class (2 * capacity <= 2^(MAXD+1)).  Node n of lane t is at shared address base + n * 256 with
-// base = (512-aligned start) + t * 8, so that with o = n * 256 the sibling of a node is at
-// (base + o) ^ 256 and the node offsets of a leaf-to-root path are (leaf offset >> level) & ~255.
+// One whole simulation on a winner tree in shared memory, run by the calling lane alone.
+// Node n is at shared address base + (n << SS); base must be a multiple of 2 << SS plus an offset
+// below 1 << SS, so that with o = n << SS the sibling of a node is at (base + o) ^ (1 << SS) and
+// the node offsets of a leaf-to-root path are (leaf offset >> level) & ~((1 << SS) - 1).
+// MAXD bounds the path length (2 * H <= 2^(MAXD+1)).  seed(i) gives slot i's first completion,
+// dur(k) the duration of the k-th remaining action, k = 0 .. steps-1.  Returns the estimate
+// (saturating sum of completions); *overflow tells that a completion reached 2^49 and the
+// packed keys cannot be trusted.
+template <int MAXD, int SS, class SeedFn, class DurFn>
+__device__ __forceinline__ i64 tree_sim(u32 base, int H, int steps, SeedFn seed, DurFn dur, bool* overflow) {
+  const u32 NM = ~((1u << SS) - 1u);
+  for (int i = 0; i < H; ++i) sts64(base + ((u32)(H + i) << SS), SIM_KEY_BIAS | (seed(i) << SIM_SLOT_BITS) | i);
+  for (int n = H - 1; n >= 1; --n)
+    sts64(base + ((u32)n << SS), key_min(lds64(base + ((u32)(2 * n) << SS)), lds64(base + ((u32)(2 * n + 1) << SS))));
+  i64 top = lds64(base + ((u32)(H > 1 ? 1 : H) << SS));   // key of the earliest completion
+  i64 tmp = 0;
+  u32 ovf = 0;
+  // durations are fetched a chunk of four ahead
+  i64 cur[4], nxt[4];
+#pragma unroll
+  for (int x = 0; x < 4; ++x) cur[x] = x < steps ? dur(x) : 0;
+  for (int k0 = 0; k0 < steps; k0 += 4) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) nxt[x] = (k0 + 4 + x < steps) ? dur(k0 + 4 + x) : 0;
+    i64 chunk = 0;                                     // four completions < 2^51: no overflow here
+#pragma unroll
+    for (int x4 = 0; x4 < 4; ++x4) {
+      if (k0 + x4 < steps) {
+        const u32 w = (u32)top & ((1u << SIM_SLOT_BITS) - 1u);
+        const i64 v = ((top >> SIM_SLOT_BITS) & ((1LL << 50) - 1)) + cur[x4];   // pop earliest, push ts + T
+        chunk += v;
+        ovf |= (u32)(v >> 32);
+        i64 c = SIM_KEY_BIAS | (v << SIM_SLOT_BITS) | (i64)w;
+        const u32 o0 = ((u32)H + w) << SS;             // byte offset of the leaf
+        sts64(base + o0, c);
+        i64 sk[MAXD]; u32 pa[MAXD];
+#pragma unroll
+        for (int x = 0; x < MAXD; ++x) {
+          pa[x] = base + ((o0 >> (x + 1)) & NM);       // parent of the level-x node
+          const u32 cu = base + ((o0 >> x) & NM);      // the level-x node itself
+          sk[x] = lds64(cu ^ (1u << SS));              // its sibling (a harmless read beyond the root)
+        }
+#pragma unroll
+        for (int x = 0; x < MAXD; ++x) {
+          if ((o0 >> (x + SS + 1)) != 0) {             // level-x node is not the root: n >= 2
+            c = key_min(c, sk[x]);
+            sts64(pa[x], c);
+          }
+        }
+        top = c;
+      }
+    }
+    tmp = sat_add(tmp, chunk);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) cur[x] = nxt[x];
+  }
+  *overflow = (ovf >> 17) != 0;                        // a completion >= 2^49
+  return tmp;
+}
+
+// One persistent warp per block, one lane per simulation (trees interleaved by lane: SS = 8).
 template <int MAXD>
 __global__ void __launch_bounds__(32) k_sims1(const __grid_constant__ Params P, TaskState* ts, const i64* seed2,
                                               const SimLists L, int cls) {
@@ -157,54 +214,11 @@ __global__ void __launch_bounds__(32) k_sims1(const __grid_constant__ Params P, 
     const int grp = L.list[(size_t)cls * L.n_groups + gi];
     const SimJob J = sim_job(P, ts, seed2, (long long)grp * SIM_PER_WARP + lane);
     if (!J.active) continue;                           // lanes are independent: no warp-wide step below
-    const int H = J.H;
-    for (int i = 0; i < H; ++i) sts64(base + (u32)(H + i) * 256u, SIM_KEY_BIAS | (J.seeds[i] << SIM_SLOT_BITS) | i);
-    for (int n = H - 1; n >= 1; --n)
-      sts64(base + (u32)n * 256u, key_min(lds64(base + (u32)(2 * n) * 256u), lds64(base + (u32)(2 * n + 1) * 256u)));
-    i64 top = lds64(base + (u32)(H > 1 ? 1 : H) * 256u);   // key of the earliest completion
-    i64 tmp = 0;
-    u32 ovf = 0;
-    // durations are fetched a chunk of four ahead (stream[0] = first action, then the list)
-    const int steps = J.n_list + 1;
-    i64 cur[4], nxt[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) cur[x] = x == 0 ? J.first_dur : (x <= J.n_list ? J.lst[x - 1] : 0);
-    for (int k0 = 0; k0 < steps; k0 += 4) {
-#pragma unroll
-      for (int x = 0; x < 4; ++x) nxt[x] = (k0 + 4 + x <= J.n_list) ? J.lst[k0 + 3 + x] : 0;
-      i64 chunk = 0;                                   // four completions < 2^51: no overflow here
-#pragma unroll
-      for (int x4 = 0; x4 < 4; ++x4) {
-        if (k0 + x4 < steps) {
-          const u32 w = (u32)top & ((1u << SIM_SLOT_BITS) - 1u);
-          const i64 v = ((top >> SIM_SLOT_BITS) & ((1LL << 50) - 1)) + cur[x4];   // pop earliest, push ts + T
-          chunk += v;
-          ovf |= (u32)(v >> 32);
-          i64 c = SIM_KEY_BIAS | (v << SIM_SLOT_BITS) | (i64)w;
-          const u32 o0 = ((u32)H + w) << 8;            // byte offset of the leaf
-          sts64(base + o0, c);
-          i64 sk[MAXD]; u32 pa[MAXD];
-#pragma unroll
-          for (int x = 0; x < MAXD; ++x) {
-            pa[x] = base + ((o0 >> (x + 1)) & ~255u);  // parent of the level-x node
-            const u32 cu = base + ((o0 >> x) & ~255u); // the level-x node itself
-            sk[x] = lds64(cu ^ 256u);                  // its sibling (a harmless read beyond the root)
-          }
-#pragma unroll
-          for (int x = 0; x < MAXD; ++x) {
-            if ((o0 >> (x + 9)) != 0) {                // level-x node is not the root: n >= 2
-              c = key_min(c, sk[x]);
-              sts64(pa[x], c);
-            }
-          }
-          top = c;
-        }
-      }
-      tmp = sat_add(tmp, chunk);
-#pragma unroll
-      for (int x = 0; x < 4; ++x) cur[x] = nxt[x];
-    }
-    if (ovf >> 17) { atomicOr(&J.st->flags, TS_REDO0 << J.e); L.count[63] = 1; }   // a completion >= 2^49
+    bool overflow;
+    const i64 tmp = tree_sim<MAXD, 8>(
+        base, J.H, J.n_list + 1, [&](int i) { return J.seeds[i]; },
+        [&](int k) { return k == 0 ? J.first_dur : J.lst[k - 1]; }, &overflow);
+    if (overflow) { atomicOr(&J.st->flags, TS_REDO0 << J.e); L.count[63] = 1; }
     else J.st->est[J.e] = tmp;
   }
 }

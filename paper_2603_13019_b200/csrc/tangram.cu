@@ -9,9 +9,9 @@
 #include "../../include/tangram.h"
 #include "common.cuh"
 #include "prefix_kernel.cuh"
+#include "sims.cuh"
 #include "select.cuh"
 #include "place.cuh"
-#include "sims.cuh"
 
 #define K2_THREADS 256
 #define TG_PROF_CALLS 256   // calls whose kernels can be timed between two queries
@@ -91,6 +91,30 @@ __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, co
   T.seeds = nullptr; T.n_seeds = 0;
   T.depth = P.depth;
   T.rsel = C.rsel; T.rkeep = C.rkeep; T.rowcand = C.rowcand;
+  T.sim_base = 0; T.sim_cap = 0;
+}
+
+// shared memory of the calling warp for winner trees inside the per-pool kernels
+#define WARP_TREE_SLOTS 448
+#define WARP_TREE_BYTES (WARP_TREE_SLOTS * 16)
+#define WARP_FAST_BYTES 0
+#define WARP_SMEM_BYTES (WARP_TREE_BYTES + WARP_FAST_BYTES)
+#define K2_DYN_SMEM ((K2_THREADS / 32) * WARP_SMEM_BYTES + 16)
+__device__ __forceinline__ void attach_warp_tree(PoolTask& T) {
+  extern __shared__ __align__(16) unsigned char k2_smem[];
+  const u32 start = ((u32)__cvta_generic_to_shared(k2_smem) + 15u) & ~15u;
+  T.sim_base = start + (threadIdx.x >> 5) * WARP_SMEM_BYTES;
+  T.sim_cap = WARP_TREE_SLOTS;
+}
+// the calling warp's scratch: shared-memory window behind its tree area, then its global slab
+__device__ __forceinline__ Slab warp_slab(const Params& P, int gw) {
+  extern __shared__ __align__(16) unsigned char k2_smem[];
+  Slab s;
+  s.base = P.slabs + (u64)gw * P.slab_bytes; s.cap = P.slab_bytes; s.used = 0;
+  const u64 start = ((u64)k2_smem + 15u) & ~(u64)15;
+  s.fbase = (char*)start + (threadIdx.x >> 5) * WARP_SMEM_BYTES + WARP_TREE_BYTES;
+  s.fcap = WARP_FAST_BYTES; s.fused = 0;
+  return s;
 }
 
 // placement on a fresh copy of the pool's topology state, then the candidates' outputs
@@ -153,6 +177,7 @@ __device__ void run_pool_task(const Params& P, int sc, int j, Slab slab, int lan
   if (mt.elastic) {
     PoolTask T;
     make_task(P, sc, j, mt, C, lane, T);
+    attach_warp_tree(T);
     keep = evict_loop(P, T, slab, lane);
     if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
   }
@@ -163,8 +188,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ P
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
   const int nw = (gridDim.x * K2_THREADS) >> 5;
-  Slab slab;
-  slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
+  const Slab slab = warp_slab(P, gw);
   const int n_tasks = P.S * P.P;
   (void)nw;
   for (;;) {
@@ -195,8 +219,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Pa
     const PoolMeta mt = P.meta[task];
     TaskState* st = W.ts + task;
     if (mt.m == 0 || !mt.elastic) { if (lane == 0) st->flags = 0; continue; }
-    Slab slab;
-    slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
+    Slab slab = warp_slab(P, gw);
     CandArrays C;
     bool ok = gather_candidates(P, sc, j, mt, slab, lane, C);
     i64 opt0 = 0, opt1 = 0;
@@ -242,8 +265,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ P
     const int sc = x % P.S, j = x / P.S, task = sc * P.P + j;
     const PoolMeta mt = P.meta[task];
     if (mt.m == 0) continue;
-    Slab slab;
-    slab.base = P.slabs + (u64)gw * P.slab_bytes; slab.cap = P.slab_bytes; slab.used = 0;
+    Slab slab = warp_slab(P, gw);
     CandArrays C;
     if (!gather_candidates(P, sc, j, mt, slab, lane, C)) {
       if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE);
@@ -264,6 +286,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ P
             __syncwarp();
             PoolTask T;
             make_task(P, sc, j, mt, C, lane, T);
+            attach_warp_tree(T);
             keep = evict_resume(P, T, slab, lane, nobj, mt.m - 1);
           }
         }
@@ -461,6 +484,8 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_prefix, cudaFuncAttributeMaxDynamicSharedMemorySize, P.V * K1_THREADS * 4);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   for (int c = 0; c < TG_N_SIM_CLASSES && e == cudaSuccess; ++c)
     e = cudaFuncSetAttribute(sim_kernel(g_sim_caps[c]), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TG_SMEM_PER_BLOCK - 1024);
@@ -596,7 +621,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   if (ev) CK(cudaEventRecord(ev[0], st));
   k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
   if (ev) CK(cudaEventRecord(ev[1], st));
-  k_solve<<<wblocks, K2_THREADS, 0, st>>>(P, r->W);
+  k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, r->W);
   if (ev) CK(cudaEventRecord(ev[2], st));
   CK(cudaMemsetAsync(r->L.count, 0, 2 * 64 * sizeof(int), st));
   k_sim_classify<<<(r->L.n_groups + 255) / 256, 256, 0, st>>>(P, r->W.ts, r->L);
@@ -616,7 +641,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   }
   k_sims_big<<<r->sim_blocks, 32, 0, st>>>(P, r->W.ts, r->W.seed2, g_sim_caps[TG_N_SIM_CLASSES - 1], r->L.count + 63);
   if (ev) CK(cudaEventRecord(ev[3], st));
-  k_finish<<<wblocks, K2_THREADS, 0, st>>>(P, r->W);
+  k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, r->W);
   if (ev) CK(cudaEventRecord(ev[4], st));
   r->launches += 5 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
@@ -723,7 +748,8 @@ extern "C" int tangram_schedule_batch_static(const tangram_round_desc* desc, con
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CK(cudaMemsetAsync(P.arena_top, 0, 256, st));           // the only part that must start at zero
   k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
-  k_select<<<P.n_workers / wpb, K2_THREADS, 0, st>>>(P);
+  CK(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM));
+  k_select<<<P.n_workers / wpb, K2_THREADS, K2_DYN_SMEM, st>>>(P);
   CK(cudaGetLastError());
   return TANGRAM_OK;
 }
