@@ -33,17 +33,13 @@ __device__ __forceinline__ void k1_scan_columns(int* sm, int* carry, int* wsum, 
     sm[v * K1_THREADS + t] = incl - x;                 // exclusive within the warp
   }
   __syncthreads();
-  for (int v = 0; v < V; ++v) {
-    int add = carry[v];
-    for (int w = 0; w < warp; ++w) add += wsum[w * K1_MAXV + v];
-    sm[v * K1_THREADS + t] += add;
+  if (t < V) {                                         // warp totals -> offsets of the warps, new carry
+    int acc = carry[t];
+    for (int w = 0; w < K1_THREADS / 32; ++w) { int x = wsum[w * K1_MAXV + t]; wsum[w * K1_MAXV + t] = acc; acc += x; }
+    carry[t] = acc;
   }
   __syncthreads();
-  if (t < V) {
-    int tot = carry[t];
-    for (int w = 0; w < K1_THREADS / 32; ++w) tot += wsum[w * K1_MAXV + t];
-    carry[t] = tot;
-  }
+  for (int v = 0; v < V; ++v) sm[v * K1_THREADS + t] += wsum[warp * K1_MAXV + v];
 }
 
 __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ Params P) {
@@ -53,6 +49,7 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
   __shared__ int s_wsum[(K1_THREADS / 32) * K1_MAXV];
   __shared__ int s_tot[TG_MAX_POOLS], s_base[TG_MAX_POOLS], s_m[TG_MAX_POOLS];
   __shared__ int s_n, s_bad, s_el;
+  __shared__ u32 s_pinfo[TG_MAX_POOLS];             // type | GPUs per node << 4 | slot0 << 8
 
   const int sc = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
   const size_t row = (size_t)sc * P.N;
@@ -64,7 +61,11 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
                    ((((size_t)P.a_pool | (size_t)P.a_unit | (size_t)P.a_mask | (size_t)P.a_s | (size_t)P.a_p |
                       (size_t)P.o_alloc | (size_t)P.o_node | (size_t)P.o_off | (size_t)P.o_act) & 15) == 0);
 
-  if (t < TG_MAX_POOLS) { s_tot[t] = 0; s_m[t] = 0; s_base[t] = 0; }
+  if (t < TG_MAX_POOLS) {
+    s_tot[t] = 0; s_m[t] = 0; s_base[t] = 0;
+    s_pinfo[t] = t < P.P ? (u32)P.pool[t].type | ((u32)(P.pool[t].type == TG_POOL_GPU ? P.pool[t].group : 0) << 4) |
+                                ((u32)P.pool[t].slot0 << 8) : 0u;
+  }
   if (t < K1_MAXV) s_carry[t] = 0;
   if (t == 0) { s_n = INT_MAX; s_bad = 0; s_el = 0; }
   if (warp < P.P) {                                 // free capacity of every demand slot
@@ -137,7 +138,10 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
         if (i < n_act) {
           const int j = rp[kk];
           if (j >= P.P) { bad = true; continue; }
-          const PoolDev& pd = P.pool[j];
+          const u32 pi = s_pinfo[j];
+          PoolDev pd;
+          pd.type = pi & 15; pd.group = (pi >> 4) & 15;
+          const int slot0 = pi >> 8;
           int g, gang; u32 eff;
           if (!decode_levels(pd, ru[kk], rm[kk], g, gang, eff)) { bad = true; continue; }
           const int rmin = __ffs(eff);
@@ -147,7 +151,7 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
           tm[kk] = duration(clamp_param(sv[h]), clamp_param(pv[h]), rmin);
           sm[(D + j) * K1_THREADS + t] += 1;
           if (!found_before)
-            for (int l = 0; l <= lz; ++l) sm[(pd.slot0 + l) * K1_THREADS + t] += units;
+            for (int l = 0; l <= lz; ++l) sm[(slot0 + l) * K1_THREADS + t] += units;
         }
       }
     }
@@ -165,11 +169,11 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
       for (int k = 0; k < K1_ITEMS; ++k) {
         if (!(info[k] & 16u)) continue;
         const int j = info[k] & 15, lz = (info[k] >> 6) & 3, units = (info[k] >> 8) & 0x1fff;
-        const PoolDev& pd = P.pool[j];
+        const int slot0 = s_pinfo[j] >> 8;
         bool over = false;
         for (int l = 0; l <= lz; ++l) {
-          int d = (sm[(pd.slot0 + l) * K1_THREADS + t] += units);
-          over |= d > s_cap[pd.slot0 + l];
+          int d = (sm[(slot0 + l) * K1_THREADS + t] += units);
+          over |= d > s_cap[slot0 + l];
         }
         if (over) atomicMin(&s_n, i_first + k);
       }
@@ -187,9 +191,6 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
     if (el_mask) atomicOr(&s_el, (int)el_mask);
     __syncthreads();
     const u32 need = one_tile ? (u32)s_el : 0xffu;
-    int cand_cnt[TG_MAX_POOLS];
-#pragma unroll
-    for (int j = 0; j < TG_MAX_POOLS; ++j) cand_cnt[j] = 0;
 #pragma unroll
     for (int k = 0; k < K1_ITEMS; ++k) {
       if (!(info[k] & 16u)) continue;
@@ -198,8 +199,7 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
       const size_t part = row + s_base[j] + pos;
       if (i < n) {
         P.order[part] = i;
-#pragma unroll
-        for (int jj = 0; jj < TG_MAX_POOLS; ++jj) cand_cnt[jj] += jj == j;
+        atomicAdd(&s_m[j], 1);
       } else if ((need >> j) & 1u) {
         P.tmin[part] = tm[k];
         // the first waiting action of a pool is looked up by position; it sits right behind the
@@ -208,9 +208,6 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
         P.order[part] = i;
       }
     }
-#pragma unroll
-    for (int j = 0; j < TG_MAX_POOLS; ++j)
-      if (cand_cnt[j]) atomicAdd(&s_m[j], cand_cnt[j]);
     // "not scheduled" outputs of everything behind the prefix (candidates are written later)
     if (full && i_first >= n) {
       const int4 z = make_int4(0, 0, 0, 0), m1 = make_int4(-1, -1, -1, -1);
