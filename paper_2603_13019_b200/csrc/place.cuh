@@ -26,8 +26,9 @@ __device__ __forceinline__ int find_block(u32 busy, int bl, int group) {
 }
 
 // nm: node busy masks of the pool (updated).  keep candidates, multiplicities r[].
+// owner (may be null): one entry per GPU of the pool, receives ids[i] for every GPU granted.
 __device__ void place_gpu(const PoolDev& pd, u8* nm, int keep, const u8* cg, const u8* r,
-                          int* pnode, int* poff, int lane) {
+                          int* pnode, int* poff, int lane, int* owner = nullptr, const int* ids = nullptr) {
   const int top = ilog2(pd.group);
   const u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;
   for (int lz = top; lz >= 0; --lz) {
@@ -50,6 +51,7 @@ __device__ void place_gpu(const PoolDev& pd, u8* nm, int keep, const u8* cg, con
         if (lane == 0) {
           nm[node] |= (u8)(((1u << z) - 1u) << start);
           if (rep == 0) { pnode[i] = node; poff[i] = start; }
+          if (owner) for (int b = 0; b < z; ++b) owner[node * pd.group + start + b] = ids[i];
         }
         __syncwarp();
       }
@@ -128,5 +130,36 @@ __device__ void place_cpu_fresh(const PoolDev& pd, int* dfree, int keep, const u
       }
       __syncwarp();
     }
+  }
+}
+
+// CPU placement on a pool with cores in use (trace replay): owner[c] < 0 marks a free core,
+// dfree the free cores per domain.  Same rule as place_cpu; a grant writes ids[i] into owner.
+__device__ void place_cpu_owner(const PoolDev& pd, int* owner, int* dfree, int keep, const u8* cg,
+                                const u8* r, const int* ids, int* pnode, int* poff, int lane) {
+  const int D = pd.capacity / pd.group;
+  for (int i = 0; i < keep; ++i) {
+    const int k = (cg[i] & 0x7f) * r[i];
+    i64 key = TG_INF;
+    for (int d = lane; d < D; d += 32) {
+      int f = dfree[d];
+      if (f >= k) key = min(key, ((i64)f << 32) | d);
+    }
+    key = warp_min64(key);
+    int lo = 0, hi = pd.capacity;
+    if (key != TG_INF) { int d = (int)(key & 0xffffffff); lo = d * pd.group; hi = lo + pd.group; }
+    // lowest free cores of [lo, hi): 32 cores per pass, each lane claims by its rank among the free
+    int need = k, first = -1;
+    for (int c0 = lo; c0 < hi && need > 0; c0 += 32) {
+      const int c = c0 + lane;
+      const bool fr = c < hi && owner[c] < 0;
+      const u32 b = __ballot_sync(TG_FULL, fr);
+      const int rank = __popc(b & ((1u << lane) - 1u));
+      if (fr && rank < need) { owner[c] = ids[i]; atomicSub(&dfree[c / pd.group], 1); }
+      if (b && first < 0) first = c0 + __ffs(b) - 1;
+      need -= min(need, __popc(b));
+    }
+    if (lane == 0) { pnode[i] = first >= 0 ? first / pd.group : -1; poff[i] = first; }
+    __syncwarp();
   }
 }

@@ -1,0 +1,383 @@
+// Device-resident trace replay (workflow of Section 3: submit, queue, schedule, execute,
+// return), one warp per scenario, no host round trips.  Every round at now = r * round_us
+//   1. refills quota pools whose window changed (Section 5.1),
+//   2. releases what has finished (cores, chunks, concurrency slots),
+//   3. admits the actions that have arrived to the waiting queue,
+//   4. runs the scheduler of Algorithm 1 on the queue with the running actions of a pool in
+//      its completion heap (Algorithm 2), using the same per-pool routines as a single round,
+//   5. starts what was selected and records the occupancy.
+// Rounds with an empty queue are skipped ahead to the next arrival or completion (their
+// occupancy rows are still written).
+#pragma once
+#include "common.cuh"
+#include "sims.cuh"
+#include "select.cuh"
+#include "place.cuh"
+
+struct ReplayWs {
+  int* wait;        // [S][N] waiting actions in queue order
+  int* run;         // [S][N] running actions
+  int* owner;       // [S][U]  action holding each core / GPU (-1 free, -2 occupied beforehand)
+  u8* nm;           // [S][nodes] GPU busy masks
+  int* dfree;       // [S][Dtot] free cores per NUMA domain
+  int* pst;         // [S][P][2] quota used in the window / concurrency slots in use
+  i64* win;         // [S][P] current quota window
+  int unit0[TG_MAX_POOLS], dom0[TG_MAX_POOLS];   // first unit / domain of every pool in a row
+  int U, Dtot;
+  i64 round_us; int max_rounds;
+  int* occupancy; int* rounds_used;
+};
+
+__device__ __forceinline__ int pool_busy_units(const Params& P, const ReplayWs& R, int sc, int j, int lane) {
+  const PoolDev& pd = P.pool[j];
+  int b = 0;
+  if (pd.type == TG_POOL_API) b = pd.window_us > 0 ? R.pst[((size_t)sc * P.P + j) * 2] : R.pst[((size_t)sc * P.P + j) * 2 + 1];
+  else {
+    const int* ow = R.owner + (size_t)sc * R.U + R.unit0[j];
+    for (int c = lane; c < pd.capacity; c += 32) b += ow[c] != -1;
+    b = warp_sum32(b);
+  }
+  return b;
+}
+
+// Candidate prefix of the waiting queue (Algorithm 1, line 2) against the pools' current state.
+// dem / cap: 4 ints per pool in the warp's scratch.  Warp-uniform result.
+__device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const int* wait, int nw,
+                             int* dem, int* cap, int lane) {
+  const size_t row = (size_t)sc * P.N;
+  for (int j = 0; j < P.P; ++j) {
+    const PoolDev& pd = P.pool[j];
+    int c[4] = {0, 0, 0, 0};
+    if (pd.type == TG_POOL_GPU) gpu_caps(pd, R.nm + (size_t)sc * P.n_nodes_total, lane, c);
+    else if (pd.type == TG_POOL_CPU) {
+      int f = 0;
+      for (int d = lane; d < pd.capacity / pd.group; d += 32) f += R.dfree[(size_t)sc * R.Dtot + R.dom0[j] + d];
+      c[0] = warp_sum32(f);
+    } else {
+      const int* ps = R.pst + ((size_t)sc * P.P + j) * 2;
+      c[0] = pd.capacity - (pd.window_us > 0 ? ps[0] : ps[1]);
+    }
+    if (lane < 4) { cap[j * 4 + lane] = c[lane]; dem[j * 4 + lane] = 0; }
+  }
+  __syncwarp();
+  int n = 0;
+  bool stop = false;
+  for (int i0 = 0; i0 < nw && !stop; i0 += 32) {
+    // every lane decodes one waiting action, then the 32 are admitted one after the other
+    int j = 0, lz = 0, units = 0;
+    if (i0 + lane < nw) {
+      const int a = wait[i0 + lane];
+      j = P.a_pool[row + a];
+      int g, gang; u32 eff;
+      decode_levels(P.pool[j], P.a_unit[row + a], P.a_mask[row + a], g, gang, eff);
+      const int rmin = __ffs(eff);
+      units = g * rmin;
+      lz = P.pool[j].type == TG_POOL_GPU ? level_of(g, gang, rmin) : 0;
+    }
+    const int nb = min(32, nw - i0);
+    for (int b = 0; b < nb; ++b) {
+      const int bj = __shfl_sync(TG_FULL, j, b), bl = __shfl_sync(TG_FULL, lz, b), bu = __shfl_sync(TG_FULL, units, b);
+      bool over = false;
+      for (int l = 0; l <= bl; ++l) over |= dem[bj * 4 + l] + bu > cap[bj * 4 + l];
+      if (over) { stop = true; break; }
+      __syncwarp();
+      if (lane <= bl) dem[bj * 4 + lane] += bu;
+      __syncwarp();
+      ++n;
+    }
+  }
+  return n;
+}
+
+// One pool of one replay round: selection among the pool's candidates (the first n waiting
+// actions that sit on pool j), placement on the pool's live state, start of what was selected.
+// Appends the started actions to run[] (nr updated).  Returns false if the scratch ran out.
+__device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, const int* wait, int nw, int n,
+                            int* run, int& nr, i64 now, Slab slab, int lane) {
+  const size_t row = (size_t)sc * P.N;
+  const PoolDev& pd = P.pool[j];
+  // members of the pool among the candidates (m) and behind them (n_ac)
+  int m = 0, n_ac = 0;
+  for (int i0 = 0; i0 < nw; i0 += 32) {
+    const int i = i0 + lane;
+    const bool mine = i < nw && P.a_pool[row + wait[i]] == j;
+    m += __popc(__ballot_sync(TG_FULL, mine && i < n));
+    n_ac += __popc(__ballot_sync(TG_FULL, mine && i >= n));
+  }
+  if (m == 0) return true;
+  CandArrays C;
+  C.cs = (i64*)slab.take((u64)m * 8); C.cp = (i64*)slab.take((u64)m * 8);
+  C.cmask = (u32*)slab.take((u64)m * 4); C.cidx = (int*)slab.take((u64)m * 4);
+  C.pnode = (int*)slab.take((u64)m * 4); C.poff = (int*)slab.take((u64)m * 4);
+  C.rowcand = (int*)slab.take((u64)m * 4);
+  C.cg = (u8*)slab.take(m); C.rsel = (u8*)slab.take(m); C.rkeep = (u8*)slab.take(m);
+  i64* ac_tmin = (i64*)slab.take((u64)(n_ac + 1) * 8);
+  i64* seeds = (i64*)slab.take((u64)(nr + 1) * 8);
+  if (!seeds) return false;
+  // fill them in queue order
+  int cm = 0, ca = 0, first_ac = -1;
+  bool elastic = false;
+  for (int i0 = 0; i0 < nw; i0 += 32) {
+    const int i = i0 + lane;
+    int a = -1; bool mine = false;
+    if (i < nw) { a = wait[i]; mine = P.a_pool[row + a] == j; }
+    const u32 bc = __ballot_sync(TG_FULL, mine && i < n), ba = __ballot_sync(TG_FULL, mine && i >= n);
+    if (mine) {
+      int g, gang; u32 eff;
+      decode_levels(pd, P.a_unit[row + a], P.a_mask[row + a], g, gang, eff);
+      const i64 s = clamp_param(P.a_s[row + a]), p = clamp_param(P.a_p[row + a]);
+      if (i < n) {
+        const int k = cm + __popc(bc & ((1u << lane) - 1u));
+        C.cidx[k] = a; C.cmask[k] = eff; C.cg[k] = (u8)(g | (gang << 7)); C.cs[k] = s; C.cp[k] = p;
+        C.rkeep[k] = (u8)__ffs(eff); C.pnode[k] = -1; C.poff[k] = -1;
+        elastic |= (eff & (eff - 1)) != 0;
+      } else {
+        ac_tmin[ca + __popc(ba & ((1u << lane) - 1u))] = duration(s, p, __ffs(eff));
+      }
+    }
+    if (first_ac < 0 && ba) first_ac = __shfl_sync(TG_FULL, a, __ffs(ba) - 1);
+    cm += __popc(bc); ca += __popc(ba);
+  }
+  elastic = __any_sync(TG_FULL, elastic);
+  // completion times (relative to now) of what runs on this pool seed the heap
+  int ns = 0;
+  for (int i0 = 0; i0 < nr; i0 += 32) {
+    const int i = i0 + lane;
+    int a = -1; bool mine = false;
+    if (i < nr) { a = run[i]; mine = P.a_pool[row + a] == j; }
+    const u32 b = __ballot_sync(TG_FULL, mine);
+    if (mine) {
+      const i64 fin = (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a];
+      seeds[ns + __popc(b & ((1u << lane) - 1u))] = fin > now ? fin - now : 0;
+    }
+    ns += __popc(b);
+  }
+  __syncwarp();
+  int keep = m;
+  if (elastic) {
+    PoolTask T;
+    T.type = pd.type; T.group = pd.group;
+    T.cap[0] = T.cap[1] = T.cap[2] = T.cap[3] = 0;
+    if (pd.type == TG_POOL_GPU) gpu_caps(pd, R.nm + (size_t)sc * P.n_nodes_total, lane, T.cap);
+    else if (pd.type == TG_POOL_CPU) {
+      int f = 0;
+      for (int d = lane; d < pd.capacity / pd.group; d += 32) f += R.dfree[(size_t)sc * R.Dtot + R.dom0[j] + d];
+      T.cap[0] = warp_sum32(f);
+    } else {
+      const int* ps = R.pst + ((size_t)sc * P.P + j) * 2;
+      T.cap[0] = pd.capacity - (pd.window_us > 0 ? ps[0] : ps[1]);
+    }
+    T.m = m; T.cs = C.cs; T.cp = C.cp; T.cmask = C.cmask; T.cg = C.cg;
+    T.n_ac = n_ac; T.ac_tmin = ac_tmin;
+    T.ac_first.s = T.ac_first.p = 0; T.ac_first.mask = 1; T.ac_first.g = 1; T.ac_first.gang = 0;
+    if (n_ac > 0) {
+      decode_levels(pd, P.a_unit[row + first_ac], P.a_mask[row + first_ac], T.ac_first.g, T.ac_first.gang, T.ac_first.mask);
+      T.ac_first.s = clamp_param(P.a_s[row + first_ac]); T.ac_first.p = clamp_param(P.a_p[row + first_ac]);
+    }
+    T.seeds = seeds; T.n_seeds = ns;
+    T.depth = P.depth;
+    T.rsel = C.rsel; T.rkeep = C.rkeep; T.rowcand = C.rowcand;
+    T.sim_base = 0; T.sim_cap = 0;
+    attach_warp_tree(T);
+    keep = evict_loop(P, T, slab, lane);
+    if (keep < 0) return false;
+  }
+  // placement on the pool's live state
+  if (pd.type == TG_POOL_GPU) {
+    place_gpu(pd, R.nm + (size_t)sc * P.n_nodes_total + pd.node0, keep, C.cg, C.rkeep, C.pnode, C.poff, lane,
+              R.owner + (size_t)sc * R.U + R.unit0[j], C.cidx);
+  } else if (pd.type == TG_POOL_CPU) {
+    place_cpu_owner(pd, R.owner + (size_t)sc * R.U + R.unit0[j], R.dfree + (size_t)sc * R.Dtot + R.dom0[j],
+                    keep, C.cg, C.rkeep, C.cidx, C.pnode, C.poff, lane);
+  } else {
+    if (lane == 0) {
+      int* ps = R.pst + ((size_t)sc * P.P + j) * 2 + (pd.window_us > 0 ? 0 : 1);
+      for (int i = 0; i < keep; ++i) { C.pnode[i] = 0; C.poff[i] = *ps; *ps += (C.cg[i] & 0x7f) * C.rkeep[i]; }
+    }
+  }
+  __syncwarp();
+  // start what was selected (Eq. 2: completion - arrival = waited so far + execution)
+  i64 tot = 0;
+  for (int i = lane; i < keep; i += 32) {
+    const size_t o = row + C.cidx[i];
+    const int r = C.rkeep[i];
+    const i64 act = (now - (P.a_arrival ? P.a_arrival[o] : 0)) + duration(C.cs[i], C.cp[i], r);
+    P.o_alloc[o] = (C.cg[i] & 0x7f) * r; P.o_node[o] = C.pnode[i]; P.o_off[o] = C.poff[i]; P.o_act[o] = act;
+    run[nr + i] = C.cidx[i];
+    tot += act;
+  }
+  tot = warp_sum64(tot);
+  if (lane == 0) { P.o_total[sc] += tot; P.o_nsel[sc] += keep; }
+  nr += keep;
+  __syncwarp();
+  return true;
+}
+
+__global__ void __launch_bounds__(K2_THREADS) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
+  const int lane = threadIdx.x & 31;
+  const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
+  const int nw_warps = (gridDim.x * K2_THREADS) >> 5;
+  for (int sc = gw; sc < P.S; sc += nw_warps) {
+    const size_t row = (size_t)sc * P.N;
+    const int n_act = min(max(P.n_actions[sc], 0), P.N);
+    int* wait = R.wait + row; int* run = R.run + row;
+    int* owner = R.owner + (size_t)sc * R.U;
+    u8* nm = R.nm + (size_t)sc * P.n_nodes_total;
+    int* dfree = R.dfree + (size_t)sc * R.Dtot;
+    int* occ = R.occupancy ? R.occupancy + (size_t)sc * R.max_rounds * P.P : nullptr;
+    // outputs and state start empty
+    for (int i = lane; i < P.N; i += 32) { P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1; }
+    int status = 0;
+    for (int i = lane; i < n_act; i += 32) {
+      const int j = P.a_pool[row + i];
+      int g, gang; u32 eff;
+      if (j >= P.P || !decode_levels(P.pool[j], P.a_unit[row + i], P.a_mask[row + i], g, gang, eff)) status |= TG_ST_BAD_ACTION;
+      if (i > 0 && P.a_arrival && P.a_arrival[row + i - 1] > P.a_arrival[row + i]) status |= TG_ST_UNSORTED;
+    }
+    for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(TG_FULL, status, o);
+    if (status & TG_ST_BAD_ACTION) status = TG_ST_BAD_ACTION;
+    for (int j = 0; j < P.P; ++j) {
+      const PoolDev& pd = P.pool[j];
+      if (pd.type == TG_POOL_API) { if (lane < 2) R.pst[((size_t)sc * P.P + j) * 2 + lane] = 0; if (lane == 0) R.win[(size_t)sc * P.P + j] = 0; continue; }
+      for (int c = lane; c < pd.capacity; c += 32) {
+        int v = -1;
+        if (pd.type == TG_POOL_GPU && P.gpu_busy && (P.gpu_busy[(size_t)sc * P.n_nodes_total + pd.node0 + c / pd.group] >> (c % pd.group) & 1)) v = -2;
+        owner[R.unit0[j] + c] = v;
+      }
+      if (pd.type == TG_POOL_GPU)
+        for (int v = lane; v < pd.n_nodes; v += 32)
+          nm[pd.node0 + v] = (P.gpu_busy ? P.gpu_busy[(size_t)sc * P.n_nodes_total + pd.node0 + v] : 0) & ((1u << pd.group) - 1u);
+      if (pd.type == TG_POOL_CPU)
+        for (int d = lane; d < pd.capacity / pd.group; d += 32) dfree[R.dom0[j] + d] = pd.group;
+    }
+    if (lane == 0) { P.o_total[sc] = 0; P.o_nsel[sc] = 0; P.o_status[sc] = status; }
+    if (occ) for (int i = lane; i < R.max_rounds * P.P; i += 32) occ[i] = 0;
+    __syncwarp();
+    int rounds = 0;
+    if (status == 0) {
+      extern __shared__ __align__(16) unsigned char k2_smem[];
+      int* dem = (int*)(k2_smem + K2_DYN_SMEM_TREES) + (threadIdx.x >> 5) * 64;   // 4 ints per pool: demand, capacity
+      int* cap = dem + 32;
+      int next = 0, nw = 0, nr = 0, r = 0;
+      bool drained = false;
+      while (r < R.max_rounds) {
+        const i64 now = (i64)r * R.round_us;
+        // 1. quota refill
+        for (int j = 0; j < P.P; ++j) {
+          const PoolDev& pd = P.pool[j];
+          if (pd.type == TG_POOL_API && pd.window_us > 0 && now / pd.window_us != R.win[(size_t)sc * P.P + j]) {
+            __syncwarp();
+            if (lane == 0) { R.win[(size_t)sc * P.P + j] = now / pd.window_us; R.pst[((size_t)sc * P.P + j) * 2] = 0; }
+            __syncwarp();
+          }
+        }
+        // 2. release what has finished; the running list is compacted in place
+        int kept = 0;
+        bool gpu_released = false;
+        for (int i0 = 0; i0 < nr; i0 += 32) {
+          const int i = i0 + lane;
+          int a = -1; bool done = false;
+          if (i < nr) { a = run[i]; done = (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a] <= now; }
+          const u32 bd = __ballot_sync(TG_FULL, done), bk = __ballot_sync(TG_FULL, i < nr && !done);
+          __syncwarp();
+          if (i < nr && !done) run[kept + __popc(bk & ((1u << lane) - 1u))] = a;
+          kept += __popc(bk);
+          u32 rest = bd;
+          while (rest) {
+            const int b = __ffs(rest) - 1; rest &= rest - 1;
+            const int fa = __shfl_sync(TG_FULL, a, b);
+            const int j = P.a_pool[row + fa];
+            const PoolDev& pd = P.pool[j];
+            if (pd.type == TG_POOL_API) { if (pd.window_us == 0 && lane == 0) R.pst[((size_t)sc * P.P + j) * 2 + 1] -= P.o_alloc[row + fa]; }
+            else {
+              for (int c = lane; c < pd.capacity; c += 32) {
+                if (owner[R.unit0[j] + c] != fa) continue;
+                owner[R.unit0[j] + c] = -1;
+                if (pd.type == TG_POOL_CPU) atomicAdd(&dfree[R.dom0[j] + c / pd.group], 1);
+                else gpu_released = true;
+              }
+            }
+            __syncwarp();
+          }
+        }
+        nr = kept;
+        if (__any_sync(TG_FULL, gpu_released)) {            // node masks follow the owner map
+          for (int j = 0; j < P.P; ++j) {
+            const PoolDev& pd = P.pool[j];
+            if (pd.type != TG_POOL_GPU) continue;
+            for (int v = lane; v < pd.n_nodes; v += 32) {
+              u32 mk = 0;
+              for (int b = 0; b < pd.group; ++b) mk |= (owner[R.unit0[j] + v * pd.group + b] != -1 ? 1u : 0u) << b;
+              nm[pd.node0 + v] = (u8)mk;
+            }
+          }
+          __syncwarp();
+        }
+        // 3. admit arrivals
+        while (next < n_act) {
+          const int i = next + lane;
+          const bool in = i < n_act && (P.a_arrival ? P.a_arrival[row + i] : 0) <= now;
+          const u32 b = __ballot_sync(TG_FULL, in);
+          const int cnt = (b == TG_FULL) ? 32 : __ffs(~b) - 1;        // arrivals are sorted: a prefix of the lanes
+          if (lane < cnt) wait[nw + lane] = i;
+          nw += cnt; next += cnt;
+          if (cnt < 32) break;
+        }
+        __syncwarp();
+        // 4. schedule
+        if (nw > 0) {
+          const int n = replay_prefix(P, R, sc, wait, nw, dem, cap, lane);
+          const int nr0 = nr;
+          bool ok = true;
+          if (n > 0)
+            for (int j = 0; j < P.P && ok; ++j) ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane);
+          if (!ok) { if (lane == 0) P.o_status[sc] |= TG_ST_WORKSPACE; break; }
+          if (nr > nr0) {                                   // drop the started actions from the queue
+            int kw = 0;
+            for (int i0 = 0; i0 < nw; i0 += 32) {
+              const int i = i0 + lane;
+              int a = -1; bool stay = false;
+              if (i < nw) { a = wait[i]; stay = P.o_act[row + a] < 0; }
+              const u32 b = __ballot_sync(TG_FULL, stay);
+              __syncwarp();
+              if (stay) wait[kw + __popc(b & ((1u << lane) - 1u))] = a;
+              kw += __popc(b);
+            }
+            nw = kw;
+            __syncwarp();
+          }
+        }
+        // 5. occupancy of this round
+        int busy[TG_MAX_POOLS];
+        for (int j = 0; j < P.P; ++j) busy[j] = pool_busy_units(P, R, sc, j, lane);
+        if (occ && lane == 0) for (int j = 0; j < P.P; ++j) occ[(size_t)r * P.P + j] = busy[j];
+        ++r;
+        if (next == n_act && nw == 0 && nr == 0) { drained = true; break; }
+        // with an empty queue nothing happens before the next arrival or completion: jump there
+        if (nw == 0) {
+          i64 t_next = next < n_act ? (P.a_arrival ? P.a_arrival[row + next] : 0) : TG_INF;
+          for (int i = lane; i < nr; i += 32) {
+            const int a = run[i];
+            t_next = min(t_next, (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a]);
+          }
+          t_next = warp_min64(t_next);
+          i64 r_next = (t_next + R.round_us - 1) / R.round_us;
+          if (r_next > R.max_rounds) r_next = R.max_rounds;
+          // skipped rounds repeat this occupancy, except that quota usage restarts with its window
+          for (i64 rr = r + lane; rr < r_next; rr += 32)
+            for (int j = 0; j < P.P; ++j) {
+              const PoolDev& pd = P.pool[j];
+              int v = busy[j];
+              if (pd.type == TG_POOL_API && pd.window_us > 0 && (rr * R.round_us) / pd.window_us != R.win[(size_t)sc * P.P + j]) v = 0;
+              if (occ) occ[(size_t)rr * P.P + j] = v;
+            }
+          if (r_next > r) r = (int)r_next;
+        }
+      }
+      rounds = drained ? r : R.max_rounds;
+      if (!drained && r < R.max_rounds) rounds = r;
+    }
+    if (R.rounds_used && lane == 0) R.rounds_used[sc] = rounds;
+    __syncwarp();
+  }
+}

@@ -100,6 +100,8 @@ __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, co
 #define WARP_FAST_BYTES 0
 #define WARP_SMEM_BYTES (WARP_TREE_BYTES + WARP_FAST_BYTES)
 #define K2_DYN_SMEM ((K2_THREADS / 32) * WARP_SMEM_BYTES + 16)
+#define K2_DYN_SMEM_TREES K2_DYN_SMEM                       // the replay kernel keeps 256 more bytes per warp behind the trees
+#define K2_DYN_SMEM_REPLAY (K2_DYN_SMEM + (K2_THREADS / 32) * 256)
 __device__ __forceinline__ void attach_warp_tree(PoolTask& T) {
   extern __shared__ __align__(16) unsigned char k2_smem[];
   const u32 start = ((u32)__cvta_generic_to_shared(k2_smem) + 15u) & ~15u;
@@ -298,6 +300,8 @@ __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ P
   }
 }
 
+#include "replay.cuh"
+
 // ---------------------------------------------------------------------------------------
 // host
 // ---------------------------------------------------------------------------------------
@@ -318,6 +322,7 @@ struct tangram_round {
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
   BatchWs W; int sim_blocks; SimLists L; int n_sm;
+  ReplayWs R;
   // the capacity classes of k_sims are independent: they run on side streams between a fork
   // and a join event so that their partial waves overlap
   cudaStream_t sim_stream[TG_N_SIM_CLASSES + 1];
@@ -464,6 +469,24 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc((void**)&r->L.count, 2 * 64 * sizeof(int)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->L.list, (size_t)TG_N_SIM_CLASSES * r->L.n_groups * sizeof(int)) != cudaSuccess;
   r->L.cursor = r->L.count ? r->L.count + 64 : nullptr;
+  if (desc->max_rounds > 0) {                              // state of the trace replay
+    ReplayWs& R = r->R;
+    int u = 0, d = 0;
+    for (int j = 0; j < P.P; ++j) {
+      R.unit0[j] = u; R.dom0[j] = d;
+      if (P.pool[j].type != TG_POOL_API) u += P.pool[j].capacity;
+      if (P.pool[j].type == TG_POOL_CPU) d += P.pool[j].capacity / P.pool[j].group;
+    }
+    R.U = u ? u : 1; R.Dtot = d ? d : 1;
+    R.round_us = desc->round_us > 0 ? desc->round_us : 1; R.max_rounds = desc->max_rounds;
+    bad |= cudaMalloc((void**)&R.wait, SN * sizeof(int)) != cudaSuccess;
+    bad |= cudaMalloc((void**)&R.run, SN * sizeof(int)) != cudaSuccess;
+    bad |= cudaMalloc((void**)&R.owner, (size_t)P.S * R.U * sizeof(int)) != cudaSuccess;
+    bad |= cudaMalloc((void**)&R.nm, (size_t)P.S * (node0 ? node0 : 1)) != cudaSuccess;
+    bad |= cudaMalloc((void**)&R.dfree, (size_t)P.S * R.Dtot * sizeof(int)) != cudaSuccess;
+    bad |= cudaMalloc((void**)&R.pst, (size_t)P.S * P.P * 2 * sizeof(int)) != cudaSuccess;
+    bad |= cudaMalloc((void**)&R.win, (size_t)P.S * P.P * sizeof(i64)) != cudaSuccess;
+  }
   bad |= cudaEventCreateWithFlags(&r->sim_fork, cudaEventDisableTiming) != cudaSuccess;
   for (int c = 0; c <= TG_N_SIM_CLASSES; ++c) {
     bad |= cudaStreamCreateWithFlags(&r->sim_stream[c], cudaStreamNonBlocking) != cudaSuccess;
@@ -486,6 +509,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   e = cudaFuncSetAttribute(k_prefix, cudaFuncAttributeMaxDynamicSharedMemorySize, P.V * K1_THREADS * 4);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM_REPLAY);
   for (int c = 0; c < TG_N_SIM_CLASSES && e == cudaSuccess; ++c)
     e = cudaFuncSetAttribute(sim_kernel(g_sim_caps[c]), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TG_SMEM_PER_BLOCK - 1024);
@@ -551,6 +575,8 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
+  cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
+  cudaFree(r->R.pst); cudaFree(r->R.win);
   if (r->sim_fork) cudaEventDestroy(r->sim_fork);
   for (int c = 0; c <= TG_N_SIM_CLASSES; ++c) {
     if (r->sim_stream[c]) cudaStreamDestroy(r->sim_stream[c]);
@@ -651,10 +677,39 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
 
 extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, tangram_result* res,
                                     void* cuda_stream) {
-  (void)r; (void)a; (void)res; (void)cuda_stream;
-  return TANGRAM_EINVAL;
+  if (!r || !check_io(a, res) || r->desc.max_rounds <= 0 || !a->arrival_us) return TANGRAM_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Params P = r->P;
+  P.now = 0;
+  ReplayWs R = r->R;
+  if (r->desc.host_buffers) {
+    int rc = stage_inputs(r, a, P, st);
+    if (rc) return rc;
+    R.occupancy = res->occupancy ? (int*)(r->d_stage + r->out_off[7]) : nullptr;
+    R.rounds_used = res->rounds_used ? (int*)(r->d_stage + r->out_off[8]) : nullptr;
+  } else {
+    bind_device_io(P, a, res);
+    R.occupancy = res->occupancy; R.rounds_used = res->rounds_used;
+  }
+  CK(cudaMemsetAsync(P.arena_top, 0, 256, st));
+  int warps = P.n_workers < P.S ? P.n_workers : (int)align_up((size_t)P.S, K2_THREADS / 32);
+  cudaEvent_t* ev = prof_begin(r, 2, -1, -1, -1);
+  if (ev) CK(cudaEventRecord(ev[0], st));
+  k_replay<<<warps / (K2_THREADS / 32), K2_THREADS, K2_DYN_SMEM_REPLAY, st>>>(P, R);
+  if (ev) CK(cudaEventRecord(ev[1], st));
+  r->launches += 1;
+  CK(cudaGetLastError());
+  if (r->desc.host_buffers) {
+    int rc = unstage_outputs(r, res, P, st);
+    if (rc) return rc;
+    if (res->occupancy)
+      CK(cudaMemcpyAsync(res->occupancy, r->d_stage + r->out_off[7],
+                         (size_t)P.S * r->desc.max_rounds * P.P * sizeof(int), cudaMemcpyDeviceToHost, st));
+    if (res->rounds_used)
+      CK(cudaMemcpyAsync(res->rounds_used, r->d_stage + r->out_off[8], (size_t)P.S * sizeof(int), cudaMemcpyDeviceToHost, st));
+  }
+  return TANGRAM_OK;
 }
-
 
 // ---------------------------------------------------------------------------------------
 // tangram_schedule_batch_static: the same round for callers that must not allocate.
