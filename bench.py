@@ -89,6 +89,14 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def _oracle_call(w, arrays, lo, hi):
+    import oracle
+    if w.replay:
+        return oracle.replay_trace(w.pools, arrays, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds,
+                                   lo=lo, hi=hi, want_occupancy=False)
+    return oracle.schedule_batch(w.pools, arrays, depth=w.depth, lo=lo, hi=hi)
+
+
 def _oracle_throughput(w, arrays, target_s: float, threads: int):
     """Times the oracle, as it stands, on a bounded sample of scenarios; returns (actions/s, sample text)."""
     import oracle
@@ -98,14 +106,14 @@ def _oracle_throughput(w, arrays, target_s: float, threads: int):
     probe = min(S, 2 * threads)
     t0 = time.perf_counter()
     with ThreadPoolExecutor(threads) as ex:
-        list(ex.map(lambda sc: oracle.schedule_batch(w.pools, arrays, depth=w.depth, lo=sc, hi=sc + 1), range(probe)))
+        list(ex.map(lambda sc: _oracle_call(w, arrays, sc, sc + 1), range(probe)))
     dt = time.perf_counter() - t0
     n = int(min(S, max(probe, target_s / max(dt / probe, 1e-9))))
     chunk = max(1, n // (threads * 8))
     starts = list(range(0, n, chunk))
     t0 = time.perf_counter()
     with ThreadPoolExecutor(threads) as ex:
-        list(ex.map(lambda lo: oracle.schedule_batch(w.pools, arrays, depth=w.depth, lo=lo, hi=min(n, lo + chunk)), starts))
+        list(ex.map(lambda lo: _oracle_call(w, arrays, lo, min(n, lo + chunk)), starts))
     dt = time.perf_counter() - t0
     acts = int(arrays["n_actions"][:n].sum())
     return acts / dt, f"first {n} of {S} scenarios of {w.name} ({acts} pending actions), {threads} threads, {dt:.1f} s"
@@ -141,7 +149,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", default="cfg4", choices=[k for k, v in CONFIGS.items() if not v.replay])
+    ap.add_argument("--config", default="cfg4", choices=list(CONFIGS))
     ap.add_argument("--scenarios", type=int, default=0, help="override the number of scenarios (smaller runs)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -184,9 +192,12 @@ def main():
         cpu = {"value": v, "unit": "actions/s", "cores": threads, "kind": "oracle", "sample": sample}
 
     dev = binding.to_device(arrays)
-    rnd = binding.Round(S, N, w.pools, depth=w.depth)
-    res = rnd.new_result()
+    rnd = binding.Round(S, N, w.pools, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds)
+    res = rnd.new_result(replay=w.replay)
     stream = torch.cuda.current_stream()
+    if w.replay:                                   # a step of a replay workload = the whole trace
+        _sb = rnd.schedule_batch
+        rnd.schedule_batch = lambda a_, now_, res_, st_: rnd.replay_trace(a_, res_, st_)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -219,9 +230,12 @@ def main():
     # end to end through host buffers (pinned), copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        hrnd = binding.Round(S, N, w.pools, depth=w.depth, host_buffers=True)
+        hrnd = binding.Round(S, N, w.pools, depth=w.depth, host_buffers=True, round_us=w.round_us,
+                             max_rounds=w.max_rounds)
         hin = binding.to_device(arrays, pin=True)
-        hres = hrnd.new_result()
+        hres = hrnd.new_result(replay=w.replay)
+        if w.replay:
+            hrnd.schedule_batch = lambda a_, now_, res_, st_: hrnd.replay_trace(a_, res_, st_)
         for _ in range(2):
             hrnd.schedule_batch(hin, 0, hres, stream)
         sync_all()

@@ -82,7 +82,8 @@ typedef struct {
   int32_t host_buffers; /* 0: tangram_actions / tangram_result hold DEVICE pointers;
                            1: they hold HOST pointers and every call copies inputs in and
                            results out on the given stream (pinned memory recommended)     */
-  int64_t workspace_bytes; /* scratch for large DP tables; 0 = default (1 GiB)             */
+  int64_t workspace_bytes; /* scratch for large DP tables; 0 = default (8 GiB): 7/8 of it
+                              are 48 reusable slots (a DP table must fit one), the rest is bump-allocated             */
   const tangram_pool_desc* pools; /* host array of n_pools entries, copied                 */
 } tangram_round_desc;
 

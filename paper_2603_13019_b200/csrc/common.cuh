@@ -141,3 +141,14 @@ __device__ __forceinline__ void gpu_caps(const PoolDev& pd, const u8* busy, int 
   F0 = warp_sum32(F0); F1 = warp_sum32(F1); F2 = warp_sum32(F2); F3 = warp_sum32(F3);
   cap[3] = F3 * 8; cap[2] = cap[3] + F2 * 4; cap[1] = cap[2] + F1 * 2; cap[0] = cap[1] + F0;
 }
+
+// The arena of large scratch: its lower 7/8 are equal slots that a warp borrows for one large DP
+// table and gives back (48 slots of at least 64 MiB when the arena allows, else down to 4
+// larger-as-possible ones); the rest is handed out by a bump pointer, never reused in a call.
+#define TG_ARENA_MAX_SLOTS 48
+__device__ __forceinline__ int arena_n_slots(const Params& P) {
+  u64 n = (P.arena_bytes / 8 * 7) >> 26;
+  return n < 4 ? 4 : (n > TG_ARENA_MAX_SLOTS ? TG_ARENA_MAX_SLOTS : (int)n);
+}
+__device__ __forceinline__ u64 arena_slot_bytes(const Params& P) { return ((P.arena_bytes / 8 * 7) / arena_n_slots(P)) & ~(u64)255; }
+__device__ __forceinline__ u64 arena_bump_base(const Params& P) { return arena_slot_bytes(P) * arena_n_slots(P); }

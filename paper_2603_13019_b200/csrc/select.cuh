@@ -30,14 +30,42 @@ struct Slab {
   }
 };
 
-// warp-uniform bump allocation from the shared arena (large DP tables only)
+// warp-uniform bump allocation from the bump part of the arena
 __device__ __forceinline__ void* arena_take(const Params& P, u64 bytes, int lane) {
   bytes = (bytes + 255) & ~(u64)255;
+  const u64 half = arena_bump_base(P);
   u64 off = 0;
   if (lane == 0) off = atomicAdd(P.arena_top, bytes);
   off = __shfl_sync(TG_FULL, off, 0);
-  if (off + bytes > P.arena_bytes) return nullptr;
-  return P.arena + off;
+  if (half + off + bytes > P.arena_bytes) return nullptr;
+  return P.arena + half + off;
+}
+// Borrow a slot (warp-uniform).  Waits, with a limit, for another warp to give one back; the
+// holders never wait for anything, so the wait ends.  Returns -1 if the table does not fit a
+// slot or the limit ran out.
+__device__ __forceinline__ int slot_acquire(const Params& P, u64 bytes, int lane) {
+  const u64 slot_bytes = arena_slot_bytes(P);
+  int got = -1;
+  if (lane == 0 && bytes <= slot_bytes) {
+    int* flags = (int*)(P.arena_top + 8);
+    const int ns = arena_n_slots(P);
+    const int start = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5) % ns;
+    for (int tries = 0; tries < 2000000 && got < 0; ++tries) {   // gives up after some seconds
+      for (int k = 0; k < ns && got < 0; ++k) {
+        const int s = (start + k) % ns;
+        if (atomicCAS(&flags[s], 0, 1) == 0) got = s;
+      }
+      if (got < 0) __nanosleep(2000);
+    }
+  }
+  return __shfl_sync(TG_FULL, got, 0);
+}
+__device__ __forceinline__ char* slot_ptr(const Params& P, int s) {
+  return P.arena + (u64)s * arena_slot_bytes(P);
+}
+__device__ __forceinline__ void slot_release(const Params& P, int s, int lane) {
+  __syncwarp();
+  if (lane == 0 && s >= 0) { __threadfence(); atomicExch((int*)(P.arena_top + 8) + s, 0); }
 }
 
 struct PoolTask {
@@ -165,9 +193,11 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
   const int ncell = (int)cells;
   i64* val = (i64*)slab.take(2 * cells * sizeof(i64));
   u8* choice = val ? (u8*)slab.take((u64)nrows * cells) : nullptr;
+  int slot = -1;
   if (!choice) {
-    char* big = (char*)arena_take(P, 2 * cells * sizeof(i64) + (u64)nrows * cells, lane);
-    if (!big) return false;
+    slot = slot_acquire(P, 2 * cells * sizeof(i64) + (u64)nrows * cells, lane);
+    if (slot < 0) return false;
+    char* big = slot_ptr(P, slot);
     val = (i64*)big; choice = (u8*)(big + 2 * cells * sizeof(i64));
   }
   i64* prev = val; i64* cur = val + cells;
@@ -209,7 +239,7 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
   i64 bv = TG_INF;
   for (int c = lane; c < ncell; c += 32) bv = min(bv, prev[c]);
   bv = warp_min64(bv);
-  if (bv == TG_INF) return false;                    // cannot happen for an accommodated prefix
+  if (bv == TG_INF) { slot_release(P, slot, lane); return false; }   // cannot happen for an accommodated prefix
   int be = INT_MAX;
   for (int c = lane; c < ncell; c += 32) if (prev[c] == bv) be = min(be, c % ext[0]);
   be = warp_min32(be);
@@ -260,6 +290,7 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
     }
   }
   fail = __shfl_sync(TG_FULL, fail, 0);
+  slot_release(P, slot, lane);
   if (fail) return false;
   __syncwarp();
   i64 sum = 0;

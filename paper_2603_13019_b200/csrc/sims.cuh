@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(32) k_sims_big(const __grid_constant__ Params 
   u64 off = 0;
   const u64 bytes = ((u64)hmax * 32 * (sizeof(i64) + 2 * sizeof(u32)) + 255) & ~(u64)255;
   if (t == 0) off = atomicAdd(P.arena_top, bytes);
-  off = __shfl_sync(TG_FULL, off, 0);
+  off = __shfl_sync(TG_FULL, off, 0) + arena_bump_base(P);                   // bump part of the arena
   if (off + bytes > P.arena_bytes) { if (J.active) atomicOr(&J.st->flags, TS_FAILED); return; }
   if (!J.active) return;
   i64* val = (i64*)(P.arena + off);

@@ -448,7 +448,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   size_t per_cand = 8 + 8 + 4 + 4 + 4 + 4 + 4 + 3 + 16 * (size_t)desc->depth;
   size_t slab = align_up((size_t)P.N * per_cand + 64 * 1024 + (1 << 20) / 4 + 4096, 256);
   P.slab_bytes = slab;
-  P.arena_bytes = desc->workspace_bytes ? (u64)desc->workspace_bytes : (1ull << 30);
+  P.arena_bytes = desc->workspace_bytes ? (u64)desc->workspace_bytes : (8ull << 30);
   bool bad = false;
   bad |= cudaMalloc(&r->d_order, SN * sizeof(int)) != cudaSuccess;
   bad |= cudaMalloc(&r->d_tmin, SN * sizeof(i64)) != cudaSuccess;

@@ -1,0 +1,51 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the whole
+batch runs on the GPU, a sample of scenarios is recomputed by the oracle one by one, and
+size-independent invariants are checked on everything."""
+import numpy as np
+import pytest
+
+from workloads import POOL_GPU, generate, make_workload
+
+pytestmark = pytest.mark.gpu
+
+KEYS = ("status", "n_selected", "total_act_us", "alloc_units", "place_node", "place_off", "act_us")
+
+
+def _run_full(name):
+    import torch
+    from paper_2603_13019_b200 import binding
+    w = make_workload(name)
+    S, N = w.n_scenarios, w.max_actions
+    chunk = max(1, (64 << 20) // N)
+    parts = [generate(w, c, min(S, c + chunk)) for c in range(0, S, chunk)]
+    a = {k: (None if parts[0][k] is None else np.concatenate([p[k] for p in parts])) for k in parts[0]}
+    rnd = binding.Round(S, N, w.pools, depth=w.depth)
+    out = rnd.schedule_batch(binding.to_device(a))
+    torch.cuda.synchronize()
+    g = {k: v.cpu().numpy() for k, v in out.items()}
+    rnd.destroy()
+    return w, a, g
+
+
+@pytest.mark.parametrize("name,n_sample", [("cfg4", 96), ("cfg1", 128), ("cfg3", 24)])
+def test_full_size_sampled_scenarios_match_oracle(oracle, name, n_sample):
+    w, a, g = _run_full(name)
+    S = w.n_scenarios
+    assert np.all(g["status"] == 0)
+    rng = np.random.default_rng(11)
+    sample = np.unique(np.concatenate([[0, S - 1], rng.integers(0, S, n_sample)]))
+    for sc in sample:
+        o = oracle.schedule_batch(w.pools, a, depth=w.depth, lo=int(sc), hi=int(sc) + 1)
+        for k in KEYS:
+            assert np.array_equal(o[k][0], g[k][sc]), f"{name}: scenario {sc}: {k} differs"
+    # invariants on every scenario: capacity per pool, totals, sentinels
+    sel = g["alloc_units"] > 0
+    assert np.array_equal(sel.sum(1), g["n_selected"])
+    assert np.array_equal(np.where(sel, g["act_us"], 0).sum(1), g["total_act_us"])
+    assert np.all(g["act_us"][~sel] == -1) and np.all(g["place_node"][~sel] == -1)
+    for j, p in enumerate(w.pools):
+        used = np.where(a["pool"] == j, g["alloc_units"], 0).sum(1)
+        busy = 0
+        if p.type == POOL_GPU and a["gpu_busy"] is not None:
+            busy = np.unpackbits(a["gpu_busy"], axis=1).sum(1)
+        assert np.all(used + busy <= p.capacity)
