@@ -163,3 +163,136 @@ __device__ void place_cpu_owner(const PoolDev& pd, int* owner, int* dfree, int k
     __syncwarp();
   }
 }
+
+// ---- register-resident fast paths of a single round (fresh CPU pool, at most 128 domains /
+// ---- GPU nodes): the state lives in lane registers, the arg-min is one redux, and every lane
+// ---- keeps the result of "its" candidate of a block of 32 for a coalesced write.
+
+// maximal free aligned blocks of a node: bit = first GPU of such a block (busy: 8 bits, padded)
+struct NodeBlocks { u32 s1, s2, s4, s8; };
+__device__ __forceinline__ NodeBlocks node_blocks(u32 busy) {
+  const u32 fr = ~busy & 0xffu;
+  const u32 pr = fr & (fr >> 1) & 0x55u;          // bit 2k: GPUs 2k, 2k+1 free
+  const u32 nb = pr & (pr >> 2) & 0x11u;          // bit 4k: GPUs 4k .. 4k+3 free
+  const u32 oc = nb & (nb >> 4) & 1u;             // the whole node free
+  NodeBlocks b;
+  b.s1 = fr & ~(pr | (pr << 1));
+  b.s2 = pr & ~(nb | (nb << 2));
+  b.s4 = nb & ~(oc | (oc << 4));
+  b.s8 = oc;
+  return b;
+}
+__device__ __forceinline__ u32 node_levels(u32 busy) {   // bit l: a maximal free block of 2^l GPUs exists
+  const NodeBlocks b = node_blocks(busy);
+  return (b.s1 ? 1u : 0u) | (b.s2 ? 2u : 0u) | (b.s4 ? 4u : 0u) | (b.s8 ? 8u : 0u);
+}
+__device__ __forceinline__ int node_block_start(u32 busy, int bl) {
+  const NodeBlocks b = node_blocks(busy);
+  const u32 m = bl == 0 ? b.s1 : (bl == 1 ? b.s2 : (bl == 2 ? b.s4 : b.s8));
+  return __ffs(m) - 1;
+}
+
+// Same placement rule as place_gpu; requires pd.n_nodes <= 128.  busy_row: the pool's node
+// masks before the round (may be null).
+__device__ void place_gpu_reg(const PoolDev& pd, const u8* busy_row, int keep, const u8* cg, const u8* r,
+                              int* pnode, int* poff, int lane) {
+  const int top = ilog2(pd.group);
+  const u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;
+  u32 nm[4], lev[4];
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const int v = lane + 32 * s;
+    nm[s] = v < pd.n_nodes ? ((busy_row ? busy_row[v] : 0u) | pad) : 0xffu;
+    lev[s] = node_levels(nm[s]);
+  }
+  for (int lz = top; lz >= 0; --lz) {
+    const int z = 1 << lz;
+    for (int i0 = 0; i0 < keep; i0 += 32) {
+      const int i = i0 + lane;
+      int nreq = 0;
+      if (i < keep) {
+        const int g = cg[i] & 0x7f, gang = cg[i] >> 7, ri = r[i];
+        nreq = gang ? (g * ri == z ? 1 : 0) : (g == z ? ri : 0);
+      }
+      int myn = -1, myo = -1;
+      u32 bm = __ballot_sync(TG_FULL, nreq > 0);
+      while (bm) {
+        const int b = __ffs(bm) - 1; bm &= bm - 1;
+        const int cnt = __shfl_sync(TG_FULL, nreq, b);
+        for (int rep = 0; rep < cnt; ++rep) {
+          u32 node = 0xffffffffu; int bl = lz;
+          for (; bl <= top; ++bl) {                     // smallest sufficient block level, lowest node
+            u32 key = 0xffffffffu;
+#pragma unroll
+            for (int s = 3; s >= 0; --s) if ((lev[s] >> bl) & 1u) key = (u32)(lane + 32 * s);
+            node = __reduce_min_sync(TG_FULL, key);
+            if (node != 0xffffffffu) break;
+          }
+          if (node == 0xffffffffu) continue;            // cannot happen: the selection fits
+          int start = 0;
+          if (lane == (int)(node & 31u)) {
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+              if (s == (int)(node >> 5)) {
+                start = node_block_start(nm[s], bl);
+                nm[s] |= ((1u << z) - 1u) << start;
+                lev[s] = node_levels(nm[s]);
+              }
+          }
+          start = __shfl_sync(TG_FULL, start, node & 31u);
+          if (rep == 0 && lane == b) { myn = (int)node; myo = start; }
+        }
+      }
+      if (i < keep && myn >= 0) { pnode[i] = myn; poff[i] = myo; }
+    }
+  }
+}
+
+// Same placement rule as place_cpu_fresh; requires at most 128 domains of fewer than 65536 cores.
+__device__ void place_cpu_fresh_reg(const PoolDev& pd, int keep, const u8* cg, const u8* r,
+                                    int* pnode, int* poff, int lane) {
+  const int D = pd.capacity / pd.group;
+  u32 df[4];
+#pragma unroll
+  for (int s = 0; s < 4; ++s) df[s] = lane + 32 * s < D ? (u32)pd.group : 0u;
+  for (int i0 = 0; i0 < keep; i0 += 32) {
+    const int i = i0 + lane;
+    const int mine = i < keep ? (cg[i] & 0x7f) * r[i] : 0;
+    int myn = -1, myo = -1;
+    const int nb = min(32, keep - i0);
+    for (int b = 0; b < nb; ++b) {
+      const u32 k = (u32)__shfl_sync(TG_FULL, mine, b);
+      u32 key = 0xffffffffu;
+#pragma unroll
+      for (int s = 0; s < 4; ++s) if (df[s] >= k) key = min(key, (df[s] << 16) | (u32)(lane + 32 * s));
+      const u32 best = __reduce_min_sync(TG_FULL, key);
+      int first = -1;
+      if (best != 0xffffffffu) {                       // best fit: fewest free cores that still fit
+        const int d = (int)(best & 0xffffu), f = (int)(best >> 16);
+        first = d * pd.group + (pd.group - f);
+        if (lane == (d & 31)) {
+#pragma unroll
+          for (int s = 0; s < 4; ++s) if (s == (d >> 5)) df[s] -= k;
+        }
+      } else {                                         // no domain fits: fill domains in ascending order
+        u32 need = k;
+        for (int d = 0; d < D && need > 0; ++d) {
+          u32 f = 0;
+#pragma unroll
+          for (int s = 0; s < 4; ++s) if (s == (d >> 5)) f = df[s];
+          f = __shfl_sync(TG_FULL, f, d & 31);
+          if (f == 0) continue;
+          if (first < 0) first = d * pd.group + (pd.group - (int)f);
+          const u32 take = min(f, need);
+          if (lane == (d & 31)) {
+#pragma unroll
+            for (int s = 0; s < 4; ++s) if (s == (d >> 5)) df[s] -= take;
+          }
+          need -= take;
+        }
+      }
+      if (lane == b) { myn = first >= 0 ? first / pd.group : -1; myo = first; }
+    }
+    if (i < keep) { pnode[i] = myn; poff[i] = myo; }
+  }
+}

@@ -24,9 +24,14 @@ struct Slab {
   char* fbase; u32 fcap; u32 fused;       // shared-memory window (generic address), may be empty
   __device__ __forceinline__ void* take(u64 bytes) {
     bytes = (bytes + 15) & ~(u64)15;
-    if (fused + bytes <= fcap) { void* p = fbase + fused; fused += (u32)bytes; return p; }
     if (used + bytes > cap) return nullptr;
     void* p = base + used; used += bytes; return p;
+  }
+  // small arrays that sequential loops read again and again: the window if there is room
+  __device__ __forceinline__ void* take_fast(u64 bytes) {
+    bytes = (bytes + 15) & ~(u64)15;
+    if (fused + bytes <= fcap) { void* p = fbase + fused; fused += (u32)bytes; return p; }
+    return take(bytes);
   }
 };
 

@@ -54,9 +54,9 @@ __device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta
   C.pnode = (int*)slab.take((u64)m * 4);
   C.poff = (int*)slab.take((u64)m * 4);
   C.rowcand = (int*)slab.take((u64)m * 4);
-  C.cg = (u8*)slab.take(m);
+  C.cg = (u8*)slab.take_fast(m);
   C.rsel = (u8*)slab.take(m);
-  C.rkeep = (u8*)slab.take(m);
+  C.rkeep = (u8*)slab.take_fast(m);
   if (!C.rkeep) return false;
   for (int i = lane; i < m; i += 32) {
     int idx = P.order[row + mt.base + i];
@@ -97,7 +97,7 @@ __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, co
 // shared memory of the calling warp for winner trees inside the per-pool kernels
 #define WARP_TREE_SLOTS 448
 #define WARP_TREE_BYTES (WARP_TREE_SLOTS * 16)
-#define WARP_FAST_BYTES 0
+#define WARP_FAST_BYTES 2048
 #define WARP_SMEM_BYTES (WARP_TREE_BYTES + WARP_FAST_BYTES)
 #define K2_DYN_SMEM ((K2_THREADS / 32) * WARP_SMEM_BYTES + 16)
 #define K2_DYN_SMEM_TREES K2_DYN_SMEM                       // the replay kernel keeps 256 more bytes per warp behind the trees
@@ -127,16 +127,21 @@ __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& 
   const size_t row = (size_t)sc * P.N;
   const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr;
   if (pd.type == TG_POOL_GPU) {
-    u8* nm = (u8*)slab.take(pd.n_nodes);
+    if (pd.n_nodes <= 128) place_gpu_reg(pd, busy_row ? busy_row + pd.node0 : nullptr, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
+    else {
+    u8* nm = (u8*)slab.take_fast(pd.n_nodes);
     if (!nm) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
     else {
       for (int v = lane; v < pd.n_nodes; v += 32) nm[v] = busy_row ? busy_row[pd.node0 + v] : 0;
       __syncwarp();
       place_gpu(pd, nm, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
     }
+    }
+  } else if (pd.type == TG_POOL_CPU && pd.capacity / pd.group <= 128 && pd.group < 65536) {
+    place_cpu_fresh_reg(pd, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
   } else if (pd.type == TG_POOL_CPU) {
     const int D = pd.capacity / pd.group;
-    int* dfree = (int*)slab.take((u64)D * 4);
+    int* dfree = (int*)slab.take_fast((u64)D * 4);
     if (!dfree) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
     else place_cpu_fresh(pd, dfree, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
   } else {
@@ -147,6 +152,7 @@ __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& 
     __syncwarp();
   }
 
+  __syncwarp();
   i64 tot = 0; int cnt = 0;
   for (int i = lane; i < m; i += 32) {
     const size_t o = row + C.cidx[i];
