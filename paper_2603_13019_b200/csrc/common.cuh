@@ -36,6 +36,7 @@ struct PoolMeta {
 struct Params {
   int S, N, P, depth, n_nodes_total, V;
   PoolDev pool[TG_MAX_POOLS];
+  int pool_order[TG_MAX_POOLS];   // pools in the order their tasks are handed out (longest tasks first)
   i64 now;
   // inputs (device)
   const u8* a_pool; const u8* a_unit; const u32* a_mask;

@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ P
   for (;;) {
     const int x = next_task(P.arena_top + 3, lane);
     if (x >= n_tasks) break;
-    run_pool_task(P, x % P.S, x / P.S, slab, lane);       // pool-major: pool 0 of every scenario first
+    run_pool_task(P, x % P.S, P.pool_order[x / P.S], slab, lane);   // pool-major, heaviest pools first
   }
 }
 
@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Pa
   for (;;) {
     const int x = next_task(P.arena_top + 1, lane);
     if (x >= n_tasks) break;
-    const int sc = x % P.S, j = x / P.S, task = sc * P.P + j;
+    const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
     const PoolMeta mt = P.meta[task];
     TaskState* st = W.ts + task;
     if (mt.m == 0 || !mt.elastic) { if (lane == 0) st->flags = 0; continue; }
@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ P
   for (;;) {
     const int x = next_task(P.arena_top + 2, lane);
     if (x >= n_tasks) break;
-    const int sc = x % P.S, j = x / P.S, task = sc * P.P + j;
+    const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
     const PoolMeta mt = P.meta[task];
     if (mt.m == 0) continue;
     Slab slab = warp_slab(P, gw);
@@ -405,6 +405,15 @@ extern "C" int64_t tangram_kernel_launches(const tangram_round* r) { return r ? 
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// GPU pools first (their tasks may go on evicting), then CPU pools, then API pools
+static void fill_pool_order(Params& P) {
+  int k = 0;
+  const int rank[3] = {TG_POOL_GPU, TG_POOL_CPU, TG_POOL_API};
+  for (int r = 0; r < 3; ++r)
+    for (int j = 0; j < P.P; ++j)
+      if (P.pool[j].type == rank[r]) P.pool_order[k++] = j;
+}
+
 extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_round** out) {
   if (!desc || !out || !desc->pools) return TANGRAM_EINVAL;
   if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
@@ -439,6 +448,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   r->desc.pools = r->pools;
   P.n_nodes_total = node0;
   P.V = slot0 + desc->n_pools;
+  fill_pool_order(P);
 
   cudaError_t e = cudaGetDevice(&r->device);
   cudaDeviceProp prop;
@@ -775,6 +785,7 @@ extern "C" int tangram_schedule_batch_static(const tangram_round_desc* desc, con
   }
   P.n_nodes_total = node0;
   P.V = slot0 + desc->n_pools;
+  fill_pool_order(P);
   P.now = now_us;
 
   // carve the array: fixed parts first, then as many worker slabs as fit, the rest is the arena
