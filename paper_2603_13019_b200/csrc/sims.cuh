@@ -11,15 +11,15 @@
 // level, hence the best depth is always the largest level tried.
 //
 // The priority queue is a winner tree of packed keys: node n of the implicit tree over H slots
-// (leaf i = node H + i) holds the smallest key of its subtree, key = 2^62 | completion << 12 |
-// slot.  Replacing the minimum only touches the path from its leaf to the root, and the
-// siblings on that path are known from the leaf alone, so their loads are all issued at once
-// and only a chain of minima remains sequential.  With bit 62 set every key is the bit pattern
-// of a positive normal double, whose order is the integer order, so a key minimum is one fmin.
+// (leaf i = node H + i) holds the smallest key of its subtree, key = completion << 12 | slot.
+// Replacing the minimum only touches the path from its leaf to the root, and the siblings on
+// that path are known from the leaf alone, so their loads are all issued at once and only a
+// chain of integer minima remains sequential (an fp64 fmin on the same bits was measured
+// slower on this part).
 // One lane runs one simulation; a warp's 32 trees live in shared memory interleaved by lane
 // (node n of lane t at n * 32 + t, conflict free).  Shared memory bounds how many simulations
 // are resident, so what matters is the latency of a step, not the number of warps.
-// A completion time that would not fit the 49 value bits sends the simulation to the exact
+// A completion time that would not fit 49 value bits sends the simulation to the exact
 // 64-bit kernel below.
 //
 // Work distribution: k_sim_classify sorts groups of 32 consecutive simulations (same pool,
@@ -34,8 +34,6 @@
 #define SIM_SLOT_BYTES 16       // shared memory per slot: two tree nodes of 8 bytes
 #define SIM_SLOT_BITS 12
 #define SIM_VALUE_LIMIT (1LL << 49)
-#define SIM_KEY_BIAS (1LL << 62)
-#define SIM_KEY_INF 0x7FE0000000000000LL
 
 // per (scenario, pool) state handed from the solve kernel to the simulations and the finish kernel
 struct TaskState {
@@ -124,10 +122,7 @@ __global__ void k_sim_classify(const __grid_constant__ Params P, const TaskState
   L.list[(size_t)c * L.n_groups + pos] = g;
 }
 
-// minimum of two keys (see the header: keys order like the doubles they spell)
-__device__ __forceinline__ i64 key_min(i64 a, i64 b) {
-  return __double_as_longlong(fmin(__longlong_as_double(a), __longlong_as_double(b)));
-}
+__device__ __forceinline__ i64 key_min(i64 a, i64 b) { return b < a ? b : a; }
 
 __device__ __forceinline__ i64 lds64(u32 addr) {
   i64 v;
@@ -149,7 +144,7 @@ __device__ __forceinline__ void sts64(u32 addr, i64 v) {
 template <int MAXD, int SS, class SeedFn, class DurFn>
 __device__ __forceinline__ i64 tree_sim(u32 base, int H, int steps, SeedFn seed, DurFn dur, bool* overflow) {
   const u32 NM = ~((1u << SS) - 1u);
-  for (int i = 0; i < H; ++i) sts64(base + ((u32)(H + i) << SS), SIM_KEY_BIAS | (seed(i) << SIM_SLOT_BITS) | i);
+  for (int i = 0; i < H; ++i) sts64(base + ((u32)(H + i) << SS), (seed(i) << SIM_SLOT_BITS) | i);
   for (int n = H - 1; n >= 1; --n)
     sts64(base + ((u32)n << SS), key_min(lds64(base + ((u32)(2 * n) << SS)), lds64(base + ((u32)(2 * n + 1) << SS))));
   i64 top = lds64(base + ((u32)(H > 1 ? 1 : H) << SS));   // key of the earliest completion
@@ -167,10 +162,10 @@ __device__ __forceinline__ i64 tree_sim(u32 base, int H, int steps, SeedFn seed,
     for (int x4 = 0; x4 < 4; ++x4) {
       if (k0 + x4 < steps) {
         const u32 w = (u32)top & ((1u << SIM_SLOT_BITS) - 1u);
-        const i64 v = ((top >> SIM_SLOT_BITS) & ((1LL << 50) - 1)) + cur[x4];   // pop earliest, push ts + T
+        const i64 v = (top >> SIM_SLOT_BITS) + cur[x4];       // pop earliest, push ts + T
         chunk += v;
         ovf |= (u32)(v >> 32);
-        i64 c = SIM_KEY_BIAS | (v << SIM_SLOT_BITS) | (i64)w;
+        i64 c = (v << SIM_SLOT_BITS) | (i64)w;
         const u32 o0 = ((u32)H + w) << SS;             // byte offset of the leaf
         sts64(base + o0, c);
         i64 sk[MAXD]; u32 pa[MAXD];
