@@ -327,7 +327,7 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab sl
     if (lane == 0) {
       bool overflow;
       const i64 fd = duration(fs, fp, nth_level_of(fm, dmax - 1));
-      val = tree_sim<9, 3>(
+      val = tree_sim2<9, 3>(
           T.sim_base, H, n_rest,
           [&](int i) { return i < T.n_seeds ? T.seeds[i]
                                             : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], T.rsel[i - T.n_seeds]); },

@@ -10,8 +10,8 @@
 // estimate is non-decreasing in the first action's duration; durations do not grow with the
 // level, hence the best depth is always the largest level tried.
 //
-// The priority queue is a winner tree of packed keys: node n of the implicit tree over H slots
-// (leaf i = node H + i) holds the smallest key of its subtree, key = completion << 12 | slot.
+// The priority queue is a winner tree of packed keys: every node of an implicit tree over H slots
+// (4-ary, see tree_sim) holds the smallest key of its subtree, key = completion << 12 | slot.
 // Replacing the minimum only touches the path from its leaf to the root, and the siblings on
 // that path are known from the leaf alone, so their loads are all issued at once and only a
 // chain of integer minima remains sequential (an fp64 fmin on the same bits was measured
@@ -31,7 +31,6 @@
 #include "common.cuh"
 
 #define SIM_PER_WARP 32         // simulations per warp
-#define SIM_SLOT_BYTES 16       // shared memory per slot: two tree nodes of 8 bytes
 #define SIM_SLOT_BITS 12
 #define SIM_VALUE_LIMIT (1LL << 49)
 
@@ -133,7 +132,80 @@ __device__ __forceinline__ void sts64(u32 addr, i64 v) {
   asm volatile("st.shared.b64 [%0], %1;" :: "r"(addr), "l"(v) : "memory");
 }
 
-// One whole simulation on a winner tree in shared memory, run by the calling lane alone.
+// nodes of the 4-ary winner tree over H slots: I internal nodes (every one with four children),
+// then 3 I + 1 leaves of which the first H are the slots and the rest hold +inf
+__host__ __device__ __forceinline__ int tree_internal(int H) { return (H + 1) / 3; }
+__host__ __device__ __forceinline__ int tree_nodes(int H) { return 4 * tree_internal(H) + 1; }
+
+// One whole simulation on a 4-ary winner tree in shared memory, run by the calling lane alone.
+// Node n (root 0, children of n: 4n+1 .. 4n+4, slot s = node I + s) is at shared address
+// base + (n << SS).  MAXD bounds the number of levels below the root.  seed(i) gives slot i's
+// first completion, dur(k) the duration of the k-th remaining action, k = 0 .. steps-1.
+// Replacing the minimum walks from its leaf to the root; the node indices of that path follow
+// from the leaf alone, so the three siblings of every level are loaded at once, their minimum
+// is taken off the critical path, and one minimum per level remains sequential.
+// Returns the estimate (saturating sum of completions); *overflow tells that a completion
+// reached 2^49 and the packed keys cannot be trusted.
+template <int MAXD, int SS, class SeedFn, class DurFn>
+__device__ __forceinline__ i64 tree_sim(u32 base, int H, int steps, SeedFn seed, DurFn dur, bool* overflow) {
+  const int I = tree_internal(H), T = 4 * I + 1;
+  for (int i = 0; i < T - I; ++i) sts64(base + ((u32)(I + i) << SS), i < H ? ((seed(i) << SIM_SLOT_BITS) | i) : TG_INF);
+  for (int n = I - 1; n >= 0; --n) {
+    const u32 c0 = base + ((u32)(4 * n + 1) << SS);
+    sts64(base + ((u32)n << SS), key_min(key_min(lds64(c0), lds64(c0 + (1u << SS))),
+                                         key_min(lds64(c0 + (2u << SS)), lds64(c0 + (3u << SS)))));
+  }
+  i64 top = lds64(base);                               // key of the earliest completion
+  i64 tmp = 0;
+  u32 ovf = 0;
+  // durations are fetched a chunk of four ahead
+  i64 cur[4], nxt[4];
+#pragma unroll
+  for (int x = 0; x < 4; ++x) cur[x] = x < steps ? dur(x) : 0;
+  for (int k0 = 0; k0 < steps; k0 += 4) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) nxt[x] = (k0 + 4 + x < steps) ? dur(k0 + 4 + x) : 0;
+    i64 chunk = 0;                                     // four completions < 2^51: no overflow here
+#pragma unroll
+    for (int x4 = 0; x4 < 4; ++x4) {
+      if (k0 + x4 < steps) {
+        const u32 w = (u32)top & ((1u << SIM_SLOT_BITS) - 1u);
+        i64 c = top + (cur[x4] << SIM_SLOT_BITS);      // pop earliest completion ts, push ts + T (same slot)
+        chunk += c >> SIM_SLOT_BITS;
+        ovf |= (u32)(c >> 32);
+        int n = I + (int)w;
+        sts64(base + ((u32)n << SS), c);
+        // siblings' minimum and parent of every level of the path
+        i64 sm[MAXD]; u32 pa[MAXD]; bool on[MAXD];
+#pragma unroll
+        for (int x = 0; x < MAXD; ++x) {
+          on[x] = n > 0;
+          const int nn = on[x] ? n : 1;                // beyond the root: a harmless read of node 1's group
+          const int g = ((nn - 1) & ~3) + 1, k = (nn - 1) & 3;
+          const i64 s1 = lds64(base + ((u32)(g + ((k + 1) & 3)) << SS));
+          const i64 s2 = lds64(base + ((u32)(g + ((k + 2) & 3)) << SS));
+          const i64 s3 = lds64(base + ((u32)(g + ((k + 3) & 3)) << SS));
+          sm[x] = key_min(s1, key_min(s2, s3));
+          n = (nn - 1) >> 2;
+          pa[x] = base + ((u32)n << SS);
+        }
+#pragma unroll
+        for (int x = 0; x < MAXD; ++x) {
+          if (on[x]) { c = key_min(c, sm[x]); sts64(pa[x], c); }
+        }
+        top = c;
+      }
+    }
+    tmp = sat_add(tmp, chunk);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) cur[x] = nxt[x];
+  }
+  *overflow = (ovf >> 29) != 0;                        // a completion >= 2^49
+  return tmp;
+}
+
+// The same simulation on a binary winner tree (more shared memory, fewer instructions per
+// step): for the single simulations of continued evictions, where latency is all that counts.
 // Node n is at shared address base + (n << SS); base must be a multiple of 2 << SS plus an offset
 // below 1 << SS, so that with o = n << SS the sibling of a node is at (base + o) ^ (1 << SS) and
 // the node offsets of a leaf-to-root path are (leaf offset >> level) & ~((1 << SS) - 1).
@@ -142,7 +214,7 @@ __device__ __forceinline__ void sts64(u32 addr, i64 v) {
 // (saturating sum of completions); *overflow tells that a completion reached 2^49 and the
 // packed keys cannot be trusted.
 template <int MAXD, int SS, class SeedFn, class DurFn>
-__device__ __forceinline__ i64 tree_sim(u32 base, int H, int steps, SeedFn seed, DurFn dur, bool* overflow) {
+__device__ __forceinline__ i64 tree_sim2(u32 base, int H, int steps, SeedFn seed, DurFn dur, bool* overflow) {
   const u32 NM = ~((1u << SS) - 1u);
   for (int i = 0; i < H; ++i) sts64(base + ((u32)(H + i) << SS), (seed(i) << SIM_SLOT_BITS) | i);
   for (int n = H - 1; n >= 1; --n)

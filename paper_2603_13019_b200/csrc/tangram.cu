@@ -344,24 +344,28 @@ static const char* const g_kernel_names[TG_N_KERNELS] = {"k_prefix", "k_select",
                                                           "k_solve", "k_sims", "k_finish"};
 // capacity classes (slots per simulation) of the shared-memory simulation kernels
 static const int g_sim_caps[TG_N_SIM_CLASSES] = {16, 32, 48, 64, 80, 96, 112, 128, 144, 160, 176, 192, 224, 256,
-                                                 320, 352, 384, 400, 416, 432, 440, 448};
+                                                 320, 384, 448, 512, 576, 608, 640, 672};
 #define TG_SMEM_PER_SM 233472   // shared memory an SM can split among resident blocks
 #define TG_SMEM_PER_BLOCK 232448
 
 typedef void (*sims_fn)(const Params, TaskState*, const i64*, const SimLists, int);
-// simulation kernel of a capacity class: path length bound = floor(log2(2 * cap - 1))
-static sims_fn sim_kernel(int cap) {
+// levels below the root of the 4-ary tree of a capacity class
+static int sim_levels(int cap) {
+  long long nodes = tree_nodes(cap), reach = 1, width = 1;
   int d = 0;
-  while ((2 * cap - 1) >> (d + 1)) ++d;
-  switch (d) {
-    case 0: case 1: case 2: case 3: case 4: return k_sims1<4>;
-    case 5: return k_sims1<5>;
-    case 6: return k_sims1<6>;
-    case 7: return k_sims1<7>;
-    case 8: return k_sims1<8>;
-    default: return k_sims1<9>;
+  while (reach < nodes) { width *= 4; reach += width; ++d; }
+  return d;
+}
+static sims_fn sim_kernel(int cap) {
+  switch (sim_levels(cap)) {
+    case 0: case 1: case 2: return k_sims1<2>;
+    case 3: return k_sims1<3>;
+    case 4: return k_sims1<4>;
+    default: return k_sims1<5>;
   }
 }
+// shared memory of a block (32 trees interleaved by lane) of a capacity class
+static int sim_smem_bytes(int cap) { return tree_nodes(cap) * 8 * SIM_PER_WARP + 512; }
 
 static cudaError_t fill_tables() {
   u64 recip[33];
@@ -671,7 +675,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   for (int c = 0; c < TG_N_SIM_CLASSES; ++c) {
     cudaStream_t ss = r->sim_stream[c];
     CK(cudaStreamWaitEvent(ss, r->sim_fork, 0));
-    const int smem = g_sim_caps[c] * SIM_PER_WARP * SIM_SLOT_BYTES + 512;
+    const int smem = sim_smem_bytes(g_sim_caps[c]);
     int per_sm = TG_SMEM_PER_SM / (smem + 1024);
     if (per_sm > 32) per_sm = 32;
     if (per_sm < 1) per_sm = 1;
