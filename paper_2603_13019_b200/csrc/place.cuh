@@ -196,13 +196,13 @@ __device__ __forceinline__ int node_block_start(u32 busy, int bl) {
 // masks before the round (may be null).
 __device__ void place_gpu_reg(const PoolDev& pd, const u8* busy_row, int keep, const u8* cg, const u8* r,
                               int* pnode, int* poff, int lane) {
-  const int top = ilog2(pd.group);
+  const int top = ilog2(pd.group), n_nodes = pd.n_nodes;
   const u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;
   u32 nm[4], lev[4];
 #pragma unroll
   for (int s = 0; s < 4; ++s) {
     const int v = lane + 32 * s;
-    nm[s] = v < pd.n_nodes ? ((busy_row ? busy_row[v] : 0u) | pad) : 0xffu;
+    nm[s] = v < n_nodes ? ((busy_row ? busy_row[v] : 0u) | pad) : 0xffu;
     lev[s] = node_levels(nm[s]);
   }
   for (int lz = top; lz >= 0; --lz) {
@@ -251,10 +251,10 @@ __device__ void place_gpu_reg(const PoolDev& pd, const u8* busy_row, int keep, c
 // Same placement rule as place_cpu_fresh; requires at most 128 domains of fewer than 65536 cores.
 __device__ void place_cpu_fresh_reg(const PoolDev& pd, int keep, const u8* cg, const u8* r,
                                     int* pnode, int* poff, int lane) {
-  const int D = pd.capacity / pd.group;
+  const int G = pd.group, D = pd.capacity / G;
   u32 df[4];
 #pragma unroll
-  for (int s = 0; s < 4; ++s) df[s] = lane + 32 * s < D ? (u32)pd.group : 0u;
+  for (int s = 0; s < 4; ++s) df[s] = lane + 32 * s < D ? (u32)G : 0u;
   for (int i0 = 0; i0 < keep; i0 += 32) {
     const int i = i0 + lane;
     const int mine = i < keep ? (cg[i] & 0x7f) * r[i] : 0;
@@ -266,10 +266,10 @@ __device__ void place_cpu_fresh_reg(const PoolDev& pd, int keep, const u8* cg, c
 #pragma unroll
       for (int s = 0; s < 4; ++s) if (df[s] >= k) key = min(key, (df[s] << 16) | (u32)(lane + 32 * s));
       const u32 best = __reduce_min_sync(TG_FULL, key);
-      int first = -1;
+      int first = -1, dom = -1;
       if (best != 0xffffffffu) {                       // best fit: fewest free cores that still fit
         const int d = (int)(best & 0xffffu), f = (int)(best >> 16);
-        first = d * pd.group + (pd.group - f);
+        first = d * G + (G - f); dom = d;
         if (lane == (d & 31)) {
 #pragma unroll
           for (int s = 0; s < 4; ++s) if (s == (d >> 5)) df[s] -= k;
@@ -282,7 +282,7 @@ __device__ void place_cpu_fresh_reg(const PoolDev& pd, int keep, const u8* cg, c
           for (int s = 0; s < 4; ++s) if (s == (d >> 5)) f = df[s];
           f = __shfl_sync(TG_FULL, f, d & 31);
           if (f == 0) continue;
-          if (first < 0) first = d * pd.group + (pd.group - (int)f);
+          if (first < 0) { first = d * G + (G - (int)f); dom = d; }
           const u32 take = min(f, need);
           if (lane == (d & 31)) {
 #pragma unroll
@@ -291,7 +291,7 @@ __device__ void place_cpu_fresh_reg(const PoolDev& pd, int keep, const u8* cg, c
           need -= take;
         }
       }
-      if (lane == b) { myn = first >= 0 ? first / pd.group : -1; myo = first; }
+      if (lane == b) { myn = dom; myo = first; }
     }
     if (i < keep) { pnode[i] = myn; poff[i] = myo; }
   }
