@@ -81,7 +81,10 @@ typedef struct {
   int32_t max_rounds;   /* replay: rounds per call and rows of `occupancy`; 0 if unused    */
   int32_t host_buffers; /* 0: tangram_actions / tangram_result hold DEVICE pointers;
                            1: they hold HOST pointers and every call copies inputs in and
-                           results out on the given stream (pinned memory recommended)     */
+                           results out (large batches in chunks on internal streams so that
+                           copies and kernels overlap; ordered after the work queued on the
+                           given stream, which in turn waits for the results; use pinned
+                           memory)                                                         */
   int64_t workspace_bytes; /* scratch for large DP tables; 0 = default (8 GiB): 7/8 of it
                               are 48 reusable slots (a DP table must fit one), the rest is bump-allocated             */
   const tangram_pool_desc* pools; /* host array of n_pools entries, copied                 */

@@ -16,6 +16,7 @@
 #define K2_THREADS 256
 #define TG_PROF_CALLS 256   // calls whose kernels can be timed between two queries
 #define TG_N_SIM_CLASSES 22
+#define TG_IO_CHUNKS 16
 #define TG_PROF_K 4         // timed intervals per call at most
 #define TG_N_KERNELS 6
 
@@ -329,6 +330,9 @@ struct tangram_round {
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
   BatchWs W; int sim_blocks; SimLists L; int n_sm;
   ReplayWs R;
+  // host-buffer mode: copy-in, kernels and copy-out of successive chunks on streams of their own
+  cudaStream_t io_in, io_comp, io_out;
+  cudaEvent_t io_begin, io_end, io_in_done[TG_IO_CHUNKS], io_comp_done[TG_IO_CHUNKS];
   // the capacity classes of k_sims are independent: they run on side streams between a fork
   // and a join event so that their partial waves overlap
   cudaStream_t sim_stream[TG_N_SIM_CLASSES + 1];
@@ -513,6 +517,15 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
     bad |= cudaEventCreateWithFlags(&r->sim_join[c], cudaEventDisableTiming) != cudaSuccess;
   }
   if (!bad && desc->host_buffers) {
+    bad |= cudaStreamCreateWithFlags(&r->io_in, cudaStreamNonBlocking) != cudaSuccess;
+    bad |= cudaStreamCreateWithFlags(&r->io_comp, cudaStreamNonBlocking) != cudaSuccess;
+    bad |= cudaStreamCreateWithFlags(&r->io_out, cudaStreamNonBlocking) != cudaSuccess;
+    bad |= cudaEventCreateWithFlags(&r->io_begin, cudaEventDisableTiming) != cudaSuccess;
+    bad |= cudaEventCreateWithFlags(&r->io_end, cudaEventDisableTiming) != cudaSuccess;
+    for (int c = 0; c < TG_IO_CHUNKS; ++c) {
+      bad |= cudaEventCreateWithFlags(&r->io_in_done[c], cudaEventDisableTiming) != cudaSuccess;
+      bad |= cudaEventCreateWithFlags(&r->io_comp_done[c], cudaEventDisableTiming) != cudaSuccess;
+    }
     size_t off = 0;
     size_t in_sz[8] = {SN, SN, SN * 4, SN * 8, SN * 8, SN * 8, (size_t)P.S * 4, (size_t)P.S * (node0 ? node0 : 1)};
     for (int k = 0; k < 8; ++k) { r->in_off[k] = off; off = align_up(off + in_sz[k], 256); }
@@ -597,6 +610,15 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
   cudaFree(r->R.pst); cudaFree(r->R.win);
+  if (r->io_in) cudaStreamDestroy(r->io_in);
+  if (r->io_comp) cudaStreamDestroy(r->io_comp);
+  if (r->io_out) cudaStreamDestroy(r->io_out);
+  if (r->io_begin) cudaEventDestroy(r->io_begin);
+  if (r->io_end) cudaEventDestroy(r->io_end);
+  for (int c = 0; c < TG_IO_CHUNKS; ++c) {
+    if (r->io_in_done[c]) cudaEventDestroy(r->io_in_done[c]);
+    if (r->io_comp_done[c]) cudaEventDestroy(r->io_comp_done[c]);
+  }
   if (r->sim_fork) cudaEventDestroy(r->sim_fork);
   for (int c = 0; c <= TG_N_SIM_CLASSES; ++c) {
     if (r->sim_stream[c]) cudaStreamDestroy(r->sim_stream[c]);
@@ -605,14 +627,9 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   delete r;
 }
 
-// In host-buffer mode: copy the caller's arrays into the staging area and point P at it.
-static int stage_inputs(tangram_round* r, const tangram_actions* a, Params& P, cudaStream_t st) {
-  const size_t SN = (size_t)P.S * P.N;
+// Host-buffer mode: the staging area holds device copies of the caller's arrays.
+static void bind_stage(tangram_round* r, const tangram_actions* a, Params& P) {
   char* d = r->d_stage;
-  const void* src[8] = {a->pool, a->unit, a->level_mask, a->s_us, a->p_us, a->arrival_us, a->n_actions, a->gpu_busy};
-  size_t sz[8] = {SN, SN, SN * 4, SN * 8, SN * 8, SN * 8, (size_t)P.S * 4, (size_t)P.S * P.n_nodes_total};
-  for (int k = 0; k < 8; ++k)
-    if (src[k] && sz[k]) CK(cudaMemcpyAsync(d + r->in_off[k], src[k], sz[k], cudaMemcpyHostToDevice, st));
   P.a_pool = (const u8*)(d + r->in_off[0]); P.a_unit = (const u8*)(d + r->in_off[1]);
   P.a_mask = (const u32*)(d + r->in_off[2]); P.a_s = (const i64*)(d + r->in_off[3]);
   P.a_p = (const i64*)(d + r->in_off[4]);
@@ -622,16 +639,30 @@ static int stage_inputs(tangram_round* r, const tangram_actions* a, Params& P, c
   P.o_alloc = (int*)(d + r->out_off[0]); P.o_node = (int*)(d + r->out_off[1]); P.o_off = (int*)(d + r->out_off[2]);
   P.o_act = (i64*)(d + r->out_off[3]); P.o_total = (i64*)(d + r->out_off[4]); P.o_nsel = (int*)(d + r->out_off[5]);
   P.o_status = (int*)(d + r->out_off[6]);
+}
+
+// inputs of scenarios [s0, s1) host -> staging
+static int copy_in(tangram_round* r, const tangram_actions* a, const Params& P, int s0, int s1, cudaStream_t st) {
+  char* d = r->d_stage;
+  const void* src[8] = {a->pool, a->unit, a->level_mask, a->s_us, a->p_us, a->arrival_us, a->n_actions, a->gpu_busy};
+  const size_t per[8] = {(size_t)P.N, (size_t)P.N, (size_t)P.N * 4, (size_t)P.N * 8, (size_t)P.N * 8, (size_t)P.N * 8,
+                         4, (size_t)P.n_nodes_total};
+  for (int k = 0; k < 8; ++k)
+    if (src[k] && per[k])
+      CK(cudaMemcpyAsync(d + r->in_off[k] + per[k] * s0, (const char*)src[k] + per[k] * s0, per[k] * (s1 - s0),
+                         cudaMemcpyHostToDevice, st));
   return TANGRAM_OK;
 }
 
-static int unstage_outputs(tangram_round* r, const tangram_result* res, const Params& P, cudaStream_t st) {
-  const size_t SN = (size_t)P.S * P.N;
+// results of scenarios [s0, s1) staging -> host
+static int copy_out(tangram_round* r, const tangram_result* res, const Params& P, int s0, int s1, cudaStream_t st) {
   char* d = r->d_stage;
   void* dst[7] = {res->alloc_units, res->place_node, res->place_off, res->act_us, res->total_act_us,
                   res->n_selected, res->status};
-  size_t sz[7] = {SN * 4, SN * 4, SN * 4, SN * 8, (size_t)P.S * 8, (size_t)P.S * 4, (size_t)P.S * 4};
-  for (int k = 0; k < 7; ++k) CK(cudaMemcpyAsync(dst[k], d + r->out_off[k], sz[k], cudaMemcpyDeviceToHost, st));
+  const size_t per[7] = {(size_t)P.N * 4, (size_t)P.N * 4, (size_t)P.N * 4, (size_t)P.N * 8, 8, 4, 4};
+  for (int k = 0; k < 7; ++k)
+    CK(cudaMemcpyAsync((char*)dst[k] + per[k] * s0, d + r->out_off[k] + per[k] * s0, per[k] * (s1 - s0),
+                       cudaMemcpyDeviceToHost, st));
   return TANGRAM_OK;
 }
 
@@ -651,26 +682,19 @@ static void bind_device_io(Params& P, const tangram_actions* a, const tangram_re
   P.o_nsel = res->n_selected; P.o_status = res->status;
 }
 
-extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a, int64_t now_us,
-                                      tangram_result* res, void* cuda_stream) {
-  if (!r || !check_io(a, res)) return TANGRAM_EINVAL;
-  cudaStream_t st = (cudaStream_t)cuda_stream;
-  Params P = r->P;
-  P.now = now_us;
-  if (r->desc.host_buffers) {
-    int rc = stage_inputs(r, a, P, st);
-    if (rc) return rc;
-  } else bind_device_io(P, a, res);
-  CK(cudaMemsetAsync(P.arena_top, 0, 256, st));          // arena top and the task counters
-  cudaEvent_t* ev = prof_begin(r, 0, 3, 4, 5);
+// The kernels of one round for the scenarios that P describes, on stream st.
+static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, const SimLists& L, cudaStream_t st,
+                        cudaEvent_t* ev) {
   const int wblocks = P.n_workers / (K2_THREADS / 32);
+  const long long n_sims = (long long)P.P * P.S * 2;
+  CK(cudaMemsetAsync(P.arena_top, 0, 256, st));          // arena top and the task counters
   if (ev) CK(cudaEventRecord(ev[0], st));
   k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
   if (ev) CK(cudaEventRecord(ev[1], st));
-  k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, r->W);
+  k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
   if (ev) CK(cudaEventRecord(ev[2], st));
-  CK(cudaMemsetAsync(r->L.count, 0, 2 * 64 * sizeof(int), st));
-  k_sim_classify<<<(r->L.n_groups + 255) / 256, 256, 0, st>>>(P, r->W.ts, r->L);
+  CK(cudaMemsetAsync(L.count, 0, 2 * 64 * sizeof(int), st));
+  k_sim_classify<<<(L.n_groups + 255) / 256, 256, 0, st>>>(P, W.ts, L);
   CK(cudaEventRecord(r->sim_fork, st));
   for (int c = 0; c < TG_N_SIM_CLASSES; ++c) {
     cudaStream_t ss = r->sim_stream[c];
@@ -680,18 +704,74 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
     if (per_sm > 32) per_sm = 32;
     if (per_sm < 1) per_sm = 1;
     int grid = r->n_sm * per_sm;
-    if (grid > r->L.n_groups) grid = r->L.n_groups;
-    sim_kernel(g_sim_caps[c])<<<grid, 32, smem, ss>>>(P, r->W.ts, r->W.seed2, r->L, c);
+    if (grid > L.n_groups) grid = L.n_groups;
+    sim_kernel(g_sim_caps[c])<<<grid, 32, smem, ss>>>(P, W.ts, W.seed2, L, c);
     CK(cudaEventRecord(r->sim_join[c], ss));
     CK(cudaStreamWaitEvent(st, r->sim_join[c], 0));
   }
-  k_sims_big<<<r->sim_blocks, 32, 0, st>>>(P, r->W.ts, r->W.seed2, g_sim_caps[TG_N_SIM_CLASSES - 1], r->L.count + 63);
+  k_sims_big<<<(int)((n_sims + 31) / 32), 32, 0, st>>>(P, W.ts, W.seed2, g_sim_caps[TG_N_SIM_CLASSES - 1], L.count + 63);
   if (ev) CK(cudaEventRecord(ev[3], st));
-  k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, r->W);
+  k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
   if (ev) CK(cudaEventRecord(ev[4], st));
   r->launches += 5 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
-  if (r->desc.host_buffers) return unstage_outputs(r, res, P, st);
+  return TANGRAM_OK;
+}
+
+extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a, int64_t now_us,
+                                      tangram_result* res, void* cuda_stream) {
+  if (!r || !check_io(a, res)) return TANGRAM_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Params P = r->P;
+  P.now = now_us;
+  if (!r->desc.host_buffers) {
+    bind_device_io(P, a, res);
+    return run_pipeline(r, P, r->W, r->L, st, prof_begin(r, 0, 3, 4, 5));
+  }
+  bind_stage(r, a, P);
+  // Host buffers: scenarios go through in chunks, so that the copy-in of a chunk, the kernels
+  // of the one before and the copy-out of the one before that overlap (three internal streams).
+  const size_t bytes = (size_t)P.S * P.N * 42;
+  int C = (int)(bytes >> 26);                              // about 64 MiB of traffic per chunk
+  if (C > TG_IO_CHUNKS) C = TG_IO_CHUNKS;
+  if (C > P.S) C = P.S;
+  if (C <= 1 || r->ev) {                                   // small batch, or per-kernel timing wanted
+    int rc = copy_in(r, a, P, 0, P.S, st);
+    if (!rc) rc = run_pipeline(r, P, r->W, r->L, st, prof_begin(r, 0, 3, 4, 5));
+    if (!rc) rc = copy_out(r, res, P, 0, P.S, st);
+    return rc;
+  }
+  CK(cudaEventRecord(r->io_begin, st));
+  CK(cudaStreamWaitEvent(r->io_in, r->io_begin, 0));
+  CK(cudaStreamWaitEvent(r->io_comp, r->io_begin, 0));
+  CK(cudaStreamWaitEvent(r->io_out, r->io_begin, 0));
+  for (int c = 0; c < C; ++c) {
+    const int s0 = (int)((long long)P.S * c / C), s1 = (int)((long long)P.S * (c + 1) / C);
+    const size_t o = (size_t)s0 * P.N;
+    int rc = copy_in(r, a, P, s0, s1, r->io_in);
+    if (rc) return rc;
+    CK(cudaEventRecord(r->io_in_done[c], r->io_in));
+    Params Q = P;                                          // this chunk's view of everything per scenario
+    Q.S = s1 - s0;
+    Q.a_pool += o; Q.a_unit += o; Q.a_mask += o; Q.a_s += o; Q.a_p += o;
+    if (Q.a_arrival) Q.a_arrival += o;
+    Q.n_actions += s0;
+    if (Q.gpu_busy) Q.gpu_busy += (size_t)s0 * P.n_nodes_total;
+    Q.o_alloc += o; Q.o_node += o; Q.o_off += o; Q.o_act += o;
+    Q.o_total += s0; Q.o_nsel += s0; Q.o_status += s0;
+    if ((int64_t)Q.n_workers > (int64_t)Q.S * P.P) Q.n_workers = (int)align_up((size_t)Q.S * P.P, K2_THREADS / 32);
+    SimLists L = r->L;
+    L.n_groups = (int)(((long long)P.P * Q.S * 2 + SIM_PER_WARP - 1) / SIM_PER_WARP);
+    CK(cudaStreamWaitEvent(r->io_comp, r->io_in_done[c], 0));
+    rc = run_pipeline(r, Q, r->W, L, r->io_comp, nullptr);   // the workspace is reused chunk after chunk
+    if (rc) return rc;
+    CK(cudaEventRecord(r->io_comp_done[c], r->io_comp));
+    CK(cudaStreamWaitEvent(r->io_out, r->io_comp_done[c], 0));
+    rc = copy_out(r, res, P, s0, s1, r->io_out);
+    if (rc) return rc;
+  }
+  CK(cudaEventRecord(r->io_end, r->io_out));
+  CK(cudaStreamWaitEvent(st, r->io_end, 0));
   return TANGRAM_OK;
 }
 
@@ -703,7 +783,8 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
   P.now = 0;
   ReplayWs R = r->R;
   if (r->desc.host_buffers) {
-    int rc = stage_inputs(r, a, P, st);
+    bind_stage(r, a, P);
+    int rc = copy_in(r, a, P, 0, P.S, st);
     if (rc) return rc;
     R.occupancy = res->occupancy ? (int*)(r->d_stage + r->out_off[7]) : nullptr;
     R.rounds_used = res->rounds_used ? (int*)(r->d_stage + r->out_off[8]) : nullptr;
@@ -720,7 +801,7 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
   r->launches += 1;
   CK(cudaGetLastError());
   if (r->desc.host_buffers) {
-    int rc = unstage_outputs(r, res, P, st);
+    int rc = copy_out(r, res, P, 0, P.S, st);
     if (rc) return rc;
     if (res->occupancy)
       CK(cudaMemcpyAsync(res->occupancy, r->d_stage + r->out_off[7],

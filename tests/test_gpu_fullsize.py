@@ -49,3 +49,20 @@ def test_full_size_sampled_scenarios_match_oracle(oracle, name, n_sample):
         if p.type == POOL_GPU and a["gpu_busy"] is not None:
             busy = np.unpackbits(a["gpu_busy"], axis=1).sum(1)
         assert np.all(used + busy <= p.capacity)
+
+
+def test_host_buffers_in_chunks_give_the_same_results():
+    """A batch large enough to go through the host-buffer path in several chunks (copy-in,
+    kernels and copy-out of successive chunks overlap) must equal the device-buffer run."""
+    import torch
+    from paper_2603_13019_b200 import binding
+    w, a, g = _run_full("cfg1")                                  # 4096 x 1024: 176 MB of traffic, 2 chunks
+    S, N = w.n_scenarios, w.max_actions
+    rnd = binding.Round(S, N, w.pools, depth=w.depth, host_buffers=True)
+    hin = binding.to_device(a, pin=True)
+    for _ in range(2):                                           # twice: the staging area is reused
+        out = rnd.schedule_batch(hin)
+        torch.cuda.synchronize()
+        for k in KEYS:
+            assert np.array_equal(out[k].numpy(), g[k]), k
+    rnd.destroy()
