@@ -224,6 +224,8 @@ def main():
     ktimes = rnd.kernel_times()
     launches = rnd.kernel_launches - launches0
     rnd.set_profiling(False)
+    act = res["act_us"]
+    mean_act = float(act[act >= 0].double().mean().item()) if bool((act >= 0).any().item()) else None
     status_bad = int((res["status"] != 0).sum().item())
     n_sel = int(res["n_selected"].sum().item())
 
@@ -275,7 +277,8 @@ def main():
                        "l2": "inputs+outputs %.0f MB per step, larger than L2" % (ALGO_BYTES_PER_ACTION * S * N / 1e6)
                        if ALGO_BYTES_PER_ACTION * S * N > 126e6 else "working set below L2; no flush",
                        "parallelism": "independent replicas" if world > 1 else "single GPU",
-                       "selected_actions": n_sel, "scenarios_with_status": status_bad},
+                       "selected_actions": n_sel, "scenarios_with_status": status_bad,
+                       "mean_act_us": mean_act},
             "clocks": clocks,
             "e2e": None if e2e is None else {"value": acts * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": "actions/s",
                                              "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],

@@ -172,7 +172,30 @@ def _replay_trace(w: Workload, d: _Draws, S: int, N: int):
     return dict(pool=pool, unit=unit, level_mask=mask, s_us=s, p_us=p, arrival_us=arrival)
 
 
-_RECIPES = {"mixed": _mixed_round, "topology": _topology_round, "replay": _replay_trace}
+def _ablation_trace(w: Workload, d: _Draws, S: int, N: int):
+    """Scheduling ablation (elastic against fixed degree of parallelism) on a coding-like trace:
+    one CPU pool; short one-core code executions and long, parallelisable reward calculations
+    (5 % serial part).  params["dop"] = 0 makes the reward calculations elastic over
+    1, 2, 4, ..., 32 cores, any other value pins them to that many cores."""
+    P = w.params
+    gap = np.floor(-np.log(d.uniform(_F_ARR)) * (1e6 / P["rate_per_s"])).astype(np.int64)
+    arrival = np.cumsum(gap, axis=1)
+    reward = d.uniform(_F_POOL) < P["reward_fraction"]
+    t_exec = np.minimum(np.floor(P["pareto_min_us"] * d.uniform(_F_DUR) ** (-1.0 / P["pareto_alpha"])),
+                        float(1 << 40)).astype(np.int64)
+    t_rew = d.lognormal_us(_F_S, P["reward_median_us"], P["reward_sigma"])
+    s_rew = t_rew // 20
+    s = np.where(reward, s_rew, t_exec)
+    p = np.where(reward, t_rew - s_rew, 0)
+    dop = int(P["dop"])
+    rew_mask = _pow2_mask(32) if dop == 0 else 1 << (dop - 1)
+    mask = np.where(reward, rew_mask, 1).astype(np.uint32)
+    return dict(pool=np.zeros((S, N), np.uint8), unit=np.ones((S, N), np.uint8), level_mask=mask,
+                s_us=s, p_us=p, arrival_us=arrival)
+
+
+_RECIPES = {"mixed": _mixed_round, "topology": _topology_round, "replay": _replay_trace,
+            "ablation": _ablation_trace}
 
 
 def _busy_masks(w: Workload, lo: int, hi: int) -> Optional[np.ndarray]:
@@ -231,6 +254,19 @@ CONFIGS: Dict[str, Workload] = {
                      "mixed", params=dict(mix=(0.50, 0.25, 0.15, 0.10), max_level=32, inelastic=0.35,
                                           sigma_s=2.0, sigma_p=2.0, outliers=0.01)),
 }
+
+
+def _ablation(dop: int) -> Workload:
+    return Workload("abl_dop%d" % dop if dop else "abl_elastic", 64, 4000, (Pool(POOL_CPU, 256, _CPU_NUMA),),
+                    "ablation", replay=True, max_rounds=12_000,
+                    params=dict(rate_per_s=110.0, reward_fraction=0.20, pareto_alpha=1.3, pareto_min_us=5_000.0,
+                                reward_median_us=4_000_000.0, reward_sigma=1.0, dop=dop))
+
+
+# scheduling ablation on a synthetic coding-like trace: elastic 1..32 against fixed DoP 4 and 16
+for _d in (0, 4, 16):
+    _w = _ablation(_d)
+    CONFIGS[_w.name] = _w
 
 
 def make_workload(name: str, n_scenarios: Optional[int] = None, max_actions: Optional[int] = None,
