@@ -311,8 +311,9 @@ __device__ __forceinline__ int nth_level(u32 mask, int d) {
 }
 
 // Completion-heap estimate (Algorithm 2, estimate) of everything that is not in the prefix
-// [0, q): evicted candidates first, then the pool's waiting actions.  Lane d simulates depth d+1.
-__device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab slab, int lane, i64* est) {
+// [0, q), whose multiplicities are alloc[0..q): evicted candidates first, then the pool's waiting
+// actions.  Lane d simulates depth d+1.
+__device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, const u8* alloc, Slab slab, int lane, i64* est) {
   const int n_ev = T.m - q;
   const int n_rest = n_ev + T.n_ac;
   if (n_rest == 0) { *est = 0; return true; }
@@ -330,7 +331,7 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab sl
       val = tree_sim2<9, 3>(
           T.sim_base, H, n_rest,
           [&](int i) { return i < T.n_seeds ? T.seeds[i]
-                                            : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], T.rsel[i - T.n_seeds]); },
+                                            : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], alloc[i - T.n_seeds]); },
           [&](int k) { return k == 0 ? fd
                             : (k < n_ev ? duration(T.cs[q + k], T.cp[q + k], __ffs(T.cmask[q + k])) : T.ac_tmin[k - n_ev]); },
           &overflow);
@@ -346,7 +347,7 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab sl
   for (int d = 0; d < dmax; ++d)
     for (int i = lane; i < H; i += 32)
       heaps[(u64)d * H + i] = i < T.n_seeds ? T.seeds[i]
-                                            : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], T.rsel[i - T.n_seeds]);
+                                            : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], alloc[i - T.n_seeds]);
   __syncwarp();
   i64 tmp = TG_INF;
   if (lane < dmax) {
@@ -385,15 +386,47 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, Slab sl
   return true;
 }
 
+// An eviction step that cannot pay.  Let the first q+1 candidates be kept with multiplicities
+// `kept`, and let `fewer` be the optimal multiplicities of the first q alone.  If the two agree on
+// the first q candidates and candidate q's kept duration is no longer than at the largest level
+// the estimate would try for it, then objective(q) >= objective(q+1):
+//   * both objectives share the duration sum of the first q candidates;
+//   * with q+1 kept, candidate q adds T_q(kept) and occupies one completion slot from T_q(kept) on;
+//     with q kept, it is the first waiting action: it adds ts + T_q(level d) >= T_q(kept), where
+//     ts >= 0 is the earliest completion, and that slot is busy until then;
+//   * so the completion multiset after the step dominates the other one slot by slot (the slot
+//     the smaller list lacks counts as never free), dominance survives every further
+//     "pop the earliest, push earliest + T" step, every popped time is >=, and every later
+//     waiting action runs at its least level in the first sum and at that or a larger level in
+//     the second.
+// Algorithm 1 stops at the first step whose objective does not decrease, so neither estimate is
+// needed.  Warp-uniform result.
+__device__ __forceinline__ bool eviction_cannot_pay(const PoolTask& T, int q, const u8* kept, const u8* fewer,
+                                                    int lane) {
+  bool same = true;
+  for (int i = lane; i < q; i += 32) same &= kept[i] == fewer[i];
+  if (!__all_sync(TG_FULL, same)) return false;
+  const u32 mk = T.cmask[q];
+  const int dmax = min(T.depth, __popc(mk));
+  return duration(T.cs[q], T.cp[q], kept[q]) <= duration(T.cs[q], T.cp[q], nth_level_of(mk, dmax - 1));
+}
+
 // Greedy eviction (Algorithm 1, lines 8-14), continued from a state in which the first `keep`
-// candidates are kept with objective `obj` and multiplicities T.rkeep.  Returns the number of
+// candidates are kept with multiplicities T.rkeep and duration sum `opt_keep`; `obj` is their
+// objective if `have_obj`, else it is computed when first needed.  Returns the number of
 // candidates finally kept, or -1 if the workspace is too small.
-__device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int lane, i64 obj, int keep) {
+__device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int lane, i64 obj, int keep,
+                            bool have_obj = true, i64 opt_keep = 0) {
   i64 opt, est;
   for (int t = T.m - keep + 1; t <= T.m - 1; ++t) {
     const int q = T.m - t;
     if (!solve_prefix(P, T, q, slab, lane, &opt)) return -1;
-    if (!estimate_rest(P, T, q, slab, lane, &est)) return -1;
+    if (eviction_cannot_pay(T, q, T.rkeep, T.rsel, lane)) break;
+    if (!have_obj) {
+      if (!estimate_rest(P, T, keep, T.rkeep, slab, lane, &est)) return -1;
+      obj = sat_add(opt_keep, est); have_obj = true;
+    }
+    if (!estimate_rest(P, T, q, T.rsel, slab, lane, &est)) return -1;
     i64 nobj = sat_add(opt, est);
     if (nobj >= obj) break;
     obj = nobj; keep = q;
@@ -405,10 +438,9 @@ __device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int l
 
 // The whole loop, starting from the full candidate list.
 __device__ int evict_loop(const Params& P, const PoolTask& T, Slab slab, int lane) {
-  i64 opt, est;
+  i64 opt;
   if (!solve_prefix(P, T, T.m, slab, lane, &opt)) return -1;
-  if (!estimate_rest(P, T, T.m, slab, lane, &est)) return -1;
   for (int i = lane; i < T.m; i += 32) T.rkeep[i] = T.rsel[i];
   __syncwarp();
-  return evict_resume(P, T, slab, lane, sat_add(opt, est), T.m);
+  return evict_resume(P, T, slab, lane, 0, T.m, false, opt);
 }

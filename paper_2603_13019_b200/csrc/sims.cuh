@@ -44,6 +44,7 @@ struct TaskState {
 #define TS_SOLVED 1   // both prefixes solved, heap seeds written
 #define TS_FAILED 2   // workspace too small
 #define TS_REDO0 4    // simulation of prefix e overflowed the packed keys: bit TS_REDO0 << e
+#define TS_DECIDED 16 // placed and written by the solve kernel: no estimate needed
 
 __device__ __forceinline__ int nth_level_of(u32 mask, int d) {
   for (int k = 0; k < d; ++k) mask &= mask - 1;

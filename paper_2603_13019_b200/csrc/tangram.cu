@@ -25,11 +25,13 @@
 //   k_select            everything in one kernel (general path: any number of evictions,
 //                       running actions in the heap; used by the allocation-free entry point),
 //   k_solve / k_finish  the batched path: k_solve computes the optimal allocations of the full
-//                       candidate list and of the list without its last candidate, k_sims
-//                       (sims.cuh) runs all completion-heap simulations one thread each,
-//                       k_finish compares the two objectives (Algorithm 1, lines 8-14), goes on
-//                       evicting in the rare case the first eviction pays, places the grants
-//                       and writes the candidates' outputs (Eq. 2).
+//                       candidate list and of the list without its last candidate; a pool
+//                       without elastic candidates, or whose first eviction step cannot pay
+//                       (eviction_cannot_pay), is placed and written at once.  For the others
+//                       k_sims (sims.cuh) runs the completion-heap simulations one thread
+//                       each, and k_finish compares the two objectives (Algorithm 1, lines
+//                       8-14), goes on evicting where the first eviction pays, places the
+//                       grants and writes the candidates' outputs (Eq. 2).
 // ---------------------------------------------------------------------------------------
 // Tasks are handed out by a counter so that long tasks do not pile up on the same warps.
 __device__ __forceinline__ int next_task(u64* counter, int lane) {
@@ -218,62 +220,74 @@ struct BatchWs {
 __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Params P, const BatchWs W) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
-  const int nw = (gridDim.x * K2_THREADS) >> 5;
   const int n_tasks = P.S * P.P;
-  (void)nw;
   for (;;) {
     const int x = next_task(P.arena_top + 1, lane);
     if (x >= n_tasks) break;
     const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
     const PoolMeta mt = P.meta[task];
     TaskState* st = W.ts + task;
-    if (mt.m == 0 || !mt.elastic) { if (lane == 0) st->flags = 0; continue; }
+    if (mt.m == 0) { if (lane == 0) st->flags = TS_DECIDED; continue; }
     Slab slab = warp_slab(P, gw);
     CandArrays C;
-    bool ok = gather_candidates(P, sc, j, mt, slab, lane, C);
-    i64 opt0 = 0, opt1 = 0;
-    if (ok) {
+    if (!gather_candidates(P, sc, j, mt, slab, lane, C)) {
+      if (lane == 0) { atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); st->flags = TS_DECIDED; }
+      continue;
+    }
+    // A pool is decided here unless its first eviction step needs the two estimates.
+    int keep = mt.m;
+    bool decided = true;
+    if (mt.elastic) {
       PoolTask T;
       make_task(P, sc, j, mt, C, lane, T);
-      const size_t pos = (size_t)sc * P.N + mt.base;
-      ok = solve_prefix(P, T, mt.m, slab, lane, &opt0);
+      i64 opt0 = 0, opt1 = 0;
+      bool ok = solve_prefix(P, T, mt.m, slab, lane, &opt0);
       if (ok) {
-        for (int i = lane; i < mt.m; i += 32) {
-          W.rs1[pos + i] = C.rsel[i];
-          P.tmin[pos + i] = duration(C.cs[i], C.cp[i], C.rsel[i]);   // heap seeds of the full list
-        }
+        for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = C.rsel[i];
         __syncwarp();
         if (mt.m >= 2) {
           ok = solve_prefix(P, T, mt.m - 1, slab, lane, &opt1);
-          if (ok)
-            for (int i = lane; i < mt.m - 1; i += 32) {
-              W.rs2[pos + i] = C.rsel[i];
-              W.seed2[pos + i] = duration(C.cs[i], C.cp[i], C.rsel[i]);
+          if (ok && !eviction_cannot_pay(T, mt.m - 1, C.rkeep, C.rsel, lane)) {
+            decided = false;
+            const size_t pos = (size_t)sc * P.N + mt.base;
+            for (int i = lane; i < mt.m; i += 32) {
+              W.rs1[pos + i] = C.rkeep[i];
+              P.tmin[pos + i] = duration(C.cs[i], C.cp[i], C.rkeep[i]);   // heap seeds of the full list
+              if (i < mt.m - 1) {
+                W.rs2[pos + i] = C.rsel[i];
+                W.seed2[pos + i] = duration(C.cs[i], C.cp[i], C.rsel[i]);
+              }
             }
+            if (lane == 0) {
+              st->opt[0] = opt0; st->opt[1] = opt1;
+              st->est[0] = (mt.count - mt.m) > 0 ? TG_INF : 0;
+              st->est[1] = TG_INF;
+              st->flags = TS_SOLVED;
+            }
+          }
         }
       }
+      if (!ok) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
     }
-    if (lane == 0) {
-      st->opt[0] = opt0; st->opt[1] = opt1;
-      st->est[0] = (mt.count - mt.m) > 0 ? TG_INF : 0;
-      st->est[1] = TG_INF;
-      st->flags = ok ? TS_SOLVED : TS_FAILED;
+    if (decided) {
+      place_and_write(P, sc, j, mt, C, keep, slab, lane);
+      if (lane == 0) st->flags = TS_DECIDED;
     }
   }
 }
 
+// The pools whose first eviction step had to be estimated.
 __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ Params P, const BatchWs W) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
-  const int nw = (gridDim.x * K2_THREADS) >> 5;
   const int n_tasks = P.S * P.P;
-  (void)nw;
   for (;;) {
     const int x = next_task(P.arena_top + 2, lane);
     if (x >= n_tasks) break;
     const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
+    const TaskState st = W.ts[task];
+    if (st.flags & TS_DECIDED) continue;
     const PoolMeta mt = P.meta[task];
-    if (mt.m == 0) continue;
     Slab slab = warp_slab(P, gw);
     CandArrays C;
     if (!gather_candidates(P, sc, j, mt, slab, lane, C)) {
@@ -281,28 +295,23 @@ __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ P
       continue;
     }
     int keep = mt.m;
-    if (mt.elastic) {
-      const TaskState st = W.ts[task];
-      if (!(st.flags & TS_SOLVED) || (st.flags & TS_FAILED)) keep = -1;
-      else {
-        const size_t pos = (size_t)sc * P.N + mt.base;
-        i64 obj = sat_add(st.opt[0], st.est[0]);
-        for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = W.rs1[pos + i];
-        if (mt.m >= 2) {
-          i64 nobj = sat_add(st.opt[1], st.est[1]);
-          if (nobj < obj) {                                  // the first eviction pays: go on (rare)
-            for (int i = lane; i < mt.m - 1; i += 32) C.rkeep[i] = W.rs2[pos + i];
-            __syncwarp();
-            PoolTask T;
-            make_task(P, sc, j, mt, C, lane, T);
-            attach_warp_tree(T);
-            keep = evict_resume(P, T, slab, lane, nobj, mt.m - 1);
-          }
-        }
+    if (!(st.flags & TS_SOLVED) || (st.flags & TS_FAILED)) keep = -1;
+    else {
+      const size_t pos = (size_t)sc * P.N + mt.base;
+      i64 obj = sat_add(st.opt[0], st.est[0]);
+      for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = W.rs1[pos + i];
+      i64 nobj = sat_add(st.opt[1], st.est[1]);
+      if (nobj < obj) {                                    // the first eviction pays: go on
+        for (int i = lane; i < mt.m - 1; i += 32) C.rkeep[i] = W.rs2[pos + i];
         __syncwarp();
+        PoolTask T;
+        make_task(P, sc, j, mt, C, lane, T);
+        attach_warp_tree(T);
+        keep = evict_resume(P, T, slab, lane, nobj, mt.m - 1);
       }
-      if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+      __syncwarp();
     }
+    if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
     place_and_write(P, sc, j, mt, C, keep, slab, lane);
   }
 }
