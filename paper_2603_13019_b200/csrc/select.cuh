@@ -120,9 +120,104 @@ __device__ __forceinline__ int best_level(i64 p, u32 mask) {
   return rmax;
 }
 
+// The box DP for boxes of at most 32 cells: lane c owns cell c, the row before lives in a
+// register and a predecessor cell is fetched with one shuffle by the flattened offset.  The rows
+// (T.rowcand[0..nrows)) are taken 32 at a time: every lane first lists, for its own row, the
+// levels that stay inside the box (multiplicity, offset, extra demand per dimension, duration),
+// then the rows are applied one after the other from broadcasts of those lists.  The choices
+// (multiplicity and offset, two bytes per cell and row) go to the warp's shared-memory scratch
+// at `scratch` (64 bytes per row).  Same recurrence and tie order as the general loop in
+// solve_prefix.  Returns 1 when T.rsel holds the optimum; 0 when several end cells tie on value
+// and units or a row has more than DPS_LEVELS levels inside the box (the caller then runs the
+// general loop).
+#define DPS_LEVELS 6
+__device__ int dp_small(const PoolTask& T, int nrows, int ncell, const int ext[4], const int stride[4],
+                        const bool kept[4], u32 scratch, int lane) {
+  // cell coordinates of this lane, one 6-bit field per dimension; bit 5 of a field is a guard
+  // that survives the subtraction of a demand iff the demand does not exceed the coordinate
+  const u32 GUARD = 0x20u | (0x20u << 6) | (0x20u << 12) | (0x20u << 18);
+  u32 pe = GUARD;
+  int e0 = 0;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    const int el = (lane / stride[l]) % ext[l];
+    if (l == 0) e0 = el;
+    pe |= (u32)el << (6 * l);
+  }
+  i64 prev = lane == 0 ? 0 : TG_INF;
+  for (int t0 = 0; t0 < nrows; t0 += 32) {
+    u32 pa[DPS_LEVELS], pb[DPS_LEVELS];                  // r | off << 8 ; demand fields
+    i64 du[DPS_LEVELS];
+    int nl = 0;
+    bool too_many = false;
+#pragma unroll
+    for (int k = 0; k < DPS_LEVELS; ++k) { pa[k] = 0; pb[k] = 0; du[k] = 0; }
+    if (t0 + lane < nrows) {
+      const int i = T.rowcand[t0 + lane];
+      const i64 s = T.cs[i], p = T.cp[i];
+      const u32 mk = T.cmask[i];
+      const int g = T.cg[i] & 0x7f, gang = T.cg[i] >> 7, r0 = __ffs(mk);
+      u32 mm = mk;
+      while (mm) {
+        const int r = __ffs(mm); mm &= mm - 1;
+        int d[4];
+        extra_demand(T.type, g, gang, r0, r, d);
+        u32 off = 0, dls = 0; bool inside = true;
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+          if (kept[l]) { const int dl = d[l] >> l; inside &= dl < ext[l]; off += dl * stride[l]; dls |= (u32)(dl & 31) << (6 * l); }
+        if (!inside) continue;
+        if (nl >= DPS_LEVELS) { too_many = true; break; }
+        const i64 dd = duration(s, p, r);
+#pragma unroll
+        for (int k = 0; k < DPS_LEVELS; ++k) if (k == nl) { pa[k] = (u32)r | (off << 8); pb[k] = dls; du[k] = dd; }
+        ++nl;
+      }
+    }
+    if (__any_sync(TG_FULL, too_many)) return 0;
+    const int nb = min(32, nrows - t0);
+    for (int b = 0; b < nb; ++b) {
+      const int nlb = __shfl_sync(TG_FULL, nl, b);
+      i64 best = TG_INF; u32 bestv = 0;
+#pragma unroll
+      for (int k = 0; k < DPS_LEVELS; ++k) {
+        if (k < nlb) {                                   // levels ascend: the first best one stays
+          const u32 va = __shfl_sync(TG_FULL, pa[k], b), vb = __shfl_sync(TG_FULL, pb[k], b);
+          const i64 dd = __shfl_sync(TG_FULL, du[k], b);
+          const i64 pv = __shfl_up_sync(TG_FULL, prev, va >> 8);
+          const bool ok = ((pe - vb) & GUARD) == GUARD && pv != TG_INF;
+          const i64 cand = pv + dd;
+          if (ok && cand < best) { best = cand; bestv = va; }
+        }
+      }
+      prev = lane < ncell ? best : TG_INF;
+      asm volatile("st.shared.u16 [%0], %1;" :: "r"(scratch + (u32)(t0 + b) * 64u + (u32)lane * 2u), "h"((unsigned short)bestv) : "memory");
+    }
+  }
+  __syncwarp();
+  // best end cell: lowest value, then fewest extra units (index along dimension 0)
+  const i64 bv = warp_min64(prev);
+  if (bv == TG_INF) return 0;
+  const int be = warp_min32(prev == bv ? e0 : INT_MAX);
+  const u32 win = __ballot_sync(TG_FULL, prev == bv && e0 == be);
+  if (__popc(win) != 1) return 0;
+  int c = __ffs(win) - 1;
+  for (int t = nrows - 1; t >= 0; --t) {                 // walk back, every lane the same path
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(scratch + (u32)t * 64u + (u32)c * 2u) : "memory");
+    if (lane == (t & 31)) T.rsel[T.rowcand[t]] = (u8)(v & 0xff);
+    c -= v >> 8;
+  }
+  __syncwarp();
+  return 1;
+}
+
 // Optimal allocation of candidates [0, q) -> T.rsel[0..q), duration sum -> *opt.
+// *all_best tells that every candidate got its best level (then so does every shorter prefix).
 // Returns false if the workspace is too small.
-__device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab slab, int lane, i64* opt) {
+__device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab slab, int lane, i64* opt,
+                             bool* all_best = nullptr) {
+  if (all_best) *all_best = false;
   const bool gpu = T.type == TG_POOL_GPU;
   int dmin[4] = {0, 0, 0, 0}, dbest[4] = {0, 0, 0, 0};
   i64 tmin_sum = 0, tbest_sum = 0;
@@ -152,6 +247,7 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
     for (int i = lane; i < q; i += 32) T.rsel[i] = (u8)best_level(T.cp[i], T.cmask[i]);
     __syncwarp();
     *opt = tbest_sum;
+    if (all_best) *all_best = true;
     return true;
   }
   if (Y[0] <= 0) {
@@ -196,6 +292,14 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
     if (cells > (1ull << 30)) return false;
   }
   const int ncell = (int)cells;
+  __syncwarp();
+  if (ncell <= 32 && T.sim_base && nrows * 4 <= T.sim_cap &&
+      dp_small(T, nrows, ncell, ext, stride, kept, T.sim_base, lane)) {
+    i64 sum = 0;
+    for (int i = lane; i < q; i += 32) sum += duration(T.cs[i], T.cp[i], T.rsel[i]);
+    *opt = warp_sum64(sum);
+    return true;
+  }
   i64* val = (i64*)slab.take(2 * cells * sizeof(i64));
   u8* choice = val ? (u8*)slab.take((u64)nrows * cells) : nullptr;
   int slot = -1;
@@ -322,7 +426,19 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, const u
   else { fs = T.ac_first.s; fp = T.ac_first.p; fm = T.ac_first.mask; }
   const int dmax = min(min(T.depth, __popc(fm)), 32);
   const int H = T.n_seeds + q;
-  if (T.sim_base && H <= T.sim_cap) {
+  if (H <= 128) {
+    // the whole warp on one simulation, one depth (the largest level tried is the best one)
+    bool overflow;
+    const i64 fd = duration(fs, fp, nth_level_of(fm, dmax - 1));
+    const i64 val = warp_sim<4>(
+        H, n_rest,
+        [&](int i) { return i < T.n_seeds ? T.seeds[i]
+                                          : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], alloc[i - T.n_seeds]); },
+        [&](int k) { return k == 0 ? fd
+                          : (k < n_ev ? duration(T.cs[q + k], T.cp[q + k], __ffs(T.cmask[q + k])) : T.ac_tmin[k - n_ev]); },
+        lane, &overflow);
+    if (!overflow) { *est = val; return true; }
+  } else if (T.sim_base && H <= T.sim_cap) {
     // one lane, one depth (the largest level tried is the best one), tree in shared memory
     i64 val = 0; int bad = 0;
     if (lane == 0) {

@@ -266,6 +266,50 @@ __device__ __forceinline__ i64 tree_sim2(u32 base, int H, int steps, SeedFn seed
   return tmp;
 }
 
+// One simulation run by a whole warp: for the single simulations of continued evictions, where
+// the latency of a step is all that counts.  Slot i lives in lane i & 31, register i >> 5
+// (H <= 32 * NS).  A step takes the minimum of the packed keys with two 32-bit warp reductions
+// (high words, then low words among the lanes that tie on the high word); the lane that owns
+// the winning slot replaces it.  Durations are loaded 32 steps at a time, one per lane.
+// Same result and overflow rule as tree_sim2.
+template <int NS, class SeedFn, class DurFn>
+__device__ __forceinline__ i64 warp_sim(int H, int steps, SeedFn seed, DurFn dur, int lane, bool* overflow) {
+  u64 key[NS];
+#pragma unroll
+  for (int j = 0; j < NS; ++j) {
+    const int i = j * 32 + lane;
+    key[j] = i < H ? (((u64)seed(i) << SIM_SLOT_BITS) | (u64)i) : ~0ull;
+  }
+  i64 total = 0;
+  u32 ovf = 0;
+  for (int k0 = 0; k0 < steps; k0 += 32) {
+    const i64 mine = k0 + lane < steps ? dur(k0 + lane) : 0;
+    const int nb = min(32, steps - k0);
+    i64 chunk = 0;                                       // 32 completions < 2^49 each
+    for (int b = 0; b < nb; ++b) {
+      const i64 d = __shfl_sync(TG_FULL, mine, b);
+      u64 lm = key[0];
+#pragma unroll
+      for (int j = 1; j < NS; ++j) lm = key[j] < lm ? key[j] : lm;
+      const u32 hi = (u32)(lm >> 32);
+      const u32 mhi = __reduce_min_sync(TG_FULL, hi);
+      const u32 mlo = __reduce_min_sync(TG_FULL, hi == mhi ? (u32)lm : 0xffffffffu);
+      const u64 top = ((u64)mhi << 32) | mlo;            // earliest completion and its slot
+      const u64 c = top + ((u64)d << SIM_SLOT_BITS);     // pop it, push ts + T into the same slot
+      chunk += (i64)(c >> SIM_SLOT_BITS);
+      ovf |= (u32)(c >> (32 + SIM_SLOT_BITS));
+      const u32 slot = mlo & ((1u << SIM_SLOT_BITS) - 1u);
+      if (lane == (int)(slot & 31u)) {
+#pragma unroll
+        for (int j = 0; j < NS; ++j) if (j == (int)(slot >> 5)) key[j] = c;
+      }
+    }
+    total = sat_add(total, chunk);
+  }
+  *overflow = (ovf >> 17) != 0;                          // a completion >= 2^49
+  return total;
+}
+
 // One persistent warp per block, one lane per simulation (trees interleaved by lane: SS = 8).
 template <int MAXD>
 __global__ void __launch_bounds__(32) k_sims1(const __grid_constant__ Params P, TaskState* ts, const i64* seed2,

@@ -240,12 +240,14 @@ __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Pa
     if (mt.elastic) {
       PoolTask T;
       make_task(P, sc, j, mt, C, lane, T);
+      attach_warp_tree(T);                               // scratch of the small-box DP
       i64 opt0 = 0, opt1 = 0;
-      bool ok = solve_prefix(P, T, mt.m, slab, lane, &opt0);
+      bool all_best;
+      bool ok = solve_prefix(P, T, mt.m, slab, lane, &opt0, &all_best);
       if (ok) {
         for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = C.rsel[i];
         __syncwarp();
-        if (mt.m >= 2) {
+        if (mt.m >= 2 && !all_best) {                      // all at their best level: eviction_cannot_pay holds
           ok = solve_prefix(P, T, mt.m - 1, slab, lane, &opt1);
           if (ok && !eviction_cannot_pay(T, mt.m - 1, C.rkeep, C.rsel, lane)) {
             decided = false;
