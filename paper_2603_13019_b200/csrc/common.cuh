@@ -27,10 +27,11 @@ struct PoolDev {
 
 // per (scenario, pool) facts produced by the prefix kernel
 struct PoolMeta {
-  int base;       // first position of the pool in the scenario's partitioned arrays
-  int count;      // actions of the pool in the queue
+  i64 base;       // the pool's positions in the partitioned arrays start at scenario * max_actions + base
+  int count;      // actions of the pool in the queue (candidates only, if nobody will read its waiting list)
   int m;          // candidates of the pool (they occupy positions base .. base+m-1)
   int elastic;    // some candidate has more than one level
+  int first_wait; // index of the pool's first waiting action, -1 if none (or the list is not needed)
 };
 
 struct Params {

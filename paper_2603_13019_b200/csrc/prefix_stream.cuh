@@ -1,0 +1,305 @@
+// First two kernels of a batched round.
+//
+// k_head, one warp per scenario, walks the queue 32 actions at a time until the candidate
+// prefix ends (Algorithm 1, line 2): lane v keeps the running least-level demand of demand
+// slot v (one slot per core / quota pool, four nested chunk levels per GPU pool), lane j the
+// number of actions of pool j seen so far; a chunk's demand goes through one warp scan per
+// slot and the first action that overflows a slot ends the prefix.  Candidates get their
+// position inside their pool (Algorithm 1, line 4) and their index is written to the pool's
+// part of `order`.  The same walk sums every slot's demand at the candidates' LARGEST levels:
+// where that fits, every candidate gets its best level, no eviction can pay and nobody will
+// read the pool's waiting list.
+//
+// k_stream, one CTA per scenario, streams everything behind the head 4096 actions at a time
+// (16 per thread, 128-bit loads and stores): the "not scheduled" outputs are written, records
+// are validated, and only for the pools that may need an estimate the least-level durations
+// (Eq. 1) of the waiting actions are appended, in queue order, to the pool's list in `tmin`.
+//
+// Partitioned arrays (order, tmin and the solver's arrays) give every (scenario, pool) its own
+// row of max_actions entries, so a position never depends on another pool's count and the
+// queue is read once.
+#pragma once
+#include "common.cuh"
+
+#define KS_THREADS 256
+#define KS_ITEMS 16
+#define KS_TILE (KS_THREADS * KS_ITEMS)
+
+// what k_head leaves for k_stream
+struct HeadState {
+  int hs;                     // first action the stream has to look at (a multiple of 32, or n_actions)
+  u32 need;                   // pools whose waiting list may be read
+  int bad;                    // an invalid record was seen
+  int pad;
+  int cur[TG_MAX_POOLS];      // actions of every pool in [0, hs)
+};
+
+__device__ __forceinline__ int warp_incl_scan32(int x, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { int y = __shfl_up_sync(TG_FULL, x, o); if (lane >= o) x += y; }
+  return x;
+}
+
+__global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, HeadState* hst) {
+  const int lane = threadIdx.x & 31;
+  const int sc = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
+  if (sc >= P.S) return;
+  const size_t row = (size_t)sc * P.N;
+  const size_t prow = (size_t)sc * P.P * P.N;       // pool j's part starts at prow + j * N
+  const int n_act = min(max(P.n_actions[sc], 0), P.N);
+  const int D = P.V - P.P;                          // demand slots
+
+  // lane v < D: capacity, running least-level demand and candidates' largest-level demand of slot v
+  // lane j < P: actions / candidates / first waiting action of pool j, and the pool's description
+  int capreg = 0, run = 0, mxd = 0, cnt = 0, mreg = 0, fwreg = -1;
+  u32 pinfo = 0;                                    // type | GPUs per node << 4 | slot0 << 8
+  for (int j = 0; j < P.P; ++j) {
+    const PoolDev& pd = P.pool[j];
+    if (pd.type == TG_POOL_GPU) {
+      int cap[4];
+      gpu_caps(pd, P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr, lane, cap);
+#pragma unroll
+      for (int l = 0; l < 4; ++l) if (lane == pd.slot0 + l) capreg = cap[l];
+    } else if (lane == pd.slot0) capreg = pd.capacity;
+    if (lane == j) pinfo = (u32)pd.type | ((u32)(pd.type == TG_POOL_GPU ? pd.group : 0) << 4) | ((u32)pd.slot0 << 8);
+  }
+
+  u32 el = 0, need = 0;
+  bool bad = false;
+  int hs = n_act;
+  const u32 lt = (1u << lane) - 1u;
+  for (int c0 = 0; c0 < n_act; c0 += 32) {
+    const int i = c0 + lane;
+    const bool present = i < n_act;
+    int j = 0; u32 un = 0, mk = 0; i64 s = 0, p = 0;
+    if (present) { j = P.a_pool[row + i]; un = P.a_unit[row + i]; mk = P.a_mask[row + i]; s = P.a_s[row + i]; p = P.a_p[row + i]; }
+    bool valid = present && j < P.P;
+    const u32 pi = __shfl_sync(TG_FULL, pinfo, valid ? j : 0);
+    PoolDev pd;
+    pd.type = pi & 15; pd.group = (pi >> 4) & 15;
+    const int slot0 = pi >> 8;
+    int g = 1, gang = 0; u32 eff = 1;
+    if (valid) valid = decode_levels(pd, (u8)un, mk, g, gang, eff);
+    bad |= present && !valid;
+    const bool gpu = pd.type == TG_POOL_GPU;
+    const int rmin = __ffs(eff), rmax = 32 - __clz(eff);
+    const int units = g * rmin, mxu = g * rmax;
+    const int lz = gpu ? level_of(g, gang, rmin) : 0, lzx = gpu ? level_of(g, gang, rmax) : 0;
+    // least-level demand: one scan per slot; the first action that overflows a slot ends the prefix
+    bool over = false;
+    for (int v = 0; v < D; ++v) {
+      const int c = (valid && v >= slot0 && v <= slot0 + lz) ? units : 0;
+      const int incl = warp_incl_scan32(c, lane);
+      const int rv = __shfl_sync(TG_FULL, run, v), cv = __shfl_sync(TG_FULL, capreg, v);
+      over |= c > 0 && rv + incl > cv;
+      const int tot = __shfl_sync(TG_FULL, incl, 31);
+      if (lane == v) run += tot;
+    }
+    const u32 ob = __ballot_sync(TG_FULL, over);
+    const int f = ob ? __ffs(ob) - 1 : 32;           // lanes >= f wait
+    const bool cand = valid && lane < f;
+    // position inside the pool
+    int pos = 0;
+    for (int jj = 0; jj < P.P; ++jj) {
+      const u32 b = __ballot_sync(TG_FULL, valid && j == jj);
+      const u32 bc = __ballot_sync(TG_FULL, cand && j == jj);
+      const int cj = __shfl_sync(TG_FULL, cnt, jj);
+      if (valid && j == jj) pos = cj + __popc(b & lt);
+      if (lane == jj) { cnt += __popc(b); mreg += __popc(bc); }
+    }
+    if (cand) {
+      P.order[prow + (size_t)j * P.N + pos] = i;
+      if (eff & (eff - 1)) el |= 1u << j;
+    }
+    for (int v = 0; v < D; ++v) {
+      const int c = (cand && v >= slot0 && v <= slot0 + lzx) ? mxu : 0;
+      const int tot = __reduce_add_sync(TG_FULL, c);
+      if (lane == v) mxd += tot;
+    }
+    if (ob) {
+      // The prefix is complete.  A pool may need its waiting list only if one of its candidates
+      // is elastic and the candidates' largest levels do not all fit.
+      const u32 unfit = __ballot_sync(TG_FULL, lane < D && mxd > capreg);
+      const u32 elw = __reduce_or_sync(TG_FULL, el);
+      for (int jj = 0; jj < P.P; ++jj) {
+        const u32 slots = ((1u << P.pool[jj].n_slots) - 1u) << P.pool[jj].slot0;
+        if (((elw >> jj) & 1u) && (unfit & slots)) need |= 1u << jj;
+      }
+      const int mj = __shfl_sync(TG_FULL, mreg, valid ? j : 0);
+      const bool waits = valid && lane >= f;
+      if (waits) {
+        P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1;
+        if ((need >> j) & 1u)
+          P.tmin[prow + (size_t)j * P.N + pos] = duration(clamp_param(s), clamp_param(p), rmin);
+      }
+      for (int jj = 0; jj < P.P; ++jj) {               // the pool's first waiting action
+        const u32 b = __ballot_sync(TG_FULL, waits && j == jj && pos == mj);
+        if (lane == jj && b) fwreg = c0 + __ffs(b) - 1;
+      }
+      hs = min(c0 + 32, n_act);
+      break;
+    }
+  }
+  const u32 elw = __reduce_or_sync(TG_FULL, el);
+  const int anybad = __any_sync(TG_FULL, bad) ? 1 : 0;
+  if (lane < P.P) {
+    PoolMeta mt;
+    mt.base = (i64)sc * (P.P - 1) * P.N + (i64)lane * P.N;   // row + base = prow + lane * N
+    mt.count = cnt; mt.m = mreg; mt.elastic = (elw >> lane) & 1u; mt.first_wait = fwreg;
+    P.meta[(size_t)sc * P.P + lane] = mt;
+    hst[sc].cur[lane] = cnt;
+  }
+  if (lane == 0) { hst[sc].hs = hs; hst[sc].need = need; hst[sc].bad = anybad; }
+}
+
+// exclusive scan of one int per thread over the CTA; *total = sum.  wsum: 8 ints of scratch.
+__device__ __forceinline__ int ks_block_scan(int x, int* wsum, int t, int* total) {
+  const int lane = t & 31, warp = t >> 5;
+  const int incl = warp_incl_scan32(x, lane);
+  if (lane == 31) wsum[warp] = incl;
+  __syncthreads();
+  int off = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < KS_THREADS / 32; ++w) { const int v = wsum[w]; if (w < warp) off += v; tot += v; }
+  __syncthreads();
+  *total = tot;
+  return off + incl - x;
+}
+
+__global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant__ Params P, const HeadState* hst) {
+  __shared__ int s_m[TG_MAX_POOLS], s_first[TG_MAX_POOLS], s_cur[TG_MAX_POOLS], s_scan[KS_THREADS / 32];
+  __shared__ int s_bad;
+  __shared__ u32 s_pinfo[TG_MAX_POOLS];             // type | GPUs per node << 4, 0xf for "no such pool"
+
+  const int sc = blockIdx.x, t = threadIdx.x;
+  const size_t row = (size_t)sc * P.N;
+  const size_t prow = (size_t)sc * P.P * P.N;
+  const int n_act = min(max(P.n_actions[sc], 0), P.N);
+  const HeadState H = hst[sc];
+  const u32 need = H.need;
+  const bool vec = (P.N % 16 == 0) &&
+                   ((((size_t)P.a_pool | (size_t)P.a_unit | (size_t)P.a_mask | (size_t)P.a_s | (size_t)P.a_p |
+                      (size_t)P.o_alloc | (size_t)P.o_node | (size_t)P.o_off | (size_t)P.o_act) & 15) == 0);
+  if (t < TG_MAX_POOLS) {
+    s_m[t] = t < P.P ? P.meta[(size_t)sc * P.P + t].m : 0;
+    s_first[t] = INT_MAX;
+    s_pinfo[t] = t < P.P ? (u32)P.pool[t].type | ((u32)(P.pool[t].type == TG_POOL_GPU ? P.pool[t].group : 0) << 4) : 0xfu;
+  }
+  if (t == 0) s_bad = H.bad;
+  __syncthreads();
+
+  int cur[TG_MAX_POOLS];                              // actions of every pool seen so far
+#pragma unroll
+  for (int j = 0; j < TG_MAX_POOLS; ++j) cur[j] = H.cur[j];
+  for (int tile0 = H.hs; tile0 < n_act; tile0 += KS_TILE) {   // a bad scenario is streamed on: its rows are rewritten below
+    const int i_first = tile0 + t * KS_ITEMS;
+    const bool full = vec && i_first + KS_ITEMS <= n_act;
+    // "not scheduled" outputs: they depend on nothing, so they go first
+    if (full) {
+      const int4 z = make_int4(0, 0, 0, 0), m1 = make_int4(-1, -1, -1, -1);
+      const longlong2 a1 = make_longlong2(-1, -1);
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; k += 4) {
+        *(int4*)(P.o_alloc + row + i_first + k) = z;
+        *(int4*)(P.o_node + row + i_first + k) = m1;
+        *(int4*)(P.o_off + row + i_first + k) = m1;
+      }
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; k += 2) *(longlong2*)(P.o_act + row + i_first + k) = a1;
+    } else {
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; ++k) {
+        const int i = i_first + k;
+        if (i < n_act) { P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1; }
+      }
+    }
+    u8 rp[KS_ITEMS], ru[KS_ITEMS];
+    u32 rm[KS_ITEMS];
+    if (full) {
+      *(uint4*)rp = *(const uint4*)(P.a_pool + row + i_first);
+      *(uint4*)ru = *(const uint4*)(P.a_unit + row + i_first);
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; k += 4) *(uint4*)(rm + k) = *(const uint4*)(P.a_mask + row + i_first + k);
+    } else {
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; ++k) {
+        const int i = i_first + k;
+        rp[k] = i < n_act ? P.a_pool[row + i] : 0;
+        ru[k] = i < n_act ? P.a_unit[row + i] : 1;
+        rm[k] = i < n_act ? P.a_mask[row + i] : 1;
+      }
+    }
+    // validate; keep the least multiplicity of the records whose pool may need its list
+    bool bad = false;
+    u32 rmin4[KS_ITEMS / 4];                          // one byte per record, 0 = not listed
+#pragma unroll
+    for (int k = 0; k < KS_ITEMS / 4; ++k) rmin4[k] = 0;
+#pragma unroll
+    for (int k = 0; k < KS_ITEMS; ++k) {
+      if (!full && i_first + k >= n_act) continue;
+      const int j = rp[k];
+      const u32 pi = s_pinfo[j & (TG_MAX_POOLS - 1)];
+      PoolDev pd;
+      pd.type = pi & 15; pd.group = (pi >> 4) & 15;
+      int g, gang; u32 eff;
+      const bool ok = j < P.P && decode_levels(pd, ru[k], rm[k], g, gang, eff);
+      bad |= !ok;
+      if (ok && ((need >> j) & 1u)) rmin4[k >> 2] |= (u32)__ffs(eff) << (8 * (k & 3));
+    }
+    if (bad) s_bad = 1;
+    // waiting lists of the pools that may need them
+#pragma unroll
+    for (int j = 0; j < TG_MAX_POOLS; ++j) {
+      if (!((need >> j) & 1u)) continue;
+      u32 mine = 0;
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; ++k)
+        if (rp[k] == j && ((rmin4[k >> 2] >> (8 * (k & 3))) & 0xffu)) mine |= 1u << k;
+      int tot;
+      const int ex = ks_block_scan(__popc(mine), s_scan, t, &tot);
+      if (mine) {
+        int pos = cur[j] + ex;
+        const int m_j = s_m[j];
+        i64* dst = P.tmin + prow + (size_t)j * P.N;
+#pragma unroll
+        for (int h = 0; h < KS_ITEMS; h += 8) {          // loads of eight records in flight at once
+          i64 sv[8], pv[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const bool on = (mine >> (h + k)) & 1u;
+            sv[k] = on ? P.a_s[row + i_first + h + k] : 0;
+            pv[k] = on ? P.a_p[row + i_first + h + k] : 0;
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            if (!((mine >> (h + k)) & 1u)) continue;
+            const int rmin = (rmin4[(h + k) >> 2] >> (8 * ((h + k) & 3))) & 0xffu;
+            dst[pos] = duration(clamp_param(sv[k]), clamp_param(pv[k]), rmin);
+            if (pos == m_j) s_first[j] = i_first + h + k;   // the pool's first waiting action
+            ++pos;
+          }
+        }
+      }
+      cur[j] += tot;
+    }
+  }
+  if (t == 0) {
+#pragma unroll
+    for (int j = 0; j < TG_MAX_POOLS; ++j) s_cur[j] = cur[j];
+  }
+  __syncthreads();
+  const bool bad = s_bad != 0;
+  // rows never looked at (beyond the scenario's queue), or everything of a bad scenario
+  for (int i = (bad ? 0 : n_act) + t; i < P.N; i += KS_THREADS) {
+    P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1;
+  }
+  if (t < P.P) {
+    PoolMeta* mt = P.meta + (size_t)sc * P.P + t;
+    if (bad) { mt->count = 0; mt->m = 0; mt->first_wait = -1; }
+    else if ((need >> t) & 1u) {
+      mt->count = s_cur[t];
+      if (s_first[t] != INT_MAX) mt->first_wait = s_first[t];
+    } else mt->count = mt->m;                          // a list nobody reads counts as empty
+  }
+  if (t == 0) { P.o_status[sc] = bad ? TG_ST_BAD_ACTION : 0; P.o_total[sc] = 0; P.o_nsel[sc] = 0; }
+}

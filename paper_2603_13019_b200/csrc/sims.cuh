@@ -87,7 +87,7 @@ __device__ __forceinline__ SimJob sim_job(const Params& P, TaskState* ts, const 
   const PoolDev& pd = P.pool[j];
   // first remaining action: the evicted last candidate (e = 1) or the first waiting one; it takes
   // the largest of its first `depth` levels (see the header for why that depth is the best)
-  const int idx = P.order[row + mt.base + mt.m - e];
+  const int idx = e ? P.order[row + mt.base + mt.m - 1] : mt.first_wait;
   int g, gang; u32 fm;
   decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], g, gang, fm);
   const int d = min(P.depth, __popc(fm)) - 1;

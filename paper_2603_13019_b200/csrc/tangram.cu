@@ -9,6 +9,7 @@
 #include "../../include/tangram.h"
 #include "common.cuh"
 #include "prefix_kernel.cuh"
+#include "prefix_stream.cuh"
 #include "sims.cuh"
 #include "select.cuh"
 #include "place.cuh"
@@ -87,7 +88,7 @@ __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, co
   T.ac_tmin = P.tmin + row + mt.base + mt.m;
   T.ac_first.s = T.ac_first.p = 0; T.ac_first.mask = 1; T.ac_first.g = 1; T.ac_first.gang = 0;
   if (T.n_ac > 0) {
-    int idx = P.order[row + mt.base + mt.m];
+    int idx = mt.first_wait;
     decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], T.ac_first.g, T.ac_first.gang, T.ac_first.mask);
     T.ac_first.s = clamp_param(P.a_s[row + idx]); T.ac_first.p = clamp_param(P.a_p[row + idx]);
   }
@@ -339,6 +340,7 @@ struct tangram_round {
   int64_t launches;
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
+  HeadState* hst;
   BatchWs W; int sim_blocks; SimLists L; int n_sm;
   ReplayWs R;
   // host-buffer mode: copy-in, kernels and copy-out of successive chunks on streams of their own
@@ -485,16 +487,17 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.slab_bytes = slab;
   P.arena_bytes = desc->workspace_bytes ? (u64)desc->workspace_bytes : (8ull << 30);
   bool bad = false;
-  bad |= cudaMalloc(&r->d_order, SN * sizeof(int)) != cudaSuccess;
-  bad |= cudaMalloc(&r->d_tmin, SN * sizeof(i64)) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_order, SN * sizeof(int) * P.P) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_tmin, SN * sizeof(i64) * P.P) != cudaSuccess;
   bad |= cudaMalloc(&r->d_meta, (size_t)P.S * P.P * sizeof(PoolMeta)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->hst, (size_t)P.S * sizeof(HeadState)) != cudaSuccess;
   bad |= cudaMalloc(&r->d_slabs, (size_t)P.n_workers * slab) != cudaSuccess;
   bad |= cudaMalloc(&r->d_arena, P.arena_bytes) != cudaSuccess;
   bad |= cudaMalloc(&r->d_arena_top, 256) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.ts, (size_t)P.S * P.P * sizeof(TaskState)) != cudaSuccess;
-  bad |= cudaMalloc((void**)&r->W.seed2, SN * sizeof(i64)) != cudaSuccess;
-  bad |= cudaMalloc((void**)&r->W.rs1, SN) != cudaSuccess;
-  bad |= cudaMalloc((void**)&r->W.rs2, SN) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.seed2, SN * sizeof(i64) * P.P) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.rs1, SN * P.P) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.rs2, SN * P.P) != cudaSuccess;
   const long long n_sims = (long long)P.P * P.S * 2;
   r->sim_blocks = (int)((n_sims + 31) / 32);
   r->n_sm = prop.multiProcessorCount;
@@ -550,8 +553,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   if (bad) { cudaGetLastError(); tangram_round_destroy(r); return TANGRAM_ENOMEM; }
   P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
-  e = cudaFuncSetAttribute(k_prefix, cudaFuncAttributeMaxDynamicSharedMemorySize, P.V * K1_THREADS * 4);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
+  e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM_REPLAY);
   for (int c = 0; c < TG_N_SIM_CLASSES && e == cudaSuccess; ++c)
@@ -616,7 +618,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
-  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage);
+  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
@@ -700,7 +702,8 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   const long long n_sims = (long long)P.P * P.S * 2;
   CK(cudaMemsetAsync(P.arena_top, 0, 256, st));          // arena top and the task counters
   if (ev) CK(cudaEventRecord(ev[0], st));
-  k_prefix<<<P.S, K1_THREADS, P.V * K1_THREADS * sizeof(int), st>>>(P);
+  k_head<<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
+  k_stream<<<P.S, KS_THREADS, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[1], st));
   k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
   if (ev) CK(cudaEventRecord(ev[2], st));
@@ -724,7 +727,7 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   if (ev) CK(cudaEventRecord(ev[3], st));
   k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
   if (ev) CK(cudaEventRecord(ev[4], st));
-  r->launches += 5 + TG_N_SIM_CLASSES;
+  r->launches += 6 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
   return TANGRAM_OK;
 }
