@@ -181,7 +181,7 @@ int64_t tangram_kernel_launches(const tangram_round* round);
  * events once; from then on every call records events around each of its kernels on the
  * call's stream (up to 256 calls between two switches).  After the caller has synchronised,
  * tangram_kernel_time_ms sums device time and launches of kernel index `kernel`
- * (0 .. 5, named by tangram_kernel_name; the launches of one kernel within a call are timed
+ * (0 .. 7, named by tangram_kernel_name; the launches of one kernel within a call are timed
  * as one interval) since profiling was last switched on;
  * tangram_set_profiling(round, 0) destroys the events. */
 int tangram_set_profiling(tangram_round* round, int enable);

@@ -204,7 +204,7 @@ class Round:
     def kernel_times(self) -> Dict[str, tuple]:
         """tangram_kernel_time_ms for every kernel: name -> (total ms, launches).  Synchronise first."""
         out = {}
-        for k in range(6):
+        for k in range(8):
             ms, n = C.c_double(0.0), C.c_int64(0)
             _check(self._lib.tangram_kernel_time_ms(self._h, k, C.byref(ms), C.byref(n)))
             out[self._lib.tangram_kernel_name(k).decode()] = (ms.value, n.value)

@@ -23,6 +23,7 @@ struct PoolDev {
   int type, capacity, group, window_us;
   int node0, n_nodes;   // GPU pools: first node in a gpu_busy row, node count
   int slot0, n_slots;   // demand slots in the prefix scan (GPU: 4 nested levels, else 1)
+  int lane_place;       // batched path: the pool is placed by k_place, one thread per scenario
 };
 
 // per (scenario, pool) facts produced by the prefix kernel
@@ -49,6 +50,8 @@ struct Params {
   int* order;        // [S][N] action index at each partitioned position
   i64* tmin;         // [S][N] duration at the least level, partitioned order
   PoolMeta* meta;    // [S][P]
+  unsigned short* preq;  // what k_place reads per kept candidate: unit byte | multiplicity << 8 (partitioned order)
+  int* keepn;        // [S][P] candidates kept, -1 = placed elsewhere
   char* slabs; u64 slab_bytes; int n_workers;
   char* arena; u64 arena_bytes; u64* arena_top;
 };

@@ -194,7 +194,23 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
   for (int tile0 = H.hs; tile0 < n_act; tile0 += KS_TILE) {   // a bad scenario is streamed on: its rows are rewritten below
     const int i_first = tile0 + t * KS_ITEMS;
     const bool full = vec && i_first + KS_ITEMS <= n_act;
-    // "not scheduled" outputs: they depend on nothing, so they go first
+    u8 rp[KS_ITEMS], ru[KS_ITEMS];
+    u32 rm[KS_ITEMS];
+    if (full) {
+      *(uint4*)rp = *(const uint4*)(P.a_pool + row + i_first);
+      *(uint4*)ru = *(const uint4*)(P.a_unit + row + i_first);
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; k += 4) *(uint4*)(rm + k) = *(const uint4*)(P.a_mask + row + i_first + k);
+    } else {
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; ++k) {
+        const int i = i_first + k;
+        rp[k] = i < n_act ? P.a_pool[row + i] : 0xff;
+        ru[k] = i < n_act ? P.a_unit[row + i] : 1;
+        rm[k] = i < n_act ? P.a_mask[row + i] : 1;
+      }
+    }
+    // "not scheduled" outputs: they depend on nothing and drain while the loads are in flight
     if (full) {
       const int4 z = make_int4(0, 0, 0, 0), m1 = make_int4(-1, -1, -1, -1);
       const longlong2 a1 = make_longlong2(-1, -1);
@@ -213,21 +229,19 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
         if (i < n_act) { P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1; }
       }
     }
-    u8 rp[KS_ITEMS], ru[KS_ITEMS];
-    u32 rm[KS_ITEMS];
-    if (full) {
-      *(uint4*)rp = *(const uint4*)(P.a_pool + row + i_first);
-      *(uint4*)ru = *(const uint4*)(P.a_unit + row + i_first);
+    // positions in the waiting lists follow from the pool bytes alone, so the CTA-wide scans come
+    // before everything else that the thread does with its records
+    u32 mine[TG_MAX_POOLS];
+    int ex[TG_MAX_POOLS];
 #pragma unroll
-      for (int k = 0; k < KS_ITEMS; k += 4) *(uint4*)(rm + k) = *(const uint4*)(P.a_mask + row + i_first + k);
-    } else {
+    for (int j = 0; j < TG_MAX_POOLS; ++j) {
+      mine[j] = 0; ex[j] = 0;
+      if (!((need >> j) & 1u)) continue;
 #pragma unroll
-      for (int k = 0; k < KS_ITEMS; ++k) {
-        const int i = i_first + k;
-        rp[k] = i < n_act ? P.a_pool[row + i] : 0;
-        ru[k] = i < n_act ? P.a_unit[row + i] : 1;
-        rm[k] = i < n_act ? P.a_mask[row + i] : 1;
-      }
+      for (int k = 0; k < KS_ITEMS; ++k) if (rp[k] == j) mine[j] |= 1u << k;
+      int tot;
+      ex[j] = cur[j] + ks_block_scan(__popc(mine[j]), s_scan, t, &tot);
+      cur[j] += tot;
     }
     // validate; keep the least multiplicity of the records whose pool may need its list
     bool bad = false;
@@ -250,37 +264,28 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
     // waiting lists of the pools that may need them
 #pragma unroll
     for (int j = 0; j < TG_MAX_POOLS; ++j) {
-      if (!((need >> j) & 1u)) continue;
-      u32 mine = 0;
+      if (!mine[j]) continue;
+      int pos = ex[j];
+      const int m_j = s_m[j];
+      i64* dst = P.tmin + prow + (size_t)j * P.N;
 #pragma unroll
-      for (int k = 0; k < KS_ITEMS; ++k)
-        if (rp[k] == j && ((rmin4[k >> 2] >> (8 * (k & 3))) & 0xffu)) mine |= 1u << k;
-      int tot;
-      const int ex = ks_block_scan(__popc(mine), s_scan, t, &tot);
-      if (mine) {
-        int pos = cur[j] + ex;
-        const int m_j = s_m[j];
-        i64* dst = P.tmin + prow + (size_t)j * P.N;
+      for (int h = 0; h < KS_ITEMS; h += 8) {            // loads of eight records in flight at once
+        i64 sv[8], pv[8];
 #pragma unroll
-        for (int h = 0; h < KS_ITEMS; h += 8) {          // loads of eight records in flight at once
-          i64 sv[8], pv[8];
+        for (int k = 0; k < 8; ++k) {
+          const bool on = (mine[j] >> (h + k)) & 1u;
+          sv[k] = on ? P.a_s[row + i_first + h + k] : 0;
+          pv[k] = on ? P.a_p[row + i_first + h + k] : 0;
+        }
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const bool on = (mine >> (h + k)) & 1u;
-            sv[k] = on ? P.a_s[row + i_first + h + k] : 0;
-            pv[k] = on ? P.a_p[row + i_first + h + k] : 0;
-          }
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            if (!((mine >> (h + k)) & 1u)) continue;
-            const int rmin = (rmin4[(h + k) >> 2] >> (8 * ((h + k) & 3))) & 0xffu;
-            dst[pos] = duration(clamp_param(sv[k]), clamp_param(pv[k]), rmin);
-            if (pos == m_j) s_first[j] = i_first + h + k;   // the pool's first waiting action
-            ++pos;
-          }
+        for (int k = 0; k < 8; ++k) {
+          if (!((mine[j] >> (h + k)) & 1u)) continue;
+          const int rmin = (rmin4[(h + k) >> 2] >> (8 * ((h + k) & 3))) & 0xffu;
+          if (rmin) dst[pos] = duration(clamp_param(sv[k]), clamp_param(pv[k]), rmin);   // 0: invalid record, the scenario is flagged
+          if (pos == m_j) s_first[j] = i_first + h + k;   // the pool's first waiting action
+          ++pos;
         }
       }
-      cur[j] += tot;
     }
   }
   if (t == 0) {

@@ -527,6 +527,76 @@ __device__ __forceinline__ bool eviction_cannot_pay(const PoolTask& T, int q, co
   return duration(T.cs[q], T.cp[q], kept[q]) <= duration(T.cs[q], T.cp[q], nth_level_of(mk, dmax - 1));
 }
 
+// Once an eviction has been accepted the loop tends to go on, and every further step is a DP plus
+// a simulation that depend on nothing but the prefix length.  So the next EVB steps are evaluated
+// at once: their DPs one after the other, their simulations side by side, one lane each, on
+// binary winner trees in the warp's shared memory; then the steps are accepted in order while
+// the objective decreases (Algorithm 1, lines 10-14).  Starts from `keep` kept candidates
+// (multiplicities T.rkeep, objective obj).  Returns the number finally kept, -1 if the workspace
+// is too small, -2 if this path does not apply (the caller goes on step by step).
+#define EVB 4
+#define EVB_SLOTS 112       // slots of one of the EVB trees
+__device__ __noinline__ int evict_batch(const Params& P, const PoolTask& T, Slab slab, int lane, i64 obj, int keep) {
+  if (!T.sim_base || T.sim_cap < EVB * EVB_SLOTS || T.n_seeds + keep - 1 > EVB_SLOTS) return -2;
+  u8* rs = (u8*)slab.take((u64)EVB * T.m);
+  if (!rs) return -2;
+  while (keep > 1) {
+    const int keep0 = keep, nb = min(EVB, keep - 1);
+    i64 optk[EVB];
+    u32 stopmask = 0;
+    int cnt = 0;
+#pragma unroll 1
+    for (int k = 0; k < EVB; ++k) {
+      optk[k] = 0;
+      if (k < nb && !stopmask) {
+        PoolTask T2 = T;
+        T2.rsel = rs + (u64)k * T.m;
+        const int q = keep0 - 1 - k;
+        if (!solve_prefix(P, T2, q, slab, lane, &optk[k])) {
+          if (k == 0) return -1;
+          break;                                         // a step the loop may never reach: decided when it comes first
+        }
+        if (eviction_cannot_pay(T, q, k == 0 ? T.rkeep : rs + (u64)(k - 1) * T.m, T2.rsel, lane)) stopmask |= 1u << k;
+        cnt = k + 1;
+      }
+    }
+    // the simulations of the steps that need one: lane k runs step k
+    i64 est = 0;
+    bool redo = false;
+    if (lane < cnt && !((stopmask >> lane) & 1u)) {
+      const int q = keep0 - 1 - lane, n_ev = T.m - q, n_rest = n_ev + T.n_ac;
+      const u8* alloc = rs + (u64)lane * T.m;
+      const u32 fm = T.cmask[q];
+      const i64 fd = duration(T.cs[q], T.cp[q], nth_level_of(fm, min(min(T.depth, __popc(fm)), 32) - 1));
+      est = tree_sim2<7, 3>(
+          T.sim_base + (u32)lane * (EVB_SLOTS * 16), T.n_seeds + q, n_rest,
+          [&](int i) { return i < T.n_seeds ? T.seeds[i]
+                                            : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], alloc[i - T.n_seeds]); },
+          [&](int k) { return k == 0 ? fd
+                            : (k < n_ev ? duration(T.cs[q + k], T.cp[q + k], __ffs(T.cmask[q + k])) : T.ac_tmin[k - n_ev]); },
+          &redo);
+    }
+    __syncwarp();
+    const u32 redomask = __ballot_sync(TG_FULL, redo);   // packed keys overflowed: exact estimate instead
+#pragma unroll 1
+    for (int k = 0; k < EVB; ++k) {
+      if (k >= cnt) break;
+      if ((stopmask >> k) & 1u) return keep;
+      const int q = keep0 - 1 - k;
+      i64 ek = __shfl_sync(TG_FULL, est, k);
+      if ((redomask >> k) & 1u) {
+        if (!estimate_rest(P, T, q, rs + (u64)k * T.m, slab, lane, &ek)) return -1;
+      }
+      const i64 nobj = sat_add(optk[k], ek);
+      if (nobj >= obj) return keep;
+      obj = nobj; keep = q;
+      for (int i = lane; i < q; i += 32) T.rkeep[i] = rs[(u64)k * T.m + i];
+      __syncwarp();
+    }
+  }
+  return keep;
+}
+
 // Greedy eviction (Algorithm 1, lines 8-14), continued from a state in which the first `keep`
 // candidates are kept with multiplicities T.rkeep and duration sum `opt_keep`; `obj` is their
 // objective if `have_obj`, else it is computed when first needed.  Returns the number of
@@ -548,6 +618,8 @@ __device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int l
     obj = nobj; keep = q;
     for (int i = lane; i < q; i += 32) T.rkeep[i] = T.rsel[i];
     __syncwarp();
+    const int kb = evict_batch(P, T, slab, lane, obj, keep);   // an eviction was accepted: look further ahead
+    if (kb != -2) return kb;
   }
   return keep;
 }

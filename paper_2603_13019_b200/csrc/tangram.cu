@@ -18,8 +18,8 @@
 #define TG_PROF_CALLS 256   // calls whose kernels can be timed between two queries
 #define TG_N_SIM_CLASSES 22
 #define TG_IO_CHUNKS 16
-#define TG_PROF_K 4         // timed intervals per call at most
-#define TG_N_KERNELS 6
+#define TG_PROF_K 6         // timed intervals per call at most
+#define TG_N_KERNELS 8
 
 // ---------------------------------------------------------------------------------------
 // Per-(scenario, pool) work of a round, one warp per task.  The pieces are shared by
@@ -125,12 +125,18 @@ __device__ __forceinline__ Slab warp_slab(const Params& P, int gw) {
 
 // placement on a fresh copy of the pool's topology state, then the candidates' outputs
 __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& mt, const CandArrays& C,
-                                int keep, Slab slab, int lane) {
+                                int keep, Slab slab, int lane, bool defer = false) {
   const int m = mt.m;
   const PoolDev& pd = P.pool[j];
   const size_t row = (size_t)sc * P.N;
   const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr;
-  if (pd.type == TG_POOL_GPU) {
+  defer = defer && pd.lane_place;
+  if (defer) {
+    // k_place will place this pool: leave it the kept requests in queue order
+    unsigned short* rq = P.preq + row + mt.base;
+    for (int i = lane; i < keep; i += 32) rq[i] = (unsigned short)(C.cg[i] | ((u32)C.rkeep[i] << 8));
+    if (lane == 0) P.keepn[(size_t)sc * P.P + j] = keep;
+  } else if (pd.type == TG_POOL_GPU) {
     if (pd.n_nodes <= 128) place_gpu_reg(pd, busy_row ? busy_row + pd.node0 : nullptr, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
     else {
     u8* nm = (u8*)slab.take_fast(pd.n_nodes);
@@ -164,7 +170,8 @@ __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& 
       int r = C.rkeep[i];
       i64 arr = P.a_arrival ? P.a_arrival[o] : 0;
       i64 act = (P.now - arr) + duration(C.cs[i], C.cp[i], r);
-      P.o_alloc[o] = (C.cg[i] & 0x7f) * r; P.o_node[o] = C.pnode[i]; P.o_off[o] = C.poff[i]; P.o_act[o] = act;
+      P.o_alloc[o] = (C.cg[i] & 0x7f) * r; P.o_act[o] = act;
+      if (!defer) { P.o_node[o] = C.pnode[i]; P.o_off[o] = C.poff[i]; }
       tot += act; ++cnt;
     } else {
       P.o_alloc[o] = 0; P.o_node[o] = -1; P.o_off[o] = -1; P.o_act[o] = -1;
@@ -228,6 +235,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Pa
     const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
     const PoolMeta mt = P.meta[task];
     TaskState* st = W.ts + task;
+    if (lane == 0) P.keepn[task] = -1;                   // nothing for k_place unless a decision says so
     if (mt.m == 0) { if (lane == 0) st->flags = TS_DECIDED; continue; }
     Slab slab = warp_slab(P, gw);
     CandArrays C;
@@ -273,7 +281,7 @@ __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Pa
       if (!ok) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
     }
     if (decided) {
-      place_and_write(P, sc, j, mt, C, keep, slab, lane);
+      place_and_write(P, sc, j, mt, C, keep, slab, lane, true);
       if (lane == 0) st->flags = TS_DECIDED;
     }
   }
@@ -315,10 +323,11 @@ __global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ P
       __syncwarp();
     }
     if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
-    place_and_write(P, sc, j, mt, C, keep, slab, lane);
+    place_and_write(P, sc, j, mt, C, keep, slab, lane, true);
   }
 }
 
+#include "place_lane.cuh"
 #include "replay.cuh"
 
 // ---------------------------------------------------------------------------------------
@@ -340,7 +349,7 @@ struct tangram_round {
   int64_t launches;
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
-  HeadState* hst;
+  HeadState* hst; void* d_preq; void* d_keepn;
   BatchWs W; int sim_blocks; SimLists L; int n_sm;
   ReplayWs R;
   // host-buffer mode: copy-in, kernels and copy-out of successive chunks on streams of their own
@@ -357,8 +366,8 @@ struct tangram_round {
   cudaEvent_t* ev; int ev_calls, ev_used; int ev_kernel[TG_PROF_CALLS][TG_PROF_K];
 };
 
-static const char* const g_kernel_names[TG_N_KERNELS] = {"k_prefix", "k_select", "k_replay",
-                                                          "k_solve", "k_sims", "k_finish"};
+static const char* const g_kernel_names[TG_N_KERNELS] = {"k_head", "k_select", "k_replay", "k_solve",
+                                                          "k_sims", "k_finish", "k_place", "k_stream"};
 // capacity classes (slots per simulation) of the shared-memory simulation kernels
 static const int g_sim_caps[TG_N_SIM_CLASSES] = {16, 32, 48, 64, 80, 96, 112, 128, 144, 160, 176, 192, 224, 256,
                                                  320, 384, 448, 512, 576, 608, 640, 672};
@@ -435,6 +444,13 @@ static void fill_pool_order(Params& P) {
       if (P.pool[j].type == rank[r]) P.pool_order[k++] = j;
 }
 
+// pools that k_place can take: its per-thread state is 128 bytes of shared memory
+static int lane_place_ok(const PoolDev& d) {
+  if (d.type == TG_POOL_API) return 1;
+  if (d.type == TG_POOL_CPU) return d.capacity / d.group <= KPL_STATE && d.group <= 255;
+  return d.n_nodes <= 64;
+}
+
 extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_round** out) {
   if (!desc || !out || !desc->pools) return TANGRAM_EINVAL;
   if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
@@ -465,6 +481,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
     node0 += d.n_nodes;
     d.slot0 = slot0; d.n_slots = pd.type == TANGRAM_POOL_GPU ? 4 : 1;
     slot0 += d.n_slots;
+    d.lane_place = lane_place_ok(d);
   }
   r->desc.pools = r->pools;
   P.n_nodes_total = node0;
@@ -498,6 +515,8 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc((void**)&r->W.seed2, SN * sizeof(i64) * P.P) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.rs1, SN * P.P) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.rs2, SN * P.P) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->d_preq, SN * P.P * sizeof(unsigned short)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->d_keepn, (size_t)P.S * P.P * sizeof(int)) != cudaSuccess;
   const long long n_sims = (long long)P.P * P.S * 2;
   r->sim_blocks = (int)((n_sims + 31) / 32);
   r->n_sm = prop.multiProcessorCount;
@@ -552,6 +571,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   }
   if (bad) { cudaGetLastError(); tangram_round_destroy(r); return TANGRAM_ENOMEM; }
   P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
+  P.preq = (unsigned short*)r->d_preq; P.keepn = (int*)r->d_keepn;
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
@@ -607,10 +627,11 @@ extern "C" int tangram_kernel_time_ms(tangram_round* r, int kernel, double* tota
 }
 
 // events of the current call, or null when timing is off or the event pool is used up
-static cudaEvent_t* prof_begin(tangram_round* r, int k0, int k1, int k2, int k3) {
+static cudaEvent_t* prof_begin(tangram_round* r, int k0, int k1, int k2, int k3, int k4 = -1, int k5 = -1) {
   if (!r->ev || r->ev_used >= TG_PROF_CALLS) return nullptr;
   int c = r->ev_used++;
   r->ev_kernel[c][0] = k0; r->ev_kernel[c][1] = k1; r->ev_kernel[c][2] = k2; r->ev_kernel[c][3] = k3;
+  r->ev_kernel[c][4] = k4; r->ev_kernel[c][5] = k5;
   return r->ev + c * (TG_PROF_K + 1);
 }
 
@@ -618,7 +639,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
-  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst);
+  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
@@ -703,10 +724,11 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   CK(cudaMemsetAsync(P.arena_top, 0, 256, st));          // arena top and the task counters
   if (ev) CK(cudaEventRecord(ev[0], st));
   k_head<<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
-  k_stream<<<P.S, KS_THREADS, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[1], st));
-  k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
+  k_stream<<<P.S, KS_THREADS, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[2], st));
+  k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
+  if (ev) CK(cudaEventRecord(ev[3], st));
   CK(cudaMemsetAsync(L.count, 0, 2 * 64 * sizeof(int), st));
   k_sim_classify<<<(L.n_groups + 255) / 256, 256, 0, st>>>(P, W.ts, L);
   CK(cudaEventRecord(r->sim_fork, st));
@@ -724,10 +746,12 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
     CK(cudaStreamWaitEvent(st, r->sim_join[c], 0));
   }
   k_sims_big<<<(int)((n_sims + 31) / 32), 32, 0, st>>>(P, W.ts, W.seed2, g_sim_caps[TG_N_SIM_CLASSES - 1], L.count + 63);
-  if (ev) CK(cudaEventRecord(ev[3], st));
-  k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
   if (ev) CK(cudaEventRecord(ev[4], st));
-  r->launches += 6 + TG_N_SIM_CLASSES;
+  k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
+  if (ev) CK(cudaEventRecord(ev[5], st));
+  k_place<<<(P.S * P.P + KPL_THREADS - 1) / KPL_THREADS, KPL_THREADS, 0, st>>>(P);
+  if (ev) CK(cudaEventRecord(ev[6], st));
+  r->launches += 7 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
   return TANGRAM_OK;
 }
@@ -740,7 +764,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   P.now = now_us;
   if (!r->desc.host_buffers) {
     bind_device_io(P, a, res);
-    return run_pipeline(r, P, r->W, r->L, st, prof_begin(r, 0, 3, 4, 5));
+    return run_pipeline(r, P, r->W, r->L, st, prof_begin(r, 0, 7, 3, 4, 5, 6));
   }
   bind_stage(r, a, P);
   // Host buffers: scenarios go through in chunks, so that the copy-in of a chunk, the kernels
@@ -751,7 +775,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   if (C > P.S) C = P.S;
   if (C <= 1 || r->ev) {                                   // small batch, or per-kernel timing wanted
     int rc = copy_in(r, a, P, 0, P.S, st);
-    if (!rc) rc = run_pipeline(r, P, r->W, r->L, st, prof_begin(r, 0, 3, 4, 5));
+    if (!rc) rc = run_pipeline(r, P, r->W, r->L, st, prof_begin(r, 0, 7, 3, 4, 5, 6));
     if (!rc) rc = copy_out(r, res, P, 0, P.S, st);
     return rc;
   }
