@@ -4,93 +4,156 @@
 // The solve and finish kernels leave, per kept candidate in queue order, its unit byte and
 // multiplicity (Params::preq) and the number kept (Params::keepn); this kernel applies the
 // same rules as place.cuh (Sections 5.1-5.3) and writes place_node / place_off.
-// Per-thread state lives in shared memory, byte v of thread t at v * KPL_THREADS + t.
+//
+// A warp holds 32 scenarios of one pool.  Its threads would touch 32 different rows with every
+// load and store, so candidates go through shared memory 32 at a time: for each of the 32
+// scenarios the warp loads that scenario's next 32 requests and indices with one coalesced
+// access each, every thread then places its own scenario's 32 candidates, and the results are
+// written back scenario by scenario.  Shared memory per warp: per-thread state (byte v of lane t
+// at v * 32 + t) and the staged chunk (entry c of lane t at c * 33 + t).
 #pragma once
 #include "common.cuh"
 #include "place.cuh"
 
-#define KPL_THREADS 128
-#define KPL_STATE 128       // state bytes per thread: NUMA domains of a core pool, nodes of a GPU pool
-#define KPL_BATCH 8         // kept candidates whose request and index are loaded at once
-#define KPL_LOAD_BATCH(i0)                                                     \
-  u32 vq[KPL_BATCH]; int vo[KPL_BATCH];                                        \
-  _Pragma("unroll") for (int b_ = 0; b_ < KPL_BATCH; ++b_) {                   \
-    const bool on_ = (i0) + b_ < keep;                                         \
-    vq[b_] = on_ ? rq[(i0) + b_] : 0u;                                         \
-    vo[b_] = on_ ? ord[(i0) + b_] : 0;                                         \
+#define KPL_WARPS 2
+#define KPL_THREADS (32 * KPL_WARPS)
+#define KPL_DOMAINS 128     // NUMA domains of a core pool at most (two state bytes each); a GPU pool has at most 64 nodes
+#define KPL_STATE (2 * KPL_DOMAINS)
+#define KPL_NONE (-2)       // staged result of a candidate that this pass did not place
+
+struct KplWarp {
+  u8 state[KPL_STATE * 32];
+  unsigned short rq[32 * 33];
+  int idx[32 * 33];
+  int off[32 * 33];
+  short node[32 * 33];
+};
+
+// stage requests and indices [c0, c0 + 32) of all 32 scenarios of the warp (eight scenarios'
+// loads in flight at once)
+__device__ __forceinline__ void kpl_load(KplWarp& W, const unsigned short* rq, const int* ord, int keep, int c0, int lane) {
+  for (int s0 = 0; s0 < 32; s0 += 8) {
+    unsigned short vq[8]; int vo[8]; bool on[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int ks = __shfl_sync(TG_FULL, keep, s0 + u);
+      const unsigned short* rs = (const unsigned short*)__shfl_sync(TG_FULL, (unsigned long long)rq, s0 + u);
+      const int* os = (const int*)__shfl_sync(TG_FULL, (unsigned long long)ord, s0 + u);
+      on[u] = c0 + lane < ks;
+      vq[u] = on[u] ? rs[c0 + lane] : (unsigned short)0;
+      vo[u] = on[u] ? os[c0 + lane] : 0;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (on[u]) { W.rq[lane * 33 + s0 + u] = vq[u]; W.idx[lane * 33 + s0 + u] = vo[u]; }
   }
+  __syncwarp();
+}
+// write the staged results of candidates [c0, c0 + 32) of all 32 scenarios
+__device__ __forceinline__ void kpl_store(const Params& P, KplWarp& W, size_t row, int keep, int c0, int lane) {
+  __syncwarp();
+#pragma unroll 8
+  for (int s = 0; s < 32; ++s) {
+    const int ks = __shfl_sync(TG_FULL, keep, s);
+    const size_t rs = (size_t)__shfl_sync(TG_FULL, (unsigned long long)row, s);
+    if (c0 + lane < ks) {
+      const int nd = W.node[lane * 33 + s];
+      if (nd != KPL_NONE) {
+        const size_t o = rs + W.idx[lane * 33 + s];
+        P.o_node[o] = nd; P.o_off[o] = W.off[lane * 33 + s];
+      }
+    }
+  }
+  __syncwarp();
+}
 
 __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ Params P) {
-  __shared__ u8 sm[KPL_STATE * KPL_THREADS];
-  const int x = blockIdx.x * KPL_THREADS + threadIdx.x;
-  if (x >= P.S * P.P) return;
-  const int sc = x % P.S, j = P.pool_order[x / P.S];     // a warp holds 32 scenarios of one pool
+  __shared__ KplWarp s_w[KPL_WARPS];
+  const int lane = threadIdx.x & 31;
+  KplWarp& W = s_w[threadIdx.x >> 5];
+  const int gw = blockIdx.x * KPL_WARPS + (threadIdx.x >> 5);
+  const int wps = (P.S + 31) / 32;                        // warps per pool
+  if (gw >= wps * P.P) return;
+  const int j = P.pool_order[gw / wps], sc = (gw % wps) * 32 + lane;
   const PoolDev& pd = P.pool[j];
   if (!pd.lane_place) return;
-  const int keep = P.keepn[(size_t)sc * P.P + j];
-  if (keep <= 0) return;
-  const size_t row = (size_t)sc * P.N;
-  const PoolMeta mt = P.meta[(size_t)sc * P.P + j];
-  const unsigned short* rq = P.preq + row + mt.base;
-  const int* ord = P.order + row + mt.base;
-  u8* st = sm + threadIdx.x;
+  int keep = sc < P.S ? P.keepn[(size_t)sc * P.P + j] : 0;
+  if (keep < 0) keep = 0;
+  const int maxkeep = warp_max32(keep);
+  if (maxkeep == 0) return;
+  const size_t row = (size_t)(sc < P.S ? sc : 0) * P.N;
+  const i64 base = sc < P.S ? P.meta[(size_t)sc * P.P + j].base : 0;
+  const unsigned short* rq = P.preq + row + base;
+  const int* ord = P.order + row + base;
+  u8* st = W.state + lane;
 
   if (pd.type == TG_POOL_API) {                           // Section 5.1: offset = units consumed before
     int used = 0;
-    for (int i0 = 0; i0 < keep; i0 += KPL_BATCH) {
-      KPL_LOAD_BATCH(i0);
-#pragma unroll
-      for (int b = 0; b < KPL_BATCH; ++b) {
-        if (i0 + b >= keep) break;
-        const u32 v = vq[b];
-        const size_t o = row + vo[b];
-        P.o_node[o] = 0; P.o_off[o] = used;
+    for (int c0 = 0; c0 < maxkeep; c0 += 32) {
+      kpl_load(W, rq, ord, keep, c0, lane);
+      const int nc = min(32, keep - c0);
+      for (int c = 0; c < nc; ++c) {
+        const u32 v = W.rq[c * 33 + lane];
+        W.node[c * 33 + lane] = 0; W.off[c * 33 + lane] = used;
         used += (int)(v & 0x7fu) * (int)(v >> 8);
       }
+      kpl_store(P, W, row, keep, c0, lane);
     }
     return;
   }
 
   if (pd.type == TG_POOL_CPU) {
     // Section 5.2 on a pool nobody occupies yet: cores are taken lowest id first, so the free
-    // count per domain is the whole state; domains at or beyond `frontier` are untouched.
+    // count per domain is the whole state.  Domains at or beyond `frontier` are untouched; of the
+    // touched ones only those with free cores left are kept, as an unordered list of
+    // (domain, free) pairs - full domains can serve nobody, and the list stays short because
+    // small requests keep filling the holes.
     const int G = pd.group, D = pd.capacity / G;
-    int frontier = 0;
-    for (int i0 = 0; i0 < keep; i0 += KPL_BATCH) {
-      KPL_LOAD_BATCH(i0);
-#pragma unroll
-      for (int b = 0; b < KPL_BATCH; ++b) {
-        if (i0 + b >= keep) break;
-        const u32 v = vq[b];
+    u8* od = st;                                          // open domain ids
+    u8* of = st + KPL_DOMAINS * 32;                       // their free cores
+    int frontier = 0, n_open = 0;
+    for (int c0 = 0; c0 < maxkeep; c0 += 32) {
+      kpl_load(W, rq, ord, keep, c0, lane);
+      const int nc = min(32, keep - c0);
+      for (int c = 0; c < nc; ++c) {
+        const u32 v = W.rq[c * 33 + lane];
         const int k = (int)(v & 0x7fu) * (int)(v >> 8);
-        int best = -1, bf = INT_MAX;
-        for (int d0 = 0; d0 < frontier; d0 += 8) {        // best fit: fewest free cores that still fit
-          int f[8];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) f[u] = d0 + u < frontier ? (int)st[(d0 + u) * KPL_THREADS] : 0;
-#pragma unroll
-          for (int u = 0; u < 8; ++u) if (f[u] >= k && f[u] < bf) { bf = f[u]; best = d0 + u; }
+        // best fit: fewest free cores that still fit, lowest domain among equals
+        int bkey = INT_MAX, bslot = -1;
+        for (int x = 0; x < n_open; ++x) {
+          const int f = of[x * 32], key = (f << 8) | od[x * 32];
+          if (f >= k && key < bkey) { bkey = key; bslot = x; }
         }
-        if (best < 0 && frontier < D && G >= k) { best = frontier++; bf = G; }
         int first = -1, dom = -1;
-        if (best >= 0) {
-          first = best * G + (G - bf); dom = best;
-          st[best * KPL_THREADS] = (u8)(bf - k);
+        if (bslot >= 0) {
+          const int f = bkey >> 8;
+          dom = bkey & 0xff; first = dom * G + (G - f);
+          if (f - k > 0) of[bslot * 32] = (u8)(f - k);
+          else { --n_open; od[bslot * 32] = od[n_open * 32]; of[bslot * 32] = of[n_open * 32]; }
+        } else if (frontier < D && G >= k) {              // an untouched domain
+          dom = frontier++; first = dom * G;
+          if (G - k > 0) { od[n_open * 32] = (u8)dom; of[n_open * 32] = (u8)(G - k); ++n_open; }
         } else {                                          // no domain fits: ascending domains
           int need = k;
-          for (int d = 0; d < D && need > 0; ++d) {
-            const int f = d < frontier ? st[d * KPL_THREADS] : G;
-            if (f == 0) continue;
+          while (need > 0) {
+            int lo = INT_MAX, ls = -1;                    // open domain of lowest id
+            for (int x = 0; x < n_open; ++x) { const int d = od[x * 32]; if (d < lo) { lo = d; ls = x; } }
+            int d, f;
+            if (ls >= 0) { d = lo; f = of[ls * 32]; }
+            else if (frontier < D) { d = frontier++; f = G; }
+            else break;                                   // cannot happen: the selection fits
             if (first < 0) { first = d * G + (G - f); dom = d; }
             const int take = min(f, need);
-            st[d * KPL_THREADS] = (u8)(f - take);
             need -= take;
-            if (d >= frontier) frontier = d + 1;
+            if (ls >= 0) {
+              if (f - take > 0) of[ls * 32] = (u8)(f - take);
+              else { --n_open; od[ls * 32] = od[n_open * 32]; of[ls * 32] = of[n_open * 32]; }
+            } else if (f - take > 0) { od[n_open * 32] = (u8)d; of[n_open * 32] = (u8)(f - take); ++n_open; }
           }
         }
-        const size_t o = row + vo[b];
-        P.o_node[o] = dom; P.o_off[o] = first;
+        W.node[c * 33 + lane] = (short)dom; W.off[c * 33 + lane] = first;
       }
+      kpl_store(P, W, row, keep, c0, lane);
     }
     return;
   }
@@ -100,48 +163,64 @@ __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ P
   // lv[l]: nodes that hold a maximal free block of 2^l GPUs.
   const int top = ilog2(pd.group), n_nodes = pd.n_nodes;
   const u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;
-  const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total + pd.node0 : nullptr;
+  const u8* busy_row = (P.gpu_busy && sc < P.S) ? P.gpu_busy + (size_t)sc * P.n_nodes_total + pd.node0 : nullptr;
   u64 lv[4] = {0, 0, 0, 0};
   for (int n = 0; n < n_nodes; ++n) {
     const u32 b = (busy_row ? busy_row[n] : 0u) | pad;
-    st[n * KPL_THREADS] = (u8)b;
+    st[n * 32] = (u8)b;
     const u32 lev = node_levels(b);
 #pragma unroll
     for (int l = 0; l < 4; ++l) lv[l] |= (u64)((lev >> l) & 1u) << n;
   }
   for (int lz = top; lz >= 0; --lz) {
     const int z = 1 << lz;
-    for (int i0 = 0; i0 < keep; i0 += KPL_BATCH) {
-      KPL_LOAD_BATCH(i0);
-#pragma unroll
-      for (int bb = 0; bb < KPL_BATCH; ++bb) {
-        if (i0 + bb >= keep) break;
-        const u32 v = vq[bb];
+    for (int c0 = 0; c0 < maxkeep; c0 += 32) {
+      kpl_load(W, rq, ord, keep, c0, lane);
+      const int nc = min(32, keep - c0);
+      // candidates of the chunk that ask for blocks of this size
+      u32 todo = 0;
+      for (int c = 0; c < nc; ++c) {
+        const u32 v = W.rq[c * 33 + lane];
         const int g = v & 0x7f, gang = (v >> 7) & 1, ri = v >> 8;
-        const int nreq = gang ? (g * ri == z ? 1 : 0) : (g == z ? ri : 0);
-        for (int rep = 0; rep < nreq; ++rep) {
+        if (gang ? g * ri == z : g == z) todo |= 1u << c;
+        W.node[c * 33 + lane] = KPL_NONE;
+      }
+      // one request per thread and turn, so that threads with few requests do not sit through
+      // the others' candidates
+      int reps = 0, cc = 0;
+      bool first = false;
+      for (;;) {
+        if (reps == 0 && todo) {
+          cc = __ffs(todo) - 1; todo &= todo - 1;
+          const u32 v = W.rq[cc * 33 + lane];
+          reps = ((v >> 7) & 1) ? 1 : (int)(v >> 8);
+          first = true;
+        }
+        if (!__any_sync(TG_FULL, reps > 0)) break;
+        if (reps > 0) {
+          --reps;
           int bl = lz;
           u64 mask = 0;
           for (; bl <= top; ++bl) {
             mask = bl == 0 ? lv[0] : (bl == 1 ? lv[1] : (bl == 2 ? lv[2] : lv[3]));
             if (mask) break;
           }
-          if (!mask) continue;                            // cannot happen: the selection fits
-          const int node = __ffsll((long long)mask) - 1;
-          u32 b = st[node * KPL_THREADS];
-          const int start = node_block_start(b, bl);
-          b |= ((1u << z) - 1u) << start;
-          st[node * KPL_THREADS] = (u8)b;
-          const u32 lev = node_levels(b);
-          const u64 bit = 1ull << node;
+          if (mask) {                                     // always: the selection fits
+            const int node = __ffsll((long long)mask) - 1;
+            u32 b = st[node * 32];
+            const int start = node_block_start(b, bl);
+            b |= ((1u << z) - 1u) << start;
+            st[node * 32] = (u8)b;
+            const u32 lev = node_levels(b);
+            const u64 bit = 1ull << node;
 #pragma unroll
-          for (int l = 0; l < 4; ++l) lv[l] = (lv[l] & ~bit) | ((u64)((lev >> l) & 1u) << node);
-          if (rep == 0) {
-            const size_t o = row + vo[bb];
-            P.o_node[o] = node; P.o_off[o] = start;
+            for (int l = 0; l < 4; ++l) lv[l] = (lv[l] & ~bit) | ((u64)((lev >> l) & 1u) << node);
+            if (first) { W.node[cc * 33 + lane] = (short)node; W.off[cc * 33 + lane] = start; }
           }
+          first = false;
         }
       }
+      kpl_store(P, W, row, keep, c0, lane);
     }
   }
 }

@@ -444,10 +444,10 @@ static void fill_pool_order(Params& P) {
       if (P.pool[j].type == rank[r]) P.pool_order[k++] = j;
 }
 
-// pools that k_place can take: its per-thread state is 128 bytes of shared memory
+// pools that k_place can take: its per-thread state is a few hundred bytes of shared memory
 static int lane_place_ok(const PoolDev& d) {
   if (d.type == TG_POOL_API) return 1;
-  if (d.type == TG_POOL_CPU) return d.capacity / d.group <= KPL_STATE && d.group <= 255;
+  if (d.type == TG_POOL_CPU) return d.capacity / d.group <= KPL_DOMAINS && d.group <= 255;
   return d.n_nodes <= 64;
 }
 
@@ -749,7 +749,7 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   if (ev) CK(cudaEventRecord(ev[4], st));
   k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
   if (ev) CK(cudaEventRecord(ev[5], st));
-  k_place<<<(P.S * P.P + KPL_THREADS - 1) / KPL_THREADS, KPL_THREADS, 0, st>>>(P);
+  k_place<<<((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS, KPL_THREADS, 0, st>>>(P);
   if (ev) CK(cudaEventRecord(ev[6], st));
   r->launches += 7 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
