@@ -287,43 +287,73 @@ __global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Pa
   }
 }
 
-// The pools whose first eviction step had to be estimated.
-__global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ Params P, const BatchWs W) {
+// One pool whose first eviction step had to be estimated: compare the two objectives, go on
+// evicting where the first eviction pays, hand the result to the placement.
+__device__ void finish_task(const Params& P, const BatchWs& W, int x, int gw, int lane) {
+  const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
+  const TaskState st = W.ts[task];
+  const PoolMeta mt = P.meta[task];
+  Slab slab = warp_slab(P, gw);
+  CandArrays C;
+  if (!gather_candidates(P, sc, j, mt, slab, lane, C)) {
+    if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE);
+    return;
+  }
+  int keep = mt.m;
+  if (!(st.flags & TS_SOLVED) || (st.flags & TS_FAILED)) keep = -1;
+  else {
+    const size_t pos = (size_t)sc * P.N + mt.base;
+    i64 obj = sat_add(st.opt[0], st.est[0]);
+    for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = W.rs1[pos + i];
+    i64 nobj = sat_add(st.opt[1], st.est[1]);
+    if (nobj < obj) {                                    // the first eviction pays: go on
+      for (int i = lane; i < mt.m - 1; i += 32) C.rkeep[i] = W.rs2[pos + i];
+      __syncwarp();
+      PoolTask T;
+      make_task(P, sc, j, mt, C, lane, T);
+      attach_warp_tree(T);
+      keep = evict_resume(P, T, slab, lane, nobj, mt.m - 1);
+    }
+    __syncwarp();
+  }
+  if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+  place_and_write(P, sc, j, mt, C, keep, slab, lane, true);
+}
+
+// Work list of k_finish: the pools that k_solve left undecided, those that go on evicting first.
+// Each of the latter is a chain of dependent DPs and simulations, so they must start as early
+// as possible.  fl: [0] number of chain tasks, [1] number of other tasks, then the chain tasks
+// from the front and the others from the back of an array of S * P entries.
+__global__ void k_finish_list(const __grid_constant__ Params P, const BatchWs W, int* fl) {
+  const int x = blockIdx.x * blockDim.x + threadIdx.x, lane = threadIdx.x & 31;
+  const int n_tasks = P.S * P.P;
+  int kind = -1;                                          // 0 chain, 1 other
+  if (x < n_tasks) {
+    const int sc = x % P.S, j = P.pool_order[x / P.S];
+    const TaskState* st = W.ts + (size_t)sc * P.P + j;
+    const int flags = st->flags;
+    if (!(flags & TS_DECIDED))
+      kind = ((flags & TS_SOLVED) && !(flags & TS_FAILED) &&
+              sat_add(st->opt[1], st->est[1]) < sat_add(st->opt[0], st->est[0])) ? 0 : 1;
+  }
+  for (int k = 0; k < 2; ++k) {
+    const u32 b = __ballot_sync(TG_FULL, kind == k);
+    if (!b) continue;
+    int at = 0;
+    if (lane == __ffs(b) - 1) at = atomicAdd(&fl[k], __popc(b));
+    at = __shfl_sync(TG_FULL, at, __ffs(b) - 1) + __popc(b & ((1u << lane) - 1u));
+    if (kind == k) fl[2 + (k == 0 ? at : n_tasks - 1 - at)] = x;
+  }
+}
+
+__global__ void __launch_bounds__(K2_THREADS) k_finish(const __grid_constant__ Params P, const BatchWs W, const int* fl) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
-  const int n_tasks = P.S * P.P;
+  const int n_tasks = P.S * P.P, n_chain = fl[0], n_all = fl[0] + fl[1];
   for (;;) {
-    const int x = next_task(P.arena_top + 2, lane);
-    if (x >= n_tasks) break;
-    const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
-    const TaskState st = W.ts[task];
-    if (st.flags & TS_DECIDED) continue;
-    const PoolMeta mt = P.meta[task];
-    Slab slab = warp_slab(P, gw);
-    CandArrays C;
-    if (!gather_candidates(P, sc, j, mt, slab, lane, C)) {
-      if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE);
-      continue;
-    }
-    int keep = mt.m;
-    if (!(st.flags & TS_SOLVED) || (st.flags & TS_FAILED)) keep = -1;
-    else {
-      const size_t pos = (size_t)sc * P.N + mt.base;
-      i64 obj = sat_add(st.opt[0], st.est[0]);
-      for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = W.rs1[pos + i];
-      i64 nobj = sat_add(st.opt[1], st.est[1]);
-      if (nobj < obj) {                                    // the first eviction pays: go on
-        for (int i = lane; i < mt.m - 1; i += 32) C.rkeep[i] = W.rs2[pos + i];
-        __syncwarp();
-        PoolTask T;
-        make_task(P, sc, j, mt, C, lane, T);
-        attach_warp_tree(T);
-        keep = evict_resume(P, T, slab, lane, nobj, mt.m - 1);
-      }
-      __syncwarp();
-    }
-    if (keep < 0) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
-    place_and_write(P, sc, j, mt, C, keep, slab, lane, true);
+    const int y = next_task(P.arena_top + 2, lane);
+    if (y >= n_all) break;
+    finish_task(P, W, fl[2 + (y < n_chain ? y : n_tasks - 1 - (y - n_chain))], gw, lane);
   }
 }
 
@@ -349,7 +379,7 @@ struct tangram_round {
   int64_t launches;
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
-  HeadState* hst; void* d_preq; void* d_keepn;
+  HeadState* hst; void* d_preq; void* d_keepn; int* d_fl;
   BatchWs W; int sim_blocks; SimLists L; int n_sm;
   ReplayWs R;
   // host-buffer mode: copy-in, kernels and copy-out of successive chunks on streams of their own
@@ -517,6 +547,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc((void**)&r->W.rs2, SN * P.P) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->d_preq, SN * P.P * sizeof(unsigned short)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->d_keepn, (size_t)P.S * P.P * sizeof(int)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->d_fl, ((size_t)P.S * P.P + 2) * sizeof(int)) != cudaSuccess;
   const long long n_sims = (long long)P.P * P.S * 2;
   r->sim_blocks = (int)((n_sims + 31) / 32);
   r->n_sm = prop.multiProcessorCount;
@@ -639,7 +670,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
-  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn);
+  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
@@ -747,11 +778,13 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   }
   k_sims_big<<<(int)((n_sims + 31) / 32), 32, 0, st>>>(P, W.ts, W.seed2, g_sim_caps[TG_N_SIM_CLASSES - 1], L.count + 63);
   if (ev) CK(cudaEventRecord(ev[4], st));
-  k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
+  CK(cudaMemsetAsync(r->d_fl, 0, 2 * sizeof(int), st));
+  k_finish_list<<<(P.S * P.P + 255) / 256, 256, 0, st>>>(P, W, r->d_fl);
+  k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W, r->d_fl);
   if (ev) CK(cudaEventRecord(ev[5], st));
   k_place<<<((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS, KPL_THREADS, 0, st>>>(P);
   if (ev) CK(cudaEventRecord(ev[6], st));
-  r->launches += 7 + TG_N_SIM_CLASSES;
+  r->launches += 8 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
   return TANGRAM_OK;
 }
