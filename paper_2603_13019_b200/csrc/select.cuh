@@ -604,6 +604,10 @@ __device__ __noinline__ int evict_batch(const Params& P, const PoolTask& T, Slab
 __device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int lane, i64 obj, int keep,
                             bool have_obj = true, i64 opt_keep = 0) {
   i64 opt, est;
+  if (have_obj && keep < T.m) {                          // an eviction has been accepted already: look further ahead
+    const int kb = evict_batch(P, T, slab, lane, obj, keep);
+    if (kb != -2) return kb;
+  }
   for (int t = T.m - keep + 1; t <= T.m - 1; ++t) {
     const int q = T.m - t;
     if (!solve_prefix(P, T, q, slab, lane, &opt)) return -1;
