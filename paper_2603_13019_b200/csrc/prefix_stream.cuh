@@ -11,9 +11,13 @@
 // read the pool's waiting list.
 //
 // k_stream, one CTA per scenario, streams everything behind the head 4096 actions at a time
-// (16 per thread, 128-bit loads and stores): the "not scheduled" outputs are written, records
-// are validated, and only for the pools that may need an estimate the least-level durations
-// (Eq. 1) of the waiting actions are appended, in queue order, to the pool's list in `tmin`.
+// (16 per thread, 128-bit loads): records are validated, and only for the pools that may need
+// an estimate the least-level durations (Eq. 1) of the waiting actions are appended, in queue
+// order, to the pool's list in `tmin`.
+//
+// k_fill writes "not scheduled" to every output row behind the candidate prefix (128-bit
+// stores).  Nothing else touches those rows, so it runs on a stream of its own beside all
+// kernels that follow k_head.
 //
 // Partitioned arrays (order, tmin and the solver's arrays) give every (scenario, pool) its own
 // row of max_actions entries, so a position never depends on another pool's count and the
@@ -30,7 +34,7 @@ struct HeadState {
   int hs;                     // first action the stream has to look at (a multiple of 32, or n_actions)
   u32 need;                   // pools whose waiting list may be read
   int bad;                    // an invalid record was seen
-  int pad;
+  int n;                      // length of the candidate prefix
   int cur[TG_MAX_POOLS];      // actions of every pool in [0, hs)
 };
 
@@ -66,7 +70,7 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
 
   u32 el = 0, need = 0;
   bool bad = false;
-  int hs = n_act;
+  int hs = n_act, n_pref = n_act;
   const u32 lt = (1u << lane) - 1u;
   for (int c0 = 0; c0 < n_act; c0 += 32) {
     const int i = c0 + lane;
@@ -127,16 +131,13 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
       }
       const int mj = __shfl_sync(TG_FULL, mreg, valid ? j : 0);
       const bool waits = valid && lane >= f;
-      if (waits) {
-        P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1;
-        if ((need >> j) & 1u)
-          P.tmin[prow + (size_t)j * P.N + pos] = duration(clamp_param(s), clamp_param(p), rmin);
-      }
+      if (waits && ((need >> j) & 1u))
+        P.tmin[prow + (size_t)j * P.N + pos] = duration(clamp_param(s), clamp_param(p), rmin);
       for (int jj = 0; jj < P.P; ++jj) {               // the pool's first waiting action
         const u32 b = __ballot_sync(TG_FULL, waits && j == jj && pos == mj);
         if (lane == jj && b) fwreg = c0 + __ffs(b) - 1;
       }
-      hs = min(c0 + 32, n_act);
+      hs = min(c0 + 32, n_act); n_pref = c0 + f;
       break;
     }
   }
@@ -149,7 +150,7 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
     P.meta[(size_t)sc * P.P + lane] = mt;
     hst[sc].cur[lane] = cnt;
   }
-  if (lane == 0) { hst[sc].hs = hs; hst[sc].need = need; hst[sc].bad = anybad; }
+  if (lane == 0) { hst[sc].hs = hs; hst[sc].need = need; hst[sc].bad = anybad; hst[sc].n = n_pref; }
 }
 
 // exclusive scan of one int per thread over the CTA; *total = sum.  wsum: 8 ints of scratch.
@@ -177,9 +178,7 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
   const int n_act = min(max(P.n_actions[sc], 0), P.N);
   const HeadState H = hst[sc];
   const u32 need = H.need;
-  const bool vec = (P.N % 16 == 0) &&
-                   ((((size_t)P.a_pool | (size_t)P.a_unit | (size_t)P.a_mask | (size_t)P.a_s | (size_t)P.a_p |
-                      (size_t)P.o_alloc | (size_t)P.o_node | (size_t)P.o_off | (size_t)P.o_act) & 15) == 0);
+  const bool vec = (P.N % 16 == 0) && ((((size_t)P.a_pool | (size_t)P.a_unit | (size_t)P.a_mask) & 15) == 0);
   if (t < TG_MAX_POOLS) {
     s_m[t] = t < P.P ? P.meta[(size_t)sc * P.P + t].m : 0;
     s_first[t] = INT_MAX;
@@ -208,25 +207,6 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
         rp[k] = i < n_act ? P.a_pool[row + i] : 0xff;
         ru[k] = i < n_act ? P.a_unit[row + i] : 1;
         rm[k] = i < n_act ? P.a_mask[row + i] : 1;
-      }
-    }
-    // "not scheduled" outputs: they depend on nothing and drain while the loads are in flight
-    if (full) {
-      const int4 z = make_int4(0, 0, 0, 0), m1 = make_int4(-1, -1, -1, -1);
-      const longlong2 a1 = make_longlong2(-1, -1);
-#pragma unroll
-      for (int k = 0; k < KS_ITEMS; k += 4) {
-        *(int4*)(P.o_alloc + row + i_first + k) = z;
-        *(int4*)(P.o_node + row + i_first + k) = m1;
-        *(int4*)(P.o_off + row + i_first + k) = m1;
-      }
-#pragma unroll
-      for (int k = 0; k < KS_ITEMS; k += 2) *(longlong2*)(P.o_act + row + i_first + k) = a1;
-    } else {
-#pragma unroll
-      for (int k = 0; k < KS_ITEMS; ++k) {
-        const int i = i_first + k;
-        if (i < n_act) { P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1; }
       }
     }
     // positions in the waiting lists follow from the pool bytes alone, so the CTA-wide scans come
@@ -294,8 +274,8 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
   }
   __syncthreads();
   const bool bad = s_bad != 0;
-  // rows never looked at (beyond the scenario's queue), or everything of a bad scenario
-  for (int i = (bad ? 0 : n_act) + t; i < P.N; i += KS_THREADS) {
+  // nobody will write the candidates of a bad scenario: their rows are "not scheduled" too
+  if (bad) for (int i = t; i < min(H.n, P.N); i += KS_THREADS) {
     P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1;
   }
   if (t < P.P) {
@@ -307,4 +287,37 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
     } else mt->count = mt->m;                          // a list nobody reads counts as empty
   }
   if (t == 0) { P.o_status[sc] = bad ? TG_ST_BAD_ACTION : 0; P.o_total[sc] = 0; P.o_nsel[sc] = 0; }
+}
+
+// "not scheduled" (Eq. 2 has no value for an action that stays queued): units 0, node -1, offset -1,
+// ACT -1 for every action behind its scenario's candidate prefix (the candidates' rows are written
+// by the kernels that decide them, which may run at the same time).  Consecutive threads take
+// consecutive groups of four actions, so a warp's store covers whole contiguous sectors.
+__global__ void __launch_bounds__(256) k_fill(const __grid_constant__ Params P, const HeadState* hst) {
+  const bool vec = (P.N % 4 == 0) &&
+                   ((((size_t)P.o_alloc | (size_t)P.o_node | (size_t)P.o_off | (size_t)P.o_act) & 15) == 0);
+  const u32 stride = gridDim.x * blockDim.x, tid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (vec) {
+    const u32 qpr = (u32)P.N / 4, quads = (u32)P.S * qpr;   // S * N <= 2^31
+    const int4 z = make_int4(0, 0, 0, 0), m1 = make_int4(-1, -1, -1, -1);
+    const longlong2 a1 = make_longlong2(-1, -1);
+    for (u32 q = tid; q < quads; q += stride) {
+      const u32 sc = q / qpr;
+      const int i0 = (int)(q - sc * qpr) * 4, n = hst[sc].n;
+      if (i0 + 4 <= n) continue;
+      const size_t o = (size_t)q * 4;
+      if (i0 >= n) {
+        *(int4*)(P.o_alloc + o) = z; *(int4*)(P.o_node + o) = m1; *(int4*)(P.o_off + o) = m1;
+        *(longlong2*)(P.o_act + o) = a1; *(longlong2*)(P.o_act + o + 2) = a1;
+      } else {
+        for (int k = n - i0; k < 4; ++k) { P.o_alloc[o + k] = 0; P.o_node[o + k] = -1; P.o_off[o + k] = -1; P.o_act[o + k] = -1; }
+      }
+    }
+  } else {
+    const size_t total = (size_t)P.S * P.N;
+    for (size_t o = tid; o < total; o += stride) {
+      if ((int)(o % P.N) < hst[o / P.N].n) continue;
+      P.o_alloc[o] = 0; P.o_node[o] = -1; P.o_off[o] = -1; P.o_act[o] = -1;
+    }
+  }
 }

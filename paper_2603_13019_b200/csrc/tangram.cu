@@ -17,6 +17,7 @@
 #define K2_THREADS 256
 #define TG_PROF_CALLS 256   // calls whose kernels can be timed between two queries
 #define TG_N_SIM_CLASSES 22
+#define TG_FILL_BLOCKS_PER_SM 4   // k_fill is a trickle beside the other kernels, not a flood
 #define TG_IO_CHUNKS 16
 #define TG_PROF_K 6         // timed intervals per call at most
 #define TG_N_KERNELS 8
@@ -225,7 +226,7 @@ struct BatchWs {
   u8* rs2;         // [S][N] ... of the first m-1
 };
 
-__global__ void __launch_bounds__(K2_THREADS) k_solve(const __grid_constant__ Params P, const BatchWs W) {
+__global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__ Params P, const BatchWs W) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
   const int n_tasks = P.S * P.P;
@@ -756,6 +757,15 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   if (ev) CK(cudaEventRecord(ev[0], st));
   k_head<<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[1], st));
+  {                                                        // the output fill runs beside everything that follows
+    cudaStream_t fs = r->sim_stream[TG_N_SIM_CLASSES];
+    CK(cudaEventRecord(r->sim_fork, st));
+    CK(cudaStreamWaitEvent(fs, r->sim_fork, 0));
+    size_t blocks = ((size_t)P.S * ((P.N + 3) / 4) + 255) / 256;
+    if (blocks > (size_t)r->n_sm * TG_FILL_BLOCKS_PER_SM) blocks = (size_t)r->n_sm * TG_FILL_BLOCKS_PER_SM;
+    k_fill<<<(unsigned)blocks, 256, 0, fs>>>(P, r->hst);
+    CK(cudaEventRecord(r->sim_join[TG_N_SIM_CLASSES], fs));
+  }
   k_stream<<<P.S, KS_THREADS, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[2], st));
   k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
@@ -783,8 +793,9 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W, r->d_fl);
   if (ev) CK(cudaEventRecord(ev[5], st));
   k_place<<<((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS, KPL_THREADS, 0, st>>>(P);
+  CK(cudaStreamWaitEvent(st, r->sim_join[TG_N_SIM_CLASSES], 0));   // the fill is part of the round
   if (ev) CK(cudaEventRecord(ev[6], st));
-  r->launches += 8 + TG_N_SIM_CLASSES;
+  r->launches += 9 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
   return TANGRAM_OK;
 }
