@@ -578,7 +578,13 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   }
   bad |= cudaEventCreateWithFlags(&r->sim_fork, cudaEventDisableTiming) != cudaSuccess;
   for (int c = 0; c <= TG_N_SIM_CLASSES; ++c) {
-    bad |= cudaStreamCreateWithFlags(&r->sim_stream[c], cudaStreamNonBlocking) != cudaSuccess;
+    if (c == TG_N_SIM_CLASSES) {
+      // the fill's stream: highest priority, so that its few blocks get in between those of k_stream
+      int lo = 0, hi = 0;
+      bad |= cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess;
+      bad |= cudaStreamCreateWithPriority(&r->sim_stream[c], cudaStreamNonBlocking, hi) != cudaSuccess;
+    } else
+      bad |= cudaStreamCreateWithFlags(&r->sim_stream[c], cudaStreamNonBlocking) != cudaSuccess;
     bad |= cudaEventCreateWithFlags(&r->sim_join[c], cudaEventDisableTiming) != cudaSuccess;
   }
   if (!bad && desc->host_buffers) {
