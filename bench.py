@@ -33,6 +33,11 @@ from workloads import CONFIGS, generate, make_workload  # noqa: E402
 
 ALGO_BYTES_PER_ACTION = 42        # 22 B read (pool, unit, mask, s, p) + 20 B written (alloc, node, off, act)
 METRIC = "actions scheduled/sec (1xB200)"
+# DRAM bytes per pending action (dram__bytes_read.sum + dram__bytes_write.sum of one launch / actions of the
+# launch) from the ncu capture summarised in profiles/batched_pipeline_cfg4_2048scn.md (cfg4 shape, 2048
+# scenarios); traffic grows in proportion to the actions, so a launch's traffic is this times its actions.
+# The k_stream interval of the per-kernel timing holds k_fill as well (it runs beside it).
+NCU_BYTES_PER_ACTION = {"cfg4": {"k_stream": 33.5, "k_head": 1.54, "k_solve": 2.21, "k_finish": 1.86, "k_place": 0.60}}
 
 
 def _peaks():
@@ -147,7 +152,7 @@ def run_reference(args, w, rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps (default: 100 for the single-round configs that take milliseconds, 5 otherwise)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="cfg4", choices=list(CONFIGS))
     ap.add_argument("--scenarios", type=int, default=0, help="override the number of scenarios (smaller runs)")
@@ -155,6 +160,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
+    if args.steps <= 0:
+        args.steps = 100 if args.config in ("cfg0", "cfg1", "cfg4") and args.impl == "ours" else 5
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))
@@ -285,7 +292,9 @@ def main():
                                              "ms_per_step": e2e["ms"] / e2e["steps"]},
             "gpu_launches": launches,
             "roofline": {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": None, "peak_source": which,
+                         "frac": achieved / peak,
+                         "traffic": (NCU_BYTES_PER_ACTION.get(w.name, {}).get(dom[0]) or 0) * S * N or None,
+                         "traffic_source": "ncu on 2048 scenarios of the same shape, scaled by actions", "peak_source": which,
                          "whole_step_achieved": step_gbs, "whole_step_frac": step_gbs / peak,
                          "kernel_ms": {k: (v[0] / max(v[1], 1)) for k, v in ktimes.items() if v[1]}},
             "cpu_baseline": cpu,

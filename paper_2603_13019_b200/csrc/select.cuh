@@ -212,6 +212,123 @@ __device__ int dp_small(const PoolTask& T, int nrows, int ncell, const int ext[4
   return 1;
 }
 
+// The same DP for several prefixes of the candidate list in one pass: the DP of a prefix is the DP
+// of a longer one cut off after the prefix's last row and read inside the prefix's own, smaller
+// box.  E lists, per prefix, the number of rows, the largest cell coordinates (6-bit fields) and
+// where the multiplicities of the rows go.  Returns the set of prefixes solved (a prefix whose
+// end cells tie is left out).
+#define DPS_PREFIXES 4
+struct DpEnds { int nq; int nrows_k[DPS_PREFIXES]; u32 lim[DPS_PREFIXES]; u8* out[DPS_PREFIXES]; };
+__device__ u32 dp_small_multi(const PoolTask& T, int nrows, int ncell, const int ext[4], const int stride[4],
+                        const bool kept[4], u32 scratch, int lane, const DpEnds& E) {
+  // cell coordinates of this lane, one 6-bit field per dimension; bit 5 of a field is a guard
+  // that survives the subtraction of a demand iff the demand does not exceed the coordinate
+  const u32 GUARD = 0x20u | (0x20u << 6) | (0x20u << 12) | (0x20u << 18);
+  u32 pe = GUARD;
+  int e0 = 0;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    const int el = (lane / stride[l]) % ext[l];
+    if (l == 0) e0 = el;
+    pe |= (u32)el << (6 * l);
+  }
+  i64 prev = lane == 0 ? 0 : TG_INF;
+  int endc[DPS_PREFIXES], endrow[DPS_PREFIXES];
+  u32 endlim[DPS_PREFIXES];
+#pragma unroll
+  for (int k = 0; k < DPS_PREFIXES; ++k) {
+    endc[k] = -1;
+    endrow[k] = k < E.nq ? E.nrows_k[k] : -1;            // in registers: the row loop looks at them every row
+    endlim[k] = E.lim[k];
+  }
+  int next_end = INT_MAX;                                // first row count at which a prefix ends
+#pragma unroll
+  for (int k = 0; k < DPS_PREFIXES; ++k) if (endrow[k] >= 1) next_end = min(next_end, endrow[k]);
+  for (int t0 = 0; t0 < nrows; t0 += 32) {
+    u32 pa[DPS_LEVELS], pb[DPS_LEVELS];                  // r | off << 8 ; demand fields
+    i64 du[DPS_LEVELS];
+    int nl = 0;
+    bool too_many = false;
+#pragma unroll
+    for (int k = 0; k < DPS_LEVELS; ++k) { pa[k] = 0; pb[k] = 0; du[k] = 0; }
+    if (t0 + lane < nrows) {
+      const int i = T.rowcand[t0 + lane];
+      const i64 s = T.cs[i], p = T.cp[i];
+      const u32 mk = T.cmask[i];
+      const int g = T.cg[i] & 0x7f, gang = T.cg[i] >> 7, r0 = __ffs(mk);
+      u32 mm = mk;
+      while (mm) {
+        const int r = __ffs(mm); mm &= mm - 1;
+        int d[4];
+        extra_demand(T.type, g, gang, r0, r, d);
+        u32 off = 0, dls = 0; bool inside = true;
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+          if (kept[l]) { const int dl = d[l] >> l; inside &= dl < ext[l]; off += dl * stride[l]; dls |= (u32)(dl & 31) << (6 * l); }
+        if (!inside) continue;
+        if (nl >= DPS_LEVELS) { too_many = true; break; }
+        const i64 dd = duration(s, p, r);
+#pragma unroll
+        for (int k = 0; k < DPS_LEVELS; ++k) if (k == nl) { pa[k] = (u32)r | (off << 8); pb[k] = dls; du[k] = dd; }
+        ++nl;
+      }
+    }
+    if (__any_sync(TG_FULL, too_many)) return 0;
+    const int nb = min(32, nrows - t0);
+    for (int b = 0; b < nb; ++b) {
+      const int nlb = __shfl_sync(TG_FULL, nl, b);
+      i64 best = TG_INF; u32 bestv = 0;
+#pragma unroll
+      for (int k = 0; k < DPS_LEVELS; ++k) {
+        if (k < nlb) {                                   // levels ascend: the first best one stays
+          const u32 va = __shfl_sync(TG_FULL, pa[k], b), vb = __shfl_sync(TG_FULL, pb[k], b);
+          const i64 dd = __shfl_sync(TG_FULL, du[k], b);
+          const i64 pv = __shfl_up_sync(TG_FULL, prev, va >> 8);
+          const bool ok = ((pe - vb) & GUARD) == GUARD && pv != TG_INF;
+          const i64 cand = pv + dd;
+          if (ok && cand < best) { best = cand; bestv = va; }
+        }
+      }
+      prev = lane < ncell ? best : TG_INF;
+      asm volatile("st.shared.u16 [%0], %1;" :: "r"(scratch + (u32)(t0 + b) * 64u + (u32)lane * 2u), "h"((unsigned short)bestv) : "memory");
+      if (t0 + b + 1 == next_end) {
+      next_end = INT_MAX;
+#pragma unroll
+      for (int k = 0; k < DPS_PREFIXES; ++k) {
+        if (endrow[k] > t0 + b + 1) next_end = min(next_end, endrow[k]);
+        if (endrow[k] == t0 + b + 1) {
+          // best end cell of this prefix inside its own box: lowest value, then fewest extra units
+          // (index along dimension 0); several such cells: left to the general loop
+          const bool in = (((endlim[k] | GUARD) - (pe & ~GUARD)) & GUARD) == GUARD;
+          const i64 pv = in ? prev : TG_INF;
+          const i64 bv = warp_min64(pv);
+          const int be = warp_min32((pv == bv && bv != TG_INF) ? e0 : INT_MAX);
+          const u32 win = __ballot_sync(TG_FULL, pv == bv && bv != TG_INF && e0 == be);
+          if (__popc(win) == 1) endc[k] = __ffs(win) - 1;
+        }
+      }
+      }
+    }
+  }
+  __syncwarp();
+  u32 solved = 0;
+#pragma unroll
+  for (int k = 0; k < DPS_PREFIXES; ++k) {
+    if (k >= E.nq || endc[k] < 0) continue;
+    int c = endc[k];
+    u8* out = E.out[k];
+    for (int t = E.nrows_k[k] - 1; t >= 0; --t) {        // walk back, every lane the same path
+      unsigned short v;
+      asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(scratch + (u32)t * 64u + (u32)c * 2u) : "memory");
+      if (lane == (t & 31)) out[T.rowcand[t]] = (u8)(v & 0xff);
+      c -= v >> 8;
+    }
+    solved |= 1u << k;
+  }
+  __syncwarp();
+  return solved;
+}
+
 // Optimal allocation of candidates [0, q) -> T.rsel[0..q), duration sum -> *opt.
 // *all_best tells that every candidate got its best level (then so does every shorter prefix).
 // Returns false if the workspace is too small.
@@ -408,6 +525,150 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
   return true;
 }
 
+// Optimal allocations of the prefixes q0, q0-1, .., q0-nq+1 (nq <= DPS_PREFIXES) in one go: out[k]
+// receives the multiplicities of prefix q0-k, opt[k] its duration sum.  Same results as
+// solve_prefix for each of them.  The sums of a shorter prefix follow from the longer one by taking
+// one candidate out, the certificates are applied per prefix, and the prefixes that need the DP
+// share one pass of dp_small over the rows of the longest.  Returns the set of prefixes done; the
+// others (a box beyond 32 cells, tied end cells, ...) are left to solve_prefix.
+// *all_best: the longest prefix, and hence every one, has all candidates at their best level.
+__device__ __noinline__ u32 solve_multi(const PoolTask& T, int q0, int nq, u8* const out[DPS_PREFIXES],
+                                        i64 opt[DPS_PREFIXES], int lane, bool* all_best) {
+  const bool gpu = T.type == TG_POOL_GPU;
+  *all_best = false;
+  // ---- the longest prefix: demand and duration sums at the least and at the best levels, rows
+  int dmin[4] = {0, 0, 0, 0}, dbest[4] = {0, 0, 0, 0}, maxex[4] = {0, 0, 0, 0};
+  i64 tmin_sum = 0, tbest_sum = 0;
+  int nrows = 0;
+  for (int i0 = 0; i0 < q0; i0 += 32) {
+    const int i = i0 + lane;
+    bool el = false;
+    if (i < q0) {
+      const int g = T.cg[i] & 0x7f, gang = T.cg[i] >> 7;
+      const u32 mk = T.cmask[i];
+      const int r0 = __ffs(mk), rb = best_level(T.cp[i], mk);
+      const int lz0 = gpu ? level_of(g, gang, r0) : 0, lzb = gpu ? level_of(g, gang, rb) : 0;
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        if (l <= lz0) dmin[l] += g * r0;
+        if (l <= lzb) dbest[l] += g * rb;
+      }
+      tmin_sum += duration(T.cs[i], T.cp[i], r0);
+      tbest_sum += duration(T.cs[i], T.cp[i], rb);
+      el = (mk & (mk - 1)) != 0;
+    }
+    const u32 b = __ballot_sync(TG_FULL, el);
+    if (el) T.rowcand[nrows + __popc(b & ((1u << lane) - 1u))] = i;
+    nrows += __popc(b);
+  }
+#pragma unroll
+  for (int l = 0; l < 4; ++l) { dmin[l] = warp_sum32(dmin[l]); dbest[l] = warp_sum32(dbest[l]); }
+  tbest_sum = warp_sum64(tbest_sum);
+  __syncwarp();
+  {
+    bool fits_best = true;
+#pragma unroll
+    for (int l = 0; l < 4; ++l) if (l == 0 || gpu) fits_best &= dbest[l] <= T.cap[l];
+    if (fits_best) {                                     // the common easy case: nothing else is needed
+      for (int i = lane; i < q0; i += 32) out[0][i] = (u8)best_level(T.cp[i], T.cmask[i]);
+      __syncwarp();
+      opt[0] = tbest_sum; *all_best = true;
+      return 1u;
+    }
+  }
+  tmin_sum = warp_sum64(tmin_sum);
+  for (int t = lane; t < nrows; t += 32) {               // largest extra demand of the rows
+    const int i = T.rowcand[t];
+    const u32 mk = T.cmask[i];
+    int d[4];
+    extra_demand(T.type, T.cg[i] & 0x7f, T.cg[i] >> 7, __ffs(mk), 32 - __clz(mk), d);
+#pragma unroll
+    for (int l = 0; l < 4; ++l) maxex[l] += d[l];
+  }
+#pragma unroll
+  for (int l = 0; l < 4; ++l) maxex[l] = warp_sum32(maxex[l]);
+
+  // ---- every prefix: certificates, box
+  bool kept[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) kept[l] = l == 0 || (gpu && T.cap[l] < T.cap[l - 1]);
+  int state[DPS_PREFIXES];                               // 0 needs the DP, 1 all at the best level, 2 all at the least
+  int ext[4] = {1, 1, 1, 1};
+  DpEnds E;
+  E.nq = 0;
+  int slot[DPS_PREFIXES];                                // prefix -> entry of E
+  u32 done = 0;
+#pragma unroll
+  for (int k = 0; k < DPS_PREFIXES; ++k) {
+    state[k] = -1; slot[k] = -1; opt[k] = 0;
+    if (k >= nq) continue;
+    if (k > 0) {                                         // take candidate q0 - k out of the sums
+      const int i = q0 - k;
+      const int g = T.cg[i] & 0x7f, gang = T.cg[i] >> 7;
+      const u32 mk = T.cmask[i];
+      const int r0 = __ffs(mk), rb = best_level(T.cp[i], mk);
+      const int lz0 = gpu ? level_of(g, gang, r0) : 0, lzb = gpu ? level_of(g, gang, rb) : 0;
+      int d[4] = {0, 0, 0, 0};
+      const bool el = (mk & (mk - 1)) != 0;
+      if (el) { extra_demand(T.type, g, gang, r0, 32 - __clz(mk), d); --nrows; }
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        if (l <= lz0) dmin[l] -= g * r0;
+        if (l <= lzb) dbest[l] -= g * rb;
+        maxex[l] -= d[l];
+      }
+      tmin_sum -= duration(T.cs[i], T.cp[i], r0);
+      tbest_sum -= duration(T.cs[i], T.cp[i], rb);
+    }
+    bool fits_best = true;
+#pragma unroll
+    for (int l = 0; l < 4; ++l) if (l == 0 || gpu) fits_best &= dbest[l] <= T.cap[l];
+    if (fits_best) { state[k] = 1; opt[k] = tbest_sum; done |= 1u << k; if (k == 0) *all_best = true; continue; }
+    if (T.cap[0] - dmin[0] <= 0) { state[k] = 2; opt[k] = tmin_sum; done |= 1u << k; continue; }
+    state[k] = 0;
+    u32 lim = 0;
+#pragma unroll
+    for (int l = 0; l < 4; ++l) {
+      const int bound = min(T.cap[l] - dmin[l], maxex[l]);
+      const int ek = kept[l] ? (max(bound, 0) >> l) + 1 : 1;
+      ext[l] = max(ext[l], ek);
+      lim |= (u32)min(ek - 1, 63) << (6 * l);
+    }
+    slot[k] = E.nq;
+#pragma unroll
+    for (int x = 0; x < DPS_PREFIXES; ++x) if (x == E.nq) { E.nrows_k[x] = nrows; E.lim[x] = lim; E.out[x] = out[k]; }
+    ++E.nq;
+  }
+  // ---- multiplicities without the DP: best level where certified, least level elsewhere
+  for (int i = lane; i < q0; i += 32) {
+    const u32 mk = T.cmask[i];
+    const u8 r0 = (u8)__ffs(mk), rb = (u8)best_level(T.cp[i], mk);
+#pragma unroll
+    for (int k = 0; k < DPS_PREFIXES; ++k)
+      if (k < nq && i < q0 - k) out[k][i] = state[k] == 1 ? rb : r0;
+  }
+  __syncwarp();
+  if (E.nq == 0) return done;
+
+  // ---- one DP pass for the prefixes that need it
+  int stride[4];
+  u64 cells = 1;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) { stride[l] = (int)cells; cells *= (u64)ext[l]; }
+  const int nrows_all = E.nrows_k[0];                    // the longest of them comes first
+  if (cells > 32 || !T.sim_base || nrows_all * 4 > T.sim_cap || nrows_all < 1) return done;
+  const u32 solved = dp_small_multi(T, nrows_all, (int)cells, ext, stride, kept, T.sim_base, lane, E);
+#pragma unroll
+  for (int k = 0; k < DPS_PREFIXES; ++k) {
+    if (k >= nq || slot[k] < 0 || !((solved >> slot[k]) & 1u)) continue;
+    i64 sum = 0;
+    for (int i = lane; i < q0 - k; i += 32) sum += duration(T.cs[i], T.cp[i], out[k][i]);
+    opt[k] = warp_sum64(sum);
+    done |= 1u << k;
+  }
+  return done;
+}
+
 // d-th smallest set bit (d = 0 is the lowest) as a multiplicity
 __device__ __forceinline__ int nth_level(u32 mask, int d) {
   for (int k = 0; k < d; ++k) mask &= mask - 1;
@@ -545,18 +806,24 @@ __device__ __noinline__ int evict_batch(const Params& P, const PoolTask& T, Slab
     i64 optk[EVB];
     u32 stopmask = 0;
     int cnt = 0;
+    u8* outs[DPS_PREFIXES];
+#pragma unroll
+    for (int k = 0; k < EVB; ++k) outs[k] = rs + (u64)k * T.m;
+    bool ab;
+    const u32 got = solve_multi(T, keep0 - 1, nb, outs, optk, lane, &ab);   // one DP pass for all steps where that applies
 #pragma unroll 1
     for (int k = 0; k < EVB; ++k) {
-      optk[k] = 0;
       if (k < nb && !stopmask) {
-        PoolTask T2 = T;
-        T2.rsel = rs + (u64)k * T.m;
         const int q = keep0 - 1 - k;
-        if (!solve_prefix(P, T2, q, slab, lane, &optk[k])) {
-          if (k == 0) return -1;
-          break;                                         // a step the loop may never reach: decided when it comes first
+        if (!((got >> k) & 1u)) {
+          PoolTask T2 = T;
+          T2.rsel = outs[k];
+          if (!solve_prefix(P, T2, q, slab, lane, &optk[k])) {
+            if (k == 0) return -1;
+            break;                                       // a step the loop may never reach: decided when it comes first
+          }
         }
-        if (eviction_cannot_pay(T, q, k == 0 ? T.rkeep : rs + (u64)(k - 1) * T.m, T2.rsel, lane)) stopmask |= 1u << k;
+        if (eviction_cannot_pay(T, q, k == 0 ? T.rkeep : outs[k - 1], outs[k], lane)) stopmask |= 1u << k;
         cnt = k + 1;
       }
     }
