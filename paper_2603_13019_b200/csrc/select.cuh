@@ -329,6 +329,158 @@ __device__ u32 dp_small_multi(const PoolTask& T, int nrows, int ncell, const int
   return solved;
 }
 
+// DPArrange on a fragmented GPU pool (Algorithm 4) when no row is a gang request: a row of chunk
+// size 2^c only ever adds requests of that size, so the rows fall into four classes that
+// interact through nothing but the nested capacities (extra GPUs at sizes >= 2^l <= Y[l]).  Per
+// class a one-dimensional DP over "extra chunks of this size" gives f_c(x) = least duration sum of
+// the class with exactly x extra chunks (same recurrence and tie order as the general loop);
+// the classes are then merged from the largest size down,
+//   G_c(e) = min over x of G_{c+1}((e - x) / 2) + f_c(x),   e <= Y[c] >> c  (e in chunks of 2^c),
+// which replaces a table over the product of the four extents by tables over each of them.
+// If two different splits between classes tie on a cell of the chosen path, the canonical order
+// among them is not decided here: the function then returns 0 and the caller runs the general
+// loop (as it does when the scratch does not suffice).  Rows are T.rowcand[0..nrows).
+#define DPC_MAX_CELLS 4096
+__device__ __noinline__ int dp_classes(const PoolTask& T, int nrows, const int Y[4], const int maxex[4], Slab slab, int lane) {
+  // class sizes
+  int rows_c[4] = {0, 0, 0, 0}, mx_c[4] = {0, 0, 0, 0};  // rows and largest extra chunks per class
+  bool gang_row = false;
+  for (int t = lane; t < nrows; t += 32) {
+    const int i = T.rowcand[t];
+    const int g = T.cg[i] & 0x7f;
+    if (T.cg[i] >> 7) gang_row = true;
+    const u32 mk = T.cmask[i];
+    const int c = ilog2(g), ex = (32 - __clz(mk)) - __ffs(mk);
+#pragma unroll
+    for (int l = 0; l < 4; ++l) if (l == c) { rows_c[l] += 1; mx_c[l] += ex; }
+  }
+  if (__any_sync(TG_FULL, gang_row)) return 0;
+  int U[4];                                               // largest useful number of extra chunks per class
+  u64 need = 0;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    rows_c[l] = warp_sum32(rows_c[l]); mx_c[l] = warp_sum32(mx_c[l]);
+    U[l] = min(max(Y[l], 0) >> l, mx_c[l]);
+    if (U[l] + 1 > DPC_MAX_CELLS || (Y[l] >> l) + 1 > 2 * DPC_MAX_CELLS) return 0;
+    need += (u64)rows_c[l] * (U[l] + 1) + 3 * (u64)(U[l] + 1) * 8 + 16 * 4;
+  }
+  (void)maxex;
+  // scratch: per class f (final values), two work rows, choices; merged tables
+  i64* f[4]; u8* ch[4];
+  i64* work = nullptr;
+  int Umax = max(max(U[0], U[1]), max(U[2], U[3]));
+  work = (i64*)slab.take(2 * (u64)(Umax + 1) * 8);
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    f[l] = (i64*)slab.take((u64)(U[l] + 1) * 8);
+    ch[l] = (u8*)slab.take((u64)max(rows_c[l], 1) * (U[l] + 1));
+  }
+  // merged tables: E[l] cells in chunks of 2^l, value, chosen cell of the level above, tie flag
+  int E[4];
+  i64* G[4]; int* gsel[4]; u8* gtie[4];
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    E[l] = max(Y[l], 0) >> l;
+    G[l] = (i64*)slab.take((u64)(E[l] + 1) * 8);
+    gsel[l] = (int*)slab.take((u64)(E[l] + 1) * 4);
+    gtie[l] = (u8*)slab.take((u64)(E[l] + 1));
+  }
+  if (!work || !gtie[3] || !gtie[0] || !ch[3] || !ch[0]) return 0;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) if (!f[l] || !ch[l] || !G[l] || !gsel[l] || !gtie[l]) return 0;
+
+  // ---- per class: one-dimensional DP over its rows, in queue order
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    i64* prev = work; i64* cur = work + (Umax + 1);
+    const int Uc = U[c];
+    for (int u = lane; u <= Uc; u += 32) prev[u] = u == 0 ? 0 : TG_INF;
+    __syncwarp();
+    int tc = 0;
+    for (int t = 0; t < nrows; ++t) {
+      const int i = T.rowcand[t];
+      if (ilog2(T.cg[i] & 0x7f) != c) continue;
+      const u32 mk = T.cmask[i];
+      const int r0 = __ffs(mk);
+      const i64 s = T.cs[i], p = T.cp[i];
+      u8* chr = ch[c] + (u64)tc * (Uc + 1);
+      for (int u = lane; u <= Uc; u += 32) {
+        i64 best = TG_INF; int bestr = 0;
+        u32 mm = mk;
+        while (mm) {
+          const int r = __ffs(mm); mm &= mm - 1;
+          const int du = r - r0;
+          if (du > u) break;                              // levels ascend
+          const i64 pv = prev[u - du];
+          if (pv == TG_INF) continue;
+          const i64 cand = pv + duration(s, p, r);
+          if (cand < best) { best = cand; bestr = r; }
+        }
+        cur[u] = best; chr[u] = (u8)bestr;
+      }
+      __syncwarp();
+      i64* tmp = prev; prev = cur; cur = tmp;
+      ++tc;
+    }
+    for (int u = lane; u <= Uc; u += 32) f[c][u] = prev[u];
+    __syncwarp();
+  }
+  // ---- merge, largest chunks first
+  for (int e = lane; e <= E[3]; e += 32) { G[3][e] = e <= U[3] ? f[3][e] : TG_INF; gsel[3][e] = 0; gtie[3][e] = 0; }
+  __syncwarp();
+#pragma unroll 1
+  for (int c = 2; c >= 0; --c) {
+    const int Ec = E[c], Uc = U[c], Eup = E[c + 1];
+    for (int e = lane; e <= Ec; e += 32) {
+      i64 best = TG_INF; int bu = 0; bool tie = false;
+      for (int up = 0; up <= Eup && 2 * up <= e; ++up) {
+        const int x = e - 2 * up;
+        if (x > Uc) continue;
+        const i64 a = G[c + 1][up], b = f[c][x];
+        if (a == TG_INF || b == TG_INF) continue;
+        const i64 cand = a + b;
+        if (cand < best) { best = cand; bu = up; tie = gtie[c + 1][up] != 0; }
+        else if (cand == best) tie = true;
+      }
+      G[c][e] = best; gsel[c][e] = bu; gtie[c][e] = tie ? 1 : 0;
+    }
+    __syncwarp();
+  }
+  // ---- best end cell: lowest value, then fewest extra GPUs
+  i64 bv = TG_INF;
+  for (int e = lane; e <= E[0]; e += 32) bv = min(bv, G[0][e]);
+  bv = warp_min64(bv);
+  if (bv == TG_INF) return 0;
+  int be = INT_MAX;
+  for (int e = lane; e <= E[0]; e += 32) if (G[0][e] == bv) be = min(be, e);
+  be = warp_min32(be);
+  // ---- walk back: cells of the merged tables, then the rows of every class
+  int cell[4];
+  cell[0] = be;
+  bool tied = gtie[0][be] != 0;
+#pragma unroll
+  for (int c = 0; c < 3; ++c) cell[c + 1] = gsel[c][cell[c]];
+  if (tied) return 0;
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    int u = c < 3 ? cell[c] - 2 * cell[c + 1] : cell[3];
+    const int Uc = U[c];
+    int tc = rows_c[c];
+    if (lane == 0) {
+      for (int t = nrows - 1; t >= 0; --t) {
+        const int i = T.rowcand[t];
+        if (ilog2(T.cg[i] & 0x7f) != c) continue;
+        --tc;
+        const int r = ch[c][(u64)tc * (Uc + 1) + u];
+        T.rsel[i] = (u8)r;
+        u -= r - __ffs(T.cmask[i]);
+      }
+    }
+  }
+  __syncwarp();
+  return 1;
+}
+
 // Optimal allocation of candidates [0, q) -> T.rsel[0..q), duration sum -> *opt.
 // *all_best tells that every candidate got its best level (then so does every shorter prefix).
 // Returns false if the workspace is too small.
@@ -405,11 +557,17 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
     int bound = min(Y[l], maxex[l]);
     ext[l] = kept[l] ? (max(bound, 0) >> l) + 1 : 1;
     stride[l] = (int)cells;
-    cells *= (u64)ext[l];
-    if (cells > (1ull << 30)) return false;
+    if (cells <= (1ull << 30)) cells *= (u64)ext[l];
   }
-  const int ncell = (int)cells;
   __syncwarp();
+  if (gpu && cells > 32 && (kept[1] || kept[2] || kept[3]) && dp_classes(T, nrows, Y, maxex, slab, lane)) {
+    i64 sum = 0;
+    for (int i = lane; i < q; i += 32) sum += duration(T.cs[i], T.cp[i], T.rsel[i]);
+    *opt = warp_sum64(sum);
+    return true;
+  }
+  if (cells > (1ull << 30)) return false;
+  const int ncell = (int)cells;
   if (ncell <= 32 && T.sim_base && nrows * 4 <= T.sim_cap &&
       dp_small(T, nrows, ncell, ext, stride, kept, T.sim_base, lane)) {
     i64 sum = 0;
