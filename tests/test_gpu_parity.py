@@ -105,3 +105,27 @@ def test_long_queue_spans_several_tiles(oracle):
     g = gpu_round(pools, a)
     assert_same(o, g)
     assert o["n_selected"].max() > 300
+
+
+@pytest.mark.parametrize("ties", [0.0, 0.6, 1.0])
+def test_fragmented_gpu_pool_of_replica_requests_matches_oracle(oracle, ties):
+    # replica requests only (no gang rows) on a fragmented pool: the per-size DPs merged through the
+    # nested capacities; with tiny durations different splits tie and the general loop takes over
+    pools = (Pool(POOL_GPU, 192, 8),)
+    w, a = random_round(4242 + int(ties * 10), 48, 220, pools, replicas=1.0, busy_fraction=0.35,
+                        small_durations=ties, inelastic=0.2, max_mult=4)
+    for depth in (1, 2):
+        o = oracle.schedule_batch(pools, a, depth=depth)
+        g = gpu_round(pools, a, depth=depth)
+        assert_same(o, g)
+    assert o["n_selected"].max() > 20
+
+
+def test_pools_beyond_the_thread_per_pool_placement_match_oracle(oracle):
+    # 160 NUMA domains and 72 GPU nodes: these pools are placed by the warp-per-pool routines
+    pools = (Pool(POOL_CPU, 160 * 4, 4), Pool(POOL_GPU, 72 * 8, 8), Pool(POOL_API, 50, 0, 1_000_000))
+    w, a = random_round(77, 24, 700, pools, busy_fraction=0.2, max_mult=6, replicas=1.0)
+    o = oracle.schedule_batch(pools, a)
+    g = gpu_round(pools, a)
+    assert_same(o, g)
+    assert o["n_selected"].max() > 100
