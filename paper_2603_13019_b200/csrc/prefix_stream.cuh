@@ -167,7 +167,7 @@ __device__ __forceinline__ int ks_block_scan(int x, int* wsum, int t, int* total
   return off + incl - x;
 }
 
-__global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant__ Params P, const HeadState* hst) {
+__global__ void __launch_bounds__(KS_THREADS, 4) k_stream(const __grid_constant__ Params P, const HeadState* hst) {
   __shared__ int s_m[TG_MAX_POOLS], s_first[TG_MAX_POOLS], s_cur[TG_MAX_POOLS], s_scan[KS_THREADS / 32];
   __shared__ int s_bad;
   __shared__ u32 s_pinfo[TG_MAX_POOLS];             // type | GPUs per node << 4, 0xf for "no such pool"
@@ -187,79 +187,72 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
   if (t == 0) s_bad = H.bad;
   __syncthreads();
 
-  int cur[TG_MAX_POOLS];                              // actions of every pool seen so far
-#pragma unroll
-  for (int j = 0; j < TG_MAX_POOLS; ++j) cur[j] = H.cur[j];
+  if (t < TG_MAX_POOLS) s_cur[t] = H.cur[t];          // actions of every pool seen so far
+  __syncthreads();
   for (int tile0 = H.hs; tile0 < n_act; tile0 += KS_TILE) {   // a bad scenario is streamed on: its rows are rewritten below
     const int i_first = tile0 + t * KS_ITEMS;
     const bool full = vec && i_first + KS_ITEMS <= n_act;
-    u8 rp[KS_ITEMS], ru[KS_ITEMS];
-    u32 rm[KS_ITEMS];
-    if (full) {
-      *(uint4*)rp = *(const uint4*)(P.a_pool + row + i_first);
-      *(uint4*)ru = *(const uint4*)(P.a_unit + row + i_first);
-#pragma unroll
-      for (int k = 0; k < KS_ITEMS; k += 4) *(uint4*)(rm + k) = *(const uint4*)(P.a_mask + row + i_first + k);
-    } else {
-#pragma unroll
-      for (int k = 0; k < KS_ITEMS; ++k) {
-        const int i = i_first + k;
-        rp[k] = i < n_act ? P.a_pool[row + i] : 0xff;
-        ru[k] = i < n_act ? P.a_unit[row + i] : 1;
-        rm[k] = i < n_act ? P.a_mask[row + i] : 1;
-      }
-    }
-    // positions in the waiting lists follow from the pool bytes alone, so the CTA-wide scans come
-    // before everything else that the thread does with its records
-    u32 mine[TG_MAX_POOLS];
-    int ex[TG_MAX_POOLS];
-#pragma unroll
-    for (int j = 0; j < TG_MAX_POOLS; ++j) {
-      mine[j] = 0; ex[j] = 0;
-      if (!((need >> j) & 1u)) continue;
-#pragma unroll
-      for (int k = 0; k < KS_ITEMS; ++k) if (rp[k] == j) mine[j] |= 1u << k;
-      int tot;
-      ex[j] = cur[j] + ks_block_scan(__popc(mine[j]), s_scan, t, &tot);
-      cur[j] += tot;
-    }
+    __align__(16) u8 rp[KS_ITEMS], ru[KS_ITEMS];
     // validate; keep the least multiplicity of the records whose pool may need its list
     bool bad = false;
     u32 rmin4[KS_ITEMS / 4];                          // one byte per record, 0 = not listed
+    {
+      __align__(16) u32 rm[KS_ITEMS];
+      if (full) {
+        *(uint4*)rp = *(const uint4*)(P.a_pool + row + i_first);
+        *(uint4*)ru = *(const uint4*)(P.a_unit + row + i_first);
 #pragma unroll
-    for (int k = 0; k < KS_ITEMS / 4; ++k) rmin4[k] = 0;
+        for (int k = 0; k < KS_ITEMS; k += 4) *(uint4*)(rm + k) = *(const uint4*)(P.a_mask + row + i_first + k);
+      } else {
 #pragma unroll
-    for (int k = 0; k < KS_ITEMS; ++k) {
-      if (!full && i_first + k >= n_act) continue;
-      const int j = rp[k];
-      const u32 pi = s_pinfo[j & (TG_MAX_POOLS - 1)];
-      PoolDev pd;
-      pd.type = pi & 15; pd.group = (pi >> 4) & 15;
-      int g, gang; u32 eff;
-      const bool ok = j < P.P && decode_levels(pd, ru[k], rm[k], g, gang, eff);
-      bad |= !ok;
-      if (ok && ((need >> j) & 1u)) rmin4[k >> 2] |= (u32)__ffs(eff) << (8 * (k & 3));
+        for (int k = 0; k < KS_ITEMS; ++k) {
+          const int i = i_first + k;
+          rp[k] = i < n_act ? P.a_pool[row + i] : 0xff;
+          ru[k] = i < n_act ? P.a_unit[row + i] : 1;
+          rm[k] = i < n_act ? P.a_mask[row + i] : 1;
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS / 4; ++k) rmin4[k] = 0;
+#pragma unroll
+      for (int k = 0; k < KS_ITEMS; ++k) {
+        if (!full && i_first + k >= n_act) continue;
+        const int j = rp[k];
+        const u32 pi = s_pinfo[j & (TG_MAX_POOLS - 1)];
+        PoolDev pd;
+        pd.type = pi & 15; pd.group = (pi >> 4) & 15;
+        int g, gang; u32 eff;
+        const bool ok = j < P.P && decode_levels(pd, ru[k], rm[k], g, gang, eff);
+        bad |= !ok;
+        if (ok && ((need >> j) & 1u)) rmin4[k >> 2] |= (u32)__ffs(eff) << (8 * (k & 3));
+      }
     }
     if (bad) s_bad = 1;
-    // waiting lists of the pools that may need them
+    // waiting lists of the pools that may need them; a position follows from the pool bytes alone
+    for (u32 nm = need; nm; nm &= nm - 1) {
+      const int j = __ffs(nm) - 1;
+      u32 mine = 0;
 #pragma unroll
-    for (int j = 0; j < TG_MAX_POOLS; ++j) {
-      if (!mine[j]) continue;
-      int pos = ex[j];
+      for (int k = 0; k < KS_ITEMS; ++k) if (rp[k] == j) mine |= 1u << k;
+      const int before = s_cur[j];
+      int tot;
+      int pos = before + ks_block_scan(__popc(mine), s_scan, t, &tot);
+      if (t == 0) s_cur[j] = before + tot;               // read again only after the barrier that ends the tile
+      if (!mine) continue;
       const int m_j = s_m[j];
       i64* dst = P.tmin + prow + (size_t)j * P.N;
 #pragma unroll
-      for (int h = 0; h < KS_ITEMS; h += 8) {            // loads of eight records in flight at once
-        i64 sv[8], pv[8];
+      for (int h = 0; h < KS_ITEMS; h += 4) {            // loads of four records in flight at once
+        i64 sv[4], pv[4];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const bool on = (mine[j] >> (h + k)) & 1u;
+        for (int k = 0; k < 4; ++k) {
+          const bool on = (mine >> (h + k)) & 1u;
           sv[k] = on ? P.a_s[row + i_first + h + k] : 0;
           pv[k] = on ? P.a_p[row + i_first + h + k] : 0;
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          if (!((mine[j] >> (h + k)) & 1u)) continue;
+        for (int k = 0; k < 4; ++k) {
+          if (!((mine >> (h + k)) & 1u)) continue;
           const int rmin = (rmin4[(h + k) >> 2] >> (8 * ((h + k) & 3))) & 0xffu;
           if (rmin) dst[pos] = duration(clamp_param(sv[k]), clamp_param(pv[k]), rmin);   // 0: invalid record, the scenario is flagged
           if (pos == m_j) s_first[j] = i_first + h + k;   // the pool's first waiting action
@@ -267,10 +260,7 @@ __global__ void __launch_bounds__(KS_THREADS, 3) k_stream(const __grid_constant_
         }
       }
     }
-  }
-  if (t == 0) {
-#pragma unroll
-    for (int j = 0; j < TG_MAX_POOLS; ++j) s_cur[j] = cur[j];
+    __syncthreads();
   }
   __syncthreads();
   const bool bad = s_bad != 0;
