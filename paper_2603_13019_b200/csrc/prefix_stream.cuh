@@ -167,7 +167,7 @@ __device__ __forceinline__ int ks_block_scan(int x, int* wsum, int t, int* total
   return off + incl - x;
 }
 
-__global__ void __launch_bounds__(KS_THREADS, 4) k_stream(const __grid_constant__ Params P, const HeadState* hst) {
+__global__ void __launch_bounds__(KS_THREADS, 5) k_stream(const __grid_constant__ Params P, const HeadState* hst) {
   __shared__ int s_m[TG_MAX_POOLS], s_first[TG_MAX_POOLS], s_cur[TG_MAX_POOLS], s_scan[KS_THREADS / 32];
   __shared__ int s_bad;
   __shared__ u32 s_pinfo[TG_MAX_POOLS];             // type | GPUs per node << 4, 0xf for "no such pool"
