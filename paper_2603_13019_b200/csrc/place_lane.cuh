@@ -14,6 +14,7 @@
 #pragma once
 #include "common.cuh"
 #include "place.cuh"
+#include "prefix_stream.cuh"
 
 #define KPL_WARPS 2
 #define KPL_THREADS (32 * KPL_WARPS)
@@ -67,7 +68,7 @@ __device__ __forceinline__ void kpl_store(const Params& P, KplWarp& W, size_t ro
   __syncwarp();
 }
 
-__global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ Params P, const HeadState* hst) {
   __shared__ KplWarp s_w[KPL_WARPS];
   const int lane = threadIdx.x & 31;
   KplWarp& W = s_w[threadIdx.x >> 5];
@@ -76,8 +77,17 @@ __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ P
   if (gw >= wps * P.P) return;
   const int j = P.pool_order[gw / wps], sc = (gw % wps) * 32 + lane;
   const PoolDev& pd = P.pool[j];
+  // A scenario with an invalid record selects nothing.  The record may sit far behind the prefix,
+  // where k_stream finds it while k_solve is already deciding the scenario's pools; so the last
+  // kernel of the round takes back whatever was written for such a scenario.
+  const bool bad = sc < P.S && (P.o_status[sc] & TG_ST_BAD_ACTION);
+  if (bad && gw / wps == 0) {
+    const size_t r0 = (size_t)sc * P.N;
+    for (int i = 0; i < min(hst[sc].n, P.N); ++i) { P.o_alloc[r0 + i] = 0; P.o_node[r0 + i] = -1; P.o_off[r0 + i] = -1; P.o_act[r0 + i] = -1; }
+    P.o_total[sc] = 0; P.o_nsel[sc] = 0; P.o_status[sc] = TG_ST_BAD_ACTION;
+  }
   if (!pd.lane_place) return;
-  int keep = sc < P.S ? P.keepn[(size_t)sc * P.P + j] : 0;
+  int keep = (sc < P.S && !bad) ? P.keepn[(size_t)sc * P.P + j] : 0;
   if (keep < 0) keep = 0;
   const int maxkeep = warp_max32(keep);
   if (maxkeep == 0) return;

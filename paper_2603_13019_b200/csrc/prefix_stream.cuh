@@ -146,11 +146,16 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
   if (lane < P.P) {
     PoolMeta mt;
     mt.base = (i64)sc * (P.P - 1) * P.N + (i64)lane * P.N;   // row + base = prow + lane * N
-    mt.count = cnt; mt.m = mreg; mt.elastic = (elw >> lane) & 1u; mt.first_wait = fwreg;
+    // an invalid record among the actions seen here: nothing of the scenario is decided
+    mt.count = anybad ? 0 : cnt; mt.m = anybad ? 0 : mreg; mt.elastic = anybad ? 0 : ((elw >> lane) & 1u);
+    mt.first_wait = anybad ? -1 : fwreg;
     P.meta[(size_t)sc * P.P + lane] = mt;
     hst[sc].cur[lane] = cnt;
   }
-  if (lane == 0) { hst[sc].hs = hs; hst[sc].need = need; hst[sc].bad = anybad; hst[sc].n = n_pref; }
+  if (lane == 0) {
+    hst[sc].hs = hs; hst[sc].need = need; hst[sc].bad = anybad; hst[sc].n = n_pref;
+    P.o_status[sc] = anybad ? TG_ST_BAD_ACTION : 0; P.o_total[sc] = 0; P.o_nsel[sc] = 0;
+  }
 }
 
 // exclusive scan of one int per thread over the CTA; *total = sum.  wsum: 8 ints of scratch.
@@ -276,7 +281,8 @@ __global__ void __launch_bounds__(KS_THREADS, 5) k_stream(const __grid_constant_
       if (s_first[t] != INT_MAX) mt->first_wait = s_first[t];
     } else mt->count = mt->m;                          // a list nobody reads counts as empty
   }
-  if (t == 0) { P.o_status[sc] = bad ? TG_ST_BAD_ACTION : 0; P.o_total[sc] = 0; P.o_nsel[sc] = 0; }
+  // status, total and count were initialised by k_head; k_solve may be adding to them already
+  if (t == 0 && bad) atomicOr(&P.o_status[sc], TG_ST_BAD_ACTION);
 }
 
 // "not scheduled" (Eq. 2 has no value for an action that stays queued): units 0, node -1, offset -1,

@@ -76,8 +76,10 @@ __device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta
   return true;
 }
 
+// with_waiting = false leaves out what is known about the pool's waiting actions (k_solve runs
+// beside k_stream, which is still counting them).
 __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, const CandArrays& C, int lane,
-                          PoolTask& T) {
+                          PoolTask& T, bool with_waiting = true) {
   const PoolDev& pd = P.pool[j];
   const size_t row = (size_t)sc * P.N;
   const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr;
@@ -85,7 +87,7 @@ __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, co
   T.cap[0] = pd.capacity; T.cap[1] = T.cap[2] = T.cap[3] = 0;
   if (pd.type == TG_POOL_GPU) gpu_caps(pd, busy_row, lane, T.cap);
   T.m = mt.m; T.cs = C.cs; T.cp = C.cp; T.cmask = C.cmask; T.cg = C.cg;
-  T.n_ac = mt.count - mt.m;
+  T.n_ac = with_waiting ? mt.count - mt.m : 0;
   T.ac_tmin = P.tmin + row + mt.base + mt.m;
   T.ac_first.s = T.ac_first.p = 0; T.ac_first.mask = 1; T.ac_first.g = 1; T.ac_first.gang = 0;
   if (T.n_ac > 0) {
@@ -249,7 +251,7 @@ __global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__
     bool decided = true;
     if (mt.elastic) {
       PoolTask T;
-      make_task(P, sc, j, mt, C, lane, T);
+      make_task(P, sc, j, mt, C, lane, T, false);
       attach_warp_tree(T);                               // scratch of the small-box DP
       i64 opt0 = 0, opt1 = 0;
       bool all_best;
@@ -272,7 +274,7 @@ __global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__
             }
             if (lane == 0) {
               st->opt[0] = opt0; st->opt[1] = opt1;
-              st->est[0] = (mt.count - mt.m) > 0 ? TG_INF : 0;
+              st->est[0] = 0;                              // stays if nothing waits behind the candidates
               st->est[1] = TG_INF;
               st->flags = TS_SOLVED;
             }
@@ -772,6 +774,8 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
     k_fill<<<(unsigned)blocks, 256, 0, fs>>>(P, r->hst);
     CK(cudaEventRecord(r->sim_join[TG_N_SIM_CLASSES], fs));
   }
+  // k_solve needs only what k_head left and could run beside k_stream; measured, the two get in each
+  // other's way on the SMs (1.6 ms together against 0.65 + 0.70 one after the other), so they do not
   k_stream<<<P.S, KS_THREADS, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[2], st));
   k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
@@ -798,7 +802,7 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   k_finish_list<<<(P.S * P.P + 255) / 256, 256, 0, st>>>(P, W, r->d_fl);
   k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W, r->d_fl);
   if (ev) CK(cudaEventRecord(ev[5], st));
-  k_place<<<((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS, KPL_THREADS, 0, st>>>(P);
+  k_place<<<((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS, KPL_THREADS, 0, st>>>(P, r->hst);
   CK(cudaStreamWaitEvent(st, r->sim_join[TG_N_SIM_CLASSES], 0));   // the fill is part of the round
   if (ev) CK(cudaEventRecord(ev[6], st));
   r->launches += 9 + TG_N_SIM_CLASSES;

@@ -129,3 +129,16 @@ def test_pools_beyond_the_thread_per_pool_placement_match_oracle(oracle):
     g = gpu_round(pools, a)
     assert_same(o, g)
     assert o["n_selected"].max() > 100
+
+
+def test_invalid_record_far_behind_the_prefix_matches_oracle(oracle):
+    # the record is found by the streaming kernel while the scenario's pools are being decided
+    w = make_workload("cfg1", n_scenarios=12)
+    a = generate(w)
+    a["level_mask"][3, 900] = 0
+    a["pool"][7, 1023] = 9
+    a["unit"][9, 600] = 0
+    o = oracle.schedule_batch(w.pools, a, depth=w.depth)
+    g = gpu_round(w.pools, a, depth=w.depth)
+    assert_same(o, g)
+    assert list(g["status"][[3, 7, 9]]) == [1, 1, 1] and g["n_selected"][3] == 0
