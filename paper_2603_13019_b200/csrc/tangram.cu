@@ -52,17 +52,19 @@ __device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta
   const int m = mt.m;
   const PoolDev& pd = P.pool[j];
   const size_t row = (size_t)sc * P.N;
-  C.cs = (i64*)slab.take((u64)m * 8);
-  C.cp = (i64*)slab.take((u64)m * 8);
-  C.cmask = (u32*)slab.take((u64)m * 4);
+  // what the sequential loops read over and over goes to the warp's shared-memory window while
+  // it lasts (most wanted first), the rest to the warp's slab in global memory
+  C.cg = (u8*)slab.take_fast(m);
+  C.rkeep = (u8*)slab.take_fast(m);
+  C.rsel = (u8*)slab.take_fast(m);
+  C.cmask = (u32*)slab.take_fast((u64)m * 4);
+  C.rowcand = (int*)slab.take_fast((u64)m * 4);
+  C.cp = (i64*)slab.take_fast((u64)m * 8);
+  C.cs = (i64*)slab.take_fast((u64)m * 8);
   C.cidx = (int*)slab.take((u64)m * 4);
   C.pnode = (int*)slab.take((u64)m * 4);
   C.poff = (int*)slab.take((u64)m * 4);
-  C.rowcand = (int*)slab.take((u64)m * 4);
-  C.cg = (u8*)slab.take_fast(m);
-  C.rsel = (u8*)slab.take(m);
-  C.rkeep = (u8*)slab.take_fast(m);
-  if (!C.rkeep) return false;
+  if (!C.cg || !C.rkeep || !C.rsel || !C.cmask || !C.rowcand || !C.cp || !C.cs || !C.poff) return false;
   for (int i = lane; i < m; i += 32) {
     int idx = P.order[row + mt.base + i];
     int g, gang; u32 eff;
