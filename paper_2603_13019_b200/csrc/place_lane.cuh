@@ -112,6 +112,72 @@ __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ P
     return;
   }
 
+  if (pd.type == TG_POOL_CPU && pd.group <= 64) {
+    // Section 5.2 on a pool nobody occupies yet: cores are taken lowest id first, so the free
+    // count per domain is the whole state.  Domains at or beyond `frontier` are untouched; the
+    // touched ones with free cores left are kept in one list per free count, ascending by domain
+    // (head[f], next[d]), and `occ` has bit f-1 set when list f is not empty: the best fit (fewest
+    // free cores that still fit, lowest domain among equals) is the head of the first list at
+    // or above the request.
+    const int G = pd.group, D = pd.capacity / G;
+    u8* head = st;                                        // head[f - 1], f = 1 .. 64
+    u8* next = st + 64 * 32;                              // next[d]
+    u64 occ = 0;
+    int frontier = 0;
+    auto push = [&](int d, int f) {                       // insert domain d into list f, ascending
+      const u64 bit = 1ull << (f - 1);
+      int prev = -1, cur = (occ & bit) ? (int)head[(f - 1) * 32] : 0xff;
+      while (cur != 0xff && cur < d) { prev = cur; cur = next[cur * 32]; }
+      next[d * 32] = (u8)cur;
+      if (prev < 0) head[(f - 1) * 32] = (u8)d; else next[prev * 32] = (u8)d;
+      occ |= bit;
+    };
+    auto pop = [&](int f) {                               // take the lowest domain off list f
+      const int d = head[(f - 1) * 32], nx = next[d * 32];
+      if (nx == 0xff) occ &= ~(1ull << (f - 1)); else head[(f - 1) * 32] = (u8)nx;
+      return d;
+    };
+    for (int c0 = 0; c0 < maxkeep; c0 += 32) {
+      kpl_load(W, rq, ord, keep, c0, lane);
+      const int nc = min(32, keep - c0);
+      for (int c = 0; c < nc; ++c) {
+        const u32 v = W.rq[c * 33 + lane];
+        const int k = (int)(v & 0x7fu) * (int)(v >> 8);
+        int first = -1, dom = -1;
+        const u64 fit = k <= 64 ? occ >> (k - 1) : 0ull;   // lists with at least k free cores
+        if (fit) {
+          const int f = k + __ffsll((long long)fit) - 1;
+          dom = pop(f); first = dom * G + (G - f);
+          if (f - k > 0) push(dom, f - k);
+        } else if (frontier < D && G >= k) {              // an untouched domain
+          dom = frontier++; first = dom * G;
+          if (G - k > 0) push(dom, G - k);
+        } else {                                          // no domain fits: ascending domains
+          int need = k;
+          while (need > 0) {
+            int lo = 0xff, lf = 0;                        // open domain of lowest id: the smallest list head
+            for (u64 o = occ; o; o &= o - 1) {
+              const int f = __ffsll((long long)o);
+              const int d = head[(f - 1) * 32];
+              if (d < lo) { lo = d; lf = f; }
+            }
+            int d, f;
+            if (lo != 0xff) { d = pop(lf); f = lf; }
+            else if (frontier < D) { d = frontier++; f = G; }
+            else break;                                   // cannot happen: the selection fits
+            if (first < 0) { first = d * G + (G - f); dom = d; }
+            const int take = min(f, need);
+            need -= take;
+            if (f - take > 0) push(d, f - take);
+          }
+        }
+        W.node[c * 33 + lane] = (short)dom; W.off[c * 33 + lane] = first;
+      }
+      kpl_store(P, W, row, keep, c0, lane);
+    }
+    return;
+  }
+
   if (pd.type == TG_POOL_CPU) {
     // Section 5.2 on a pool nobody occupies yet: cores are taken lowest id first, so the free
     // count per domain is the whole state.  Domains at or beyond `frontier` are untouched; of the
