@@ -72,11 +72,18 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
   bool bad = false;
   int hs = n_act, n_pref = n_act;
   const u32 lt = (1u << lane) - 1u;
+  // the records of the next chunk are loaded while this one is worked on
+  int nj = 0; u32 nun = 0, nmk = 0; i64 ns = 0, np_ = 0;
+  if (lane < n_act) { nj = P.a_pool[row + lane]; nun = P.a_unit[row + lane]; nmk = P.a_mask[row + lane]; ns = P.a_s[row + lane]; np_ = P.a_p[row + lane]; }
   for (int c0 = 0; c0 < n_act; c0 += 32) {
     const int i = c0 + lane;
     const bool present = i < n_act;
-    int j = 0; u32 un = 0, mk = 0; i64 s = 0, p = 0;
-    if (present) { j = P.a_pool[row + i]; un = P.a_unit[row + i]; mk = P.a_mask[row + i]; s = P.a_s[row + i]; p = P.a_p[row + i]; }
+    const int j = nj; const u32 un = nun, mk = nmk; const i64 s = ns, p = np_;
+    {
+      const int i2 = i + 32;
+      nj = 0; nun = 0; nmk = 0; ns = 0; np_ = 0;
+      if (i2 < n_act) { nj = P.a_pool[row + i2]; nun = P.a_unit[row + i2]; nmk = P.a_mask[row + i2]; ns = P.a_s[row + i2]; np_ = P.a_p[row + i2]; }
+    }
     bool valid = present && j < P.P;
     const u32 pi = __shfl_sync(TG_FULL, pinfo, valid ? j : 0);
     PoolDev pd;
@@ -90,15 +97,24 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
     const int units = g * rmin, mxu = g * rmax;
     const int lz = gpu ? level_of(g, gang, rmin) : 0, lzx = gpu ? level_of(g, gang, rmax) : 0;
     // least-level demand: one scan per slot; the first action that overflows a slot ends the prefix
-    bool over = false;
+    // First the chunk's total per slot (one warp reduction each): only the chunk in which a slot
+    // overflows needs the scans that tell which action does it.
+    int tot_mine = 0;                                  // lane v: the chunk's demand on slot v
     for (int v = 0; v < D; ++v) {
       const int c = (valid && v >= slot0 && v <= slot0 + lz) ? units : 0;
-      const int incl = warp_incl_scan32(c, lane);
-      const int rv = __shfl_sync(TG_FULL, run, v), cv = __shfl_sync(TG_FULL, capreg, v);
-      over |= c > 0 && rv + incl > cv;
-      const int tot = __shfl_sync(TG_FULL, incl, 31);
-      if (lane == v) run += tot;
+      const int tot = __reduce_add_sync(TG_FULL, c);
+      if (lane == v) tot_mine = tot;
     }
+    bool over = false;
+    if (__any_sync(TG_FULL, lane < D && run + tot_mine > capreg)) {
+      for (int v = 0; v < D; ++v) {
+        const int c = (valid && v >= slot0 && v <= slot0 + lz) ? units : 0;
+        const int incl = warp_incl_scan32(c, lane);
+        const int rv = __shfl_sync(TG_FULL, run, v), cv = __shfl_sync(TG_FULL, capreg, v);
+        over |= c > 0 && rv + incl > cv;
+      }
+    }
+    run += tot_mine;                                   // beyond the prefix the totals are not used any more
     const u32 ob = __ballot_sync(TG_FULL, over);
     const int f = ob ? __ffs(ob) - 1 : 32;           // lanes >= f wait
     const bool cand = valid && lane < f;
