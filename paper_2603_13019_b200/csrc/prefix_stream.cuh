@@ -119,13 +119,12 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
     const int f = ob ? __ffs(ob) - 1 : 32;           // lanes >= f wait
     const bool cand = valid && lane < f;
     // position inside the pool
-    int pos = 0;
+    int pos = __shfl_sync(TG_FULL, cnt, valid ? j : 0);  // the pool's count before this chunk
+    const u32 below_f = f >= 32 ? TG_FULL : ((1u << f) - 1u);
     for (int jj = 0; jj < P.P; ++jj) {
       const u32 b = __ballot_sync(TG_FULL, valid && j == jj);
-      const u32 bc = __ballot_sync(TG_FULL, cand && j == jj);
-      const int cj = __shfl_sync(TG_FULL, cnt, jj);
-      if (valid && j == jj) pos = cj + __popc(b & lt);
-      if (lane == jj) { cnt += __popc(b); mreg += __popc(bc); }
+      if (valid && j == jj) pos += __popc(b & lt);
+      if (lane == jj) { cnt += __popc(b); mreg += __popc(b & below_f); }
     }
     if (cand) {
       P.order[prow + (size_t)j * P.N + pos] = i;
