@@ -109,12 +109,13 @@ struct SimLists {
   int cap[32];     // capacity (slots) of every class, ascending; a group goes to the first that fits
 };
 
+// one warp per group, one lane per simulation
 __global__ void k_sim_classify(const __grid_constant__ Params P, const TaskState* ts, const SimLists L) {
-  const int g = blockIdx.x * blockDim.x + threadIdx.x;
+  const long long sim = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int g = (int)(sim / SIM_PER_WARP);
   if (g >= L.n_groups) return;
-  int hmax = 0;
-  for (int s = 0; s < SIM_PER_WARP; ++s) hmax = max(hmax, sim_slots(P, ts, (long long)g * SIM_PER_WARP + s));
-  if (hmax == 0) return;
+  const int hmax = warp_max32(sim_slots(P, ts, sim));
+  if (hmax == 0 || (threadIdx.x & 31) != 0) return;
   int c = 0;
   while (c < L.n_classes && hmax > L.cap[c]) ++c;
   if (c == L.n_classes) { L.count[63] = 1; return; }  // beyond shared memory: k_sims_big takes it

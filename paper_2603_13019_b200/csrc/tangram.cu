@@ -783,7 +783,7 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
   if (ev) CK(cudaEventRecord(ev[3], st));
   CK(cudaMemsetAsync(L.count, 0, 2 * 64 * sizeof(int), st));
-  k_sim_classify<<<(L.n_groups + 255) / 256, 256, 0, st>>>(P, W.ts, L);
+  k_sim_classify<<<(L.n_groups + 7) / 8, 256, 0, st>>>(P, W.ts, L);
   CK(cudaEventRecord(r->sim_fork, st));
   for (int c = 0; c < TG_N_SIM_CLASSES; ++c) {
     cudaStream_t ss = r->sim_stream[c];
