@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(32) k_sims1(const __grid_constant__ Params P, 
                                               const SimLists L, int cls) {
   extern __shared__ __align__(16) unsigned char sim_smem[];
   const int lane = threadIdx.x;
-  const u32 base = (((u32)__cvta_generic_to_shared(sim_smem) + 511u) & ~511u) + (u32)lane * 8u;
+  const u32 base = (u32)__cvta_generic_to_shared(sim_smem) + (u32)lane * 8u;   // 16-byte aligned, no padding: it would cost a resident block
   const int count = L.count[cls];
   for (;;) {
     int gi = 0;

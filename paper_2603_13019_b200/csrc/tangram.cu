@@ -426,7 +426,7 @@ static sims_fn sim_kernel(int cap) {
   }
 }
 // shared memory of a block (32 trees interleaved by lane) of a capacity class
-static int sim_smem_bytes(int cap) { return tree_nodes(cap) * 8 * SIM_PER_WARP + 512; }
+static int sim_smem_bytes(int cap) { return tree_nodes(cap) * 8 * SIM_PER_WARP; }
 
 static cudaError_t fill_tables() {
   u64 recip[33];
