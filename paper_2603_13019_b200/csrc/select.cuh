@@ -145,6 +145,7 @@ __device__ int dp_small(const PoolTask& T, int nrows, int ncell, const int ext[4
     pe |= (u32)el << (6 * l);
   }
   i64 prev = lane == 0 ? 0 : TG_INF;
+  const bool via_smem = nrows <= 64;
   for (int t0 = 0; t0 < nrows; t0 += 32) {
     u32 pa[DPS_LEVELS], pb[DPS_LEVELS];                  // r | off << 8 ; demand fields
     i64 du[DPS_LEVELS];
@@ -176,6 +177,35 @@ __device__ int dp_small(const PoolTask& T, int nrows, int ncell, const int ext[4
     }
     if (__any_sync(TG_FULL, too_many)) return 0;
     const int nb = min(32, nrows - t0);
+    if (via_smem) {
+      // up to 64 rows leave room behind the choices for the level lists of a block of rows: a row's
+      // levels are then one broadcast load each instead of four shuffles
+      const u32 lists = scratch + 4096u;
+      __syncwarp();
+#pragma unroll
+      for (int k = 0; k < DPS_LEVELS; ++k)
+        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" :: "r"(lists + (u32)(lane * DPS_LEVELS + k) * 16u),
+                     "r"(pa[k]), "r"(pb[k]), "r"((u32)du[k]), "r"((u32)((u64)du[k] >> 32)) : "memory");
+      __syncwarp();
+      for (int b = 0; b < nb; ++b) {
+        i64 best = TG_INF; u32 bestv = 0;
+#pragma unroll
+        for (int k = 0; k < DPS_LEVELS; ++k) {
+          u32 va, vb, dlo, dhi;
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(va), "=r"(vb), "=r"(dlo), "=r"(dhi)
+                       : "r"(lists + (u32)(b * DPS_LEVELS + k) * 16u) : "memory");
+          if (va == 0) break;                            // the row has no further level (a multiplicity is never 0)
+          const i64 dd = (i64)(((u64)dhi << 32) | dlo);
+          const i64 pv = __shfl_up_sync(TG_FULL, prev, va >> 8);
+          const bool ok = ((pe - vb) & GUARD) == GUARD && pv != TG_INF;
+          const i64 cand = pv + dd;
+          if (ok && cand < best) { best = cand; bestv = va; }
+        }
+        prev = lane < ncell ? best : TG_INF;
+        asm volatile("st.shared.u16 [%0], %1;" :: "r"(scratch + (u32)(t0 + b) * 64u + (u32)lane * 2u), "h"((unsigned short)bestv) : "memory");
+      }
+      continue;
+    }
     for (int b = 0; b < nb; ++b) {
       const int nlb = __shfl_sync(TG_FULL, nl, b);
       i64 best = TG_INF; u32 bestv = 0;
