@@ -107,31 +107,25 @@ __device__ __forceinline__ i64 duration(i64 s, i64 p, int r) { return s + div_sm
 // Chunk-size level that a grant of multiplicity r asks for
 __device__ __forceinline__ int level_of(int g, int gang, int r) { return ilog2(gang ? g * r : g); }
 
-__device__ __forceinline__ i64 warp_min64(i64 v) {
-#pragma unroll
-  for (int o = 16; o; o >>= 1) { i64 t = __shfl_xor_sync(TG_FULL, v, o); v = t < v ? t : v; }
-  return v;
+// Warp reductions.  The SM moves one shuffle per cycle or two for all its warps, so the 32-bit
+// ones use the reduction unit (one instruction), and the 64-bit ones are put together from
+// 32-bit reductions.
+__device__ __forceinline__ i64 warp_min64(i64 v) {      // any signed values
+  const u64 u = (u64)v ^ 0x8000000000000000ull;          // order-preserving map to unsigned
+  const u32 hi = (u32)(u >> 32);
+  const u32 mhi = __reduce_min_sync(TG_FULL, hi);
+  const u32 mlo = __reduce_min_sync(TG_FULL, hi == mhi ? (u32)u : 0xffffffffu);
+  return (i64)((((u64)mhi << 32) | mlo) ^ 0x8000000000000000ull);
 }
-__device__ __forceinline__ i64 warp_sum64(i64 v) {
-#pragma unroll
-  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(TG_FULL, v, o);
-  return v;
+__device__ __forceinline__ i64 warp_sum64(i64 v) {      // 0 <= v, sum below 2^63
+  const u32 a = __reduce_add_sync(TG_FULL, (u32)v & 0x3fffffu);
+  const u32 b = __reduce_add_sync(TG_FULL, (u32)(v >> 22) & 0x3fffffu);
+  const u32 c = __reduce_add_sync(TG_FULL, (u32)((u64)v >> 44));
+  return (i64)((u64)a + ((u64)b << 22) + ((u64)c << 44));
 }
-__device__ __forceinline__ int warp_sum32(int v) {
-#pragma unroll
-  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(TG_FULL, v, o);
-  return v;
-}
-__device__ __forceinline__ int warp_min32(int v) {
-#pragma unroll
-  for (int o = 16; o; o >>= 1) v = min(v, __shfl_xor_sync(TG_FULL, v, o));
-  return v;
-}
-__device__ __forceinline__ int warp_max32(int v) {
-#pragma unroll
-  for (int o = 16; o; o >>= 1) v = max(v, __shfl_xor_sync(TG_FULL, v, o));
-  return v;
-}
+__device__ __forceinline__ int warp_sum32(int v) { return (int)__reduce_add_sync(TG_FULL, (u32)v); }
+__device__ __forceinline__ int warp_min32(int v) { return __reduce_min_sync(TG_FULL, v); }
+__device__ __forceinline__ int warp_max32(int v) { return __reduce_max_sync(TG_FULL, v); }
 
 // Free capacity per chunk level of a GPU pool: cap[l] = GPUs held in maximal free aligned
 // blocks of size >= 2^l.  `busy` may be null (all free).  Warp-cooperative.
