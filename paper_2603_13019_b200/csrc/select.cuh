@@ -590,7 +590,8 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
     if (cells <= (1ull << 30)) cells *= (u64)ext[l];
   }
   __syncwarp();
-  if (gpu && cells > 32 && (kept[1] || kept[2] || kept[3]) && dp_classes(T, nrows, Y, maxex, slab, lane)) {
+  // (the out-of-line routines get a copy of the task, so that this one can stay in registers)
+  if (gpu && cells > 32 && (kept[1] || kept[2] || kept[3]) && dp_classes(PoolTask(T), nrows, Y, maxex, slab, lane)) {
     i64 sum = 0;
     for (int i = lane; i < q; i += 32) sum += duration(T.cs[i], T.cp[i], T.rsel[i]);
     *opt = warp_sum64(sum);
@@ -1060,7 +1061,7 @@ __device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int l
                             bool have_obj = true, i64 opt_keep = 0) {
   i64 opt, est;
   if (have_obj && keep < T.m) {                          // an eviction has been accepted already: look further ahead
-    const int kb = evict_batch(P, T, slab, lane, obj, keep);
+    const int kb = evict_batch(P, PoolTask(T), slab, lane, obj, keep);
     if (kb != -2) return kb;
   }
   for (int t = T.m - keep + 1; t <= T.m - 1; ++t) {
@@ -1077,7 +1078,7 @@ __device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int l
     obj = nobj; keep = q;
     for (int i = lane; i < q; i += 32) T.rkeep[i] = T.rsel[i];
     __syncwarp();
-    const int kb = evict_batch(P, T, slab, lane, obj, keep);   // an eviction was accepted: look further ahead
+    const int kb = evict_batch(P, PoolTask(T), slab, lane, obj, keep);   // an eviction was accepted: look further ahead
     if (kb != -2) return kb;
   }
   return keep;
