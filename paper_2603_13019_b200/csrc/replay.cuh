@@ -213,7 +213,7 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
   return true;
 }
 
-__global__ void __launch_bounds__(K2_THREADS) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
+__global__ void __launch_bounds__(K2_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
   const int nw_warps = (gridDim.x * K2_THREADS) >> 5;
