@@ -291,7 +291,7 @@ def main():
                                              "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                                              "ms_per_step": e2e["ms"] / e2e["steps"]},
             "gpu_launches": launches,
-            "roofline": {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "roofline": {"bound": "hbm", "kernel": dom[0] + (" (+ k_fill, which runs beside it)" if dom[0] == "k_stream" else ""), "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak,
                          "traffic": (NCU_BYTES_PER_ACTION.get(w.name, {}).get(dom[0]) or 0) * S * N or None,
                          "traffic_source": "ncu on 2048 scenarios of the same shape, scaled by actions", "peak_source": which,
