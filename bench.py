@@ -34,7 +34,7 @@ from workloads import CONFIGS, generate, make_workload  # noqa: E402
 ALGO_BYTES_PER_ACTION = 42        # 22 B read (pool, unit, mask, s, p) + 20 B written (alloc, node, off, act)
 METRIC = "actions scheduled/sec (1xB200)"
 # DRAM bytes per pending action (dram__bytes_read.sum + dram__bytes_write.sum of one launch / actions of the
-# launch) from the ncu capture summarised in profiles/batched_pipeline_cfg4_2048scn.md (cfg4 shape, 2048
+# launch) from the ncu capture summarised under profiles/ (cfg4 shape, 2048
 # scenarios); traffic grows in proportion to the actions, so a launch's traffic is this times its actions.
 # The k_stream interval of the per-kernel timing holds k_fill as well (it runs beside it).
 NCU_BYTES_PER_ACTION = {"cfg4": {"k_stream": 36.7, "k_head": 1.72, "k_solve": 2.06, "k_finish": 1.87, "k_place": 0.60}}
