@@ -261,21 +261,23 @@ __global__ void __launch_bounds__(KS_THREADS, 5) k_stream(const __grid_constant_
       if (!mine) continue;
       const int m_j = s_m[j];
       i64* dst = P.tmin + prow + (size_t)j * P.N;
+      // the thread's listed records, four at a time: their s / p loads are in flight together
+      const u64 rlo = (u64)rmin4[0] | ((u64)rmin4[1] << 32), rhi = (u64)rmin4[2] | ((u64)rmin4[3] << 32);
+      for (u32 rest = mine; rest;) {
+        i64 sv[4], pv[4]; int kk[4];
 #pragma unroll
-      for (int h = 0; h < KS_ITEMS; h += 4) {            // loads of four records in flight at once
-        i64 sv[4], pv[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const bool on = (mine >> (h + k)) & 1u;
-          sv[k] = on ? P.a_s[row + i_first + h + k] : 0;
-          pv[k] = on ? P.a_p[row + i_first + h + k] : 0;
+        for (int x = 0; x < 4; ++x) {
+          kk[x] = rest ? __ffs(rest) - 1 : -1;
+          rest &= rest - 1;
+          sv[x] = kk[x] >= 0 ? P.a_s[row + i_first + kk[x]] : 0;
+          pv[x] = kk[x] >= 0 ? P.a_p[row + i_first + kk[x]] : 0;
         }
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (!((mine >> (h + k)) & 1u)) continue;
-          const int rmin = (rmin4[(h + k) >> 2] >> (8 * ((h + k) & 3))) & 0xffu;
-          if (rmin) dst[pos] = duration(clamp_param(sv[k]), clamp_param(pv[k]), rmin);   // 0: invalid record, the scenario is flagged
-          if (pos == m_j) s_first[j] = i_first + h + k;   // the pool's first waiting action
+        for (int x = 0; x < 4; ++x) {
+          if (kk[x] < 0) continue;
+          const int rmin = (int)(((kk[x] < 8 ? rlo : rhi) >> (8 * (kk[x] & 7))) & 0xffu);
+          if (rmin) dst[pos] = duration(clamp_param(sv[x]), clamp_param(pv[x]), rmin);   // 0: invalid record, the scenario is flagged
+          if (pos == m_j) s_first[j] = i_first + kk[x];   // the pool's first waiting action
           ++pos;
         }
       }
