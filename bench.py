@@ -37,7 +37,7 @@ METRIC = "actions scheduled/sec (1xB200)"
 # launch) from the ncu capture summarised under profiles/ (cfg4 shape, 2048
 # scenarios); traffic grows in proportion to the actions, so a launch's traffic is this times its actions.
 # The k_stream interval of the per-kernel timing holds k_fill as well (it runs beside it).
-NCU_BYTES_PER_ACTION = {"cfg4": {"k_stream": 36.7, "k_head": 1.72, "k_solve": 2.06, "k_finish": 1.87, "k_place": 0.60}}
+NCU_BYTES_PER_ACTION = {"cfg4": {"k_stream": 35.0, "k_head": 1.72, "k_solve": 2.07, "k_finish": 1.89, "k_place": 0.59}}
 
 
 def _peaks():
