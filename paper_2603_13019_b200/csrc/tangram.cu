@@ -65,14 +65,29 @@ __device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta
   C.pnode = (int*)slab.take((u64)m * 4);
   C.poff = (int*)slab.take((u64)m * 4);
   if (!C.cg || !C.rkeep || !C.rsel || !C.cmask || !C.rowcand || !C.cp || !C.cs || !C.poff) return false;
-  for (int i = lane; i < m; i += 32) {
-    int idx = P.order[row + mt.base + i];
-    int g, gang; u32 eff;
-    decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], g, gang, eff);
-    C.cidx[i] = idx; C.cmask[i] = eff; C.cg[i] = (u8)(g | (gang << 7));
-    C.cs[i] = clamp_param(P.a_s[row + idx]); C.cp[i] = clamp_param(P.a_p[row + idx]);
-    C.rkeep[i] = (u8)__ffs(eff);
-    C.pnode[i] = -1; C.poff[i] = -1;
+  // four candidates per lane at a time: first all their indices, then all their records, so that a
+  // pool of up to 128 candidates costs two rounds of loads instead of two per 32 candidates
+  for (int i0 = lane; i0 < m; i0 += 128) {
+    int idx[4]; u8 un[4]; u32 mk[4]; i64 sv[4], pv[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) idx[x] = i0 + 32 * x < m ? P.order[row + mt.base + i0 + 32 * x] : 0;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const bool on = i0 + 32 * x < m;
+      un[x] = on ? P.a_unit[row + idx[x]] : 1; mk[x] = on ? P.a_mask[row + idx[x]] : 1;
+      sv[x] = on ? P.a_s[row + idx[x]] : 0; pv[x] = on ? P.a_p[row + idx[x]] : 0;
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const int i = i0 + 32 * x;
+      if (i >= m) break;
+      int g, gang; u32 eff;
+      decode_levels(pd, un[x], mk[x], g, gang, eff);
+      C.cidx[i] = idx[x]; C.cmask[i] = eff; C.cg[i] = (u8)(g | (gang << 7));
+      C.cs[i] = clamp_param(sv[x]); C.cp[i] = clamp_param(pv[x]);
+      C.rkeep[i] = (u8)__ffs(eff);
+      C.pnode[i] = -1; C.poff[i] = -1;
+    }
   }
   __syncwarp();
   return true;
