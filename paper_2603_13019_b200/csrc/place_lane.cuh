@@ -30,13 +30,13 @@ struct KplWarp {
   short node[32 * 33];
 };
 
-// stage requests and indices [c0, c0 + 32) of all 32 scenarios of the warp (eight scenarios'
+// stage requests and indices [c0, c0 + 32) of all 32 scenarios of the warp (sixteen scenarios'
 // loads in flight at once)
 __device__ __forceinline__ void kpl_load(KplWarp& W, const unsigned short* rq, const int* ord, int keep, int c0, int lane) {
-  for (int s0 = 0; s0 < 32; s0 += 8) {
-    unsigned short vq[8]; int vo[8]; bool on[8];
+  for (int s0 = 0; s0 < 32; s0 += 16) {
+    unsigned short vq[16]; int vo[16]; bool on[16];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
+    for (int u = 0; u < 16; ++u) {
       const int ks = __shfl_sync(TG_FULL, keep, s0 + u);
       const unsigned short* rs = (const unsigned short*)__shfl_sync(TG_FULL, (unsigned long long)rq, s0 + u);
       const int* os = (const int*)__shfl_sync(TG_FULL, (unsigned long long)ord, s0 + u);
@@ -45,7 +45,7 @@ __device__ __forceinline__ void kpl_load(KplWarp& W, const unsigned short* rq, c
       vo[u] = on[u] ? os[c0 + lane] : 0;
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u)
+    for (int u = 0; u < 16; ++u)
       if (on[u]) { W.rq[lane * 33 + s0 + u] = vq[u]; W.idx[lane * 33 + s0 + u] = vo[u]; }
   }
   __syncwarp();
