@@ -454,3 +454,118 @@ def test_invalid_records_are_flagged(oracle):
     assert o["status"][0] == 1
     o = _round(oracle, [(GPU, 8, 8, 0)], [(0, 1 | GANG, 0x4, 1, 1)])           # gang level 3 only
     assert o["status"][0] == 1
+
+
+# ------------------------------------------------------------------ Algorithm 1, eviction loop worked by hand
+def test_two_evictions_pay_and_the_third_does_not(oracle):
+    # One core pool of 10, four candidates (s, p, levels), nothing else waits, depth 2:
+    #   a1 (0, 3600, {1,4,6})   a2 (0, 2400, {1,4,6})   a3 (0, 1200, {3})   a4 (0, 3600, {3,4,6})
+    # keep 4: least demand 8, two spare cores; the only level they reach is a4 at 4 (1200 -> 900):
+    #         3600 + 2400 + 400 + 900 = 7300, nothing remains                        objective 7300
+    # keep 3: a3 takes 3, seven cores for a1, a2: (6,1) = 600 + 2400 beats (4,1) = 3300 and (1,6) = 4000;
+    #         completions {600, 2400, 400}; a4 waits: earliest slot 400, second level (4): 400 + 900
+    #         3400 + 1300                                                            objective 4700
+    # keep 2: (6,4) = 600 + 600; completions {600, 600}; a3 (one level, so only depth 1): 600 + 400 = 1000,
+    #         a4 at its least level: 600 + 1200 = 1800;  1200 + 2800                 objective 4000
+    # keep 1: a1 at 6 = 600; completions {600}; a2 at its second level (4): 600 + 600 = 1200, a3: 1600,
+    #         a4: 2800 (depth 1 would give 3000 + 3400 + 4600);  600 + 5600          objective 6200
+    # 7300 > 4700 > 4000 < 6200: two evictions are accepted, the third is not.  Comparing with the
+    # initial 7300 would accept the third (6200 < 7300) and keep a1 alone; stopping after the first
+    # accepted step would keep three.
+    rows = [(0, 1, 0x29, 0, 3600), (0, 1, 0x29, 0, 2400), (0, 1, 0x04, 0, 1200), (0, 1, 0x2C, 0, 3600)]
+    o = _round(oracle, [(CPU, 10, 10, 0)], rows, depth=2)
+    assert list(o["alloc_units"][0]) == [6, 4, 0, 0]
+    assert list(o["act_us"][0]) == [600, 600, -1, -1]
+    assert o["n_selected"][0] == 2 and o["total_act_us"][0] == 1200
+    # at depth 1 the step to three costs 3400 + (400 + 1200) = 5000 < 7300, the step to two stays 4000,
+    # the step to one 600 + 11000: the same two evictions
+    o = _round(oracle, [(CPU, 10, 10, 0)], rows, depth=1)
+    assert list(o["alloc_units"][0]) == [6, 4, 0, 0]
+
+
+def test_evicted_candidates_come_before_the_waiting_actions(oracle):
+    # Two cores; candidates a1 (0, 2400, {1,2}), a2 (300, 2400, {1,2}); behind them waits w (0, 1200, {1}),
+    # which does not fit (the prefix ends before it).  Depth 2.
+    # keep 2: 2400 + 2700, completions {2400, 2700}, w: 2400 + 1200 = 3600             objective 8700
+    # keep 1: a1 at 2 = 1200, completions {1200}; remaining = [a2, w] (evicted first):
+    #         a2 is the first remaining action, so it may try its second level: 1200 + 1500 = 2700,
+    #         then w: 2700 + 1200 = 3900;  1200 + 6600                                  objective 7800
+    # 7800 < 8700: a2 is evicted.  With w ahead of a2 the first remaining action has one level only:
+    # w 2400, a2 at its least level 2400 + 2700 = 5100, objective 1200 + 7500 = 8700, no eviction.
+    rows = [(0, 1, 0x3, 0, 2400), (0, 1, 0x3, 300, 2400), (0, 1, 0x1, 0, 1200)]
+    o = _round(oracle, [(CPU, 2, 2, 0)], rows, depth=2)
+    assert list(o["alloc_units"][0]) == [2, 0, 0]
+    assert o["act_us"][0, 0] == 1200 and o["n_selected"][0] == 1
+
+
+def _replay(oracle, pools, rows, round_us, max_rounds, depth=2):
+    from workloads import Pool
+    n = len(rows)
+    a = dict(pool=np.array([[r[0] for r in rows]], np.uint8), unit=np.array([[r[1] for r in rows]], np.uint8),
+             level_mask=np.array([[r[2] for r in rows]], np.uint32), s_us=np.array([[r[3] for r in rows]], np.int64),
+             p_us=np.array([[r[4] for r in rows]], np.int64), arrival_us=np.array([[r[5] for r in rows]], np.int64),
+             n_actions=np.array([n], np.int32), gpu_busy=None)
+    return oracle.replay_trace([Pool(*p) for p in pools], a, depth=depth, round_us=round_us, max_rounds=max_rounds)
+
+
+def test_running_actions_of_the_same_pool_seed_the_completion_heap(oracle):
+    # Rounds every 1000 us.  Pool 0 has three cores, pool 1 one core.  At t = 0: x (pool 0, one core, runs D)
+    # and z (pool 1, one core, runs 1001) start.  At t = 1000 two actions y1, y2 = (600, 1000, {1,2}) that
+    # arrived at 500 find two free cores on pool 0 and x still running there.
+    # keep both: 1600 + 1600 = 3200.
+    # keep y1 at 2 cores (1100): completions {D - 1000, 1100}; y2 at its second level:
+    #     min(D - 1000, 1100) + 1100;  objective 2200 + min(D - 1000, 1100).
+    # D = 1100: 2300 < 3200, y2 is evicted in this round and starts in the next.
+    # D = 2100: 3300 >= 3200, both start with one core each.
+    # Were the running action left out of the heap the objective would be 3300 for either D; were z's
+    # completion (1 us after the round, but on the other pool) let in, it would be 2201 for either D.
+    pools = [(CPU, 3, 3, 0), (CPU, 1, 1, 0)]
+    for D, evicted in ((1100, True), (2100, False)):
+        rows = [(0, 1, 1, D, 0, 0), (1, 1, 1, 1001, 0, 0), (0, 1, 3, 600, 1000, 500), (0, 1, 3, 600, 1000, 500)]
+        o = _replay(oracle, pools, rows, 1000, 16)
+        assert o["status"][0] == 0
+        assert list(o["alloc_units"][0][:2]) == [1, 1] and list(o["act_us"][0][:2]) == [D, 1001]
+        if evicted:
+            # y1: waited 500, runs 1100 on two cores.  Round 2 (t = 2000): x is gone (finished 1100), y1 runs
+            # until 2100 on two cores, one core is free: y2 is the only candidate, takes it, 1600 us:
+            # completion 3600 - arrival 500
+            assert list(o["alloc_units"][0][2:]) == [2, 1]
+            assert list(o["act_us"][0][2:]) == [500 + 1100, 1500 + 1600]
+        else:
+            assert list(o["alloc_units"][0][2:]) == [1, 1]
+            assert list(o["act_us"][0][2:]) == [500 + 1600, 500 + 1600]
+        # occupancy after the scheduling of rounds 0 and 1
+        assert list(o["occupancy"][0, 0]) == [1, 1]
+        assert list(o["occupancy"][0, 1]) == [3, 1]
+
+
+def test_objective_sums_saturate(oracle):
+    # Two cores, n identical actions (2^40, 2^40, {1,2}): T(1) = 2^41, T(2) = 2^40 + 2^39.  The candidates
+    # are the first two.  With both kept the n - 2 waiting actions start in pairs every 2^41 us: their
+    # completions sum to about 2^41 (n/2)^2.  With one kept there is a single slot and the sum is about
+    # 2^40 n^2, twice as much.
+    # n = 3500: the first objective is about 2^62.6 and exact, the second passes 2^63 and is clamped to
+    # INT64_MAX, which is not smaller: no eviction.  A sum that wrapped around instead would turn
+    # negative and win.
+    # n = 6000: both objectives are INT64_MAX; equal is not smaller, so again no eviction.
+    for n in (3500, 6000):
+        rows = [(0, 1, 0x3, 1 << 40, 1 << 40)] * n
+        o = _round(oracle, [(CPU, 2, 2, 0)], rows, depth=2)
+        assert o["status"][0] == 0 and o["n_selected"][0] == 2
+        assert list(o["alloc_units"][0][:3]) == [1, 1, 0]
+        assert list(o["act_us"][0][:3]) == [1 << 41, 1 << 41, -1]
+        assert o["total_act_us"][0] == 1 << 42
+    # parameters beyond 2^40 are clamped to it (R1), so this is the same round
+    rows = [(0, 1, 0x3, 1 << 45, 1 << 62)] * 3500
+    o = _round(oracle, [(CPU, 2, 2, 0)], rows, depth=2)
+    assert list(o["alloc_units"][0][:3]) == [1, 1, 0] and o["total_act_us"][0] == 1 << 42
+
+
+def test_quota_pool_reports_units_consumed_before_each_grant(oracle):
+    # Section 5.1: three calls of 1, 2 and 3 tokens on a quota pool take tokens 0, 1..2 and 3..5
+    o = _round(oracle, [(API, 10, 0, 1_000_000)], [(0, 1, 1, 5, 0), (0, 2, 1, 5, 0), (0, 3, 1, 5, 0), (0, 5, 1, 5, 0)])
+    assert list(o["alloc_units"][0]) == [1, 2, 3, 0]                 # the fourth call needs 5 of the 4 left
+    assert list(o["place_off"][0]) == [0, 1, 3, -1] and list(o["place_node"][0]) == [0, 0, 0, -1]
+    # a concurrency-limited pool counts the same way within a round
+    o = _round(oracle, [(API, 6, 0, 0)], [(0, 3, 1, 5, 0), (0, 2, 1, 5, 0), (0, 1, 1, 5, 0)])
+    assert list(o["place_off"][0]) == [0, 3, 5]
