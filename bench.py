@@ -8,7 +8,8 @@ row of the hot path: duration model, candidate prefix, per-pool selection, place
 predicted completion times).  Prints ONE JSON line:
   value      actions scheduled per second with inputs resident in HBM (device time, CUDA events)
   e2e        the same through host buffers (host->device and device->host copies timed)
-  roofline   algorithmic bytes of a step / measured duration of the dominant kernel
+  roofline   algorithmic bytes of a step / measured duration of the step, against the measured HBM
+             copy peak; per kernel interval the DRAM bytes ncu counted for it over its own duration
   cpu_baseline  the CPU oracle timed on this machine's cores over a bounded sample
 With --impl reference the oracle itself is timed (bounded sample per step) on the host cores.
 N > 1 runs one independent replica per GPU (scenarios are independent, no collective on the
@@ -38,6 +39,7 @@ METRIC = "actions scheduled/sec (1xB200)"
 # scenarios); traffic grows in proportion to the actions, so a launch's traffic is this times its actions.
 # The k_stream interval of the per-kernel timing holds k_fill as well (it runs beside it).
 NCU_BYTES_PER_ACTION = {"cfg4": {"k_stream": 35.0, "k_head": 1.72, "k_solve": 2.07, "k_finish": 1.89, "k_place": 0.59}}
+NCU_TRAFFIC_SOURCE = "ncu on 2048 scenarios of the same shape, scaled by actions (profiles/)"
 
 
 def _peaks():
@@ -196,7 +198,9 @@ def main():
     if rank == 0 and not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
         v, sample = _oracle_throughput(w, arrays, 15.0, threads)
-        cpu = {"value": v, "unit": "actions/s", "cores": threads, "kind": "oracle", "sample": sample}
+        v1, sample1 = _oracle_throughput(w, arrays, 5.0, 1)
+        cpu = {"value": v, "unit": "actions/s", "cores": threads, "kind": "oracle", "sample": sample,
+               "one_thread": {"value": v1, "unit": "actions/s", "cores": 1, "sample": sample1}}
 
     dev = binding.to_device(arrays)
     rnd = binding.Round(S, N, w.pools, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds)
@@ -271,14 +275,19 @@ def main():
     if rank == 0:
         acts = S * N * world
         peak, which = _peaks()
-        longest = max(ktimes.items(), key=lambda kv: kv[1][0])
-        # the HBM roofline is reported for the kernel interval that moves the bytes (k_stream with k_fill
-        # beside it: 35 of the step's ~42 B per action); it and k_solve, which is bound by instruction issue
-        # and hardly touches DRAM, are the two longest intervals of a step, within a few percent of each other
-        dom = ("k_stream", ktimes["k_stream"]) if ktimes.get("k_stream", (0, 0))[1] else longest
-        dom_ms = dom[1][0] / max(dom[1][1], 1)
-        achieved = ALGO_BYTES_PER_ACTION * S * N / (dom_ms * 1e-3) / 1e9
-        step_gbs = ALGO_BYTES_PER_ACTION * S * N / (ms / args.steps * 1e-3) / 1e9
+        per_step = {k: v[0] / max(v[1], 1) for k, v in ktimes.items() if v[1]}     # ms of each kernel interval per step
+        longest = max(per_step.items(), key=lambda kv: kv[1]) if per_step else ("", 0.0)
+        # The roofline fraction is that of the whole step: the algorithmic bytes of one round (42 B per
+        # pending action) over the step's duration.  Beside it, per kernel interval, the DRAM bytes that ncu
+        # counted for it (scaled by actions) over its own duration.
+        step_ms = ms / args.steps
+        achieved = ALGO_BYTES_PER_ACTION * S * N / (step_ms * 1e-3) / 1e9
+        ncu = NCU_BYTES_PER_ACTION.get(w.name, {})
+        on_traffic = {k: {"ms": per_step[k], "dram_bytes": ncu[k] * S * N,
+                          "achieved_on_traffic_gbs": ncu[k] * S * N / (per_step[k] * 1e-3) / 1e9,
+                          "frac_of_peak": ncu[k] * S * N / (per_step[k] * 1e-3) / 1e9 / peak}
+                      for k in per_step if k in ncu and per_step[k] > 0}
+        traffic = sum(ncu.values()) * S * N if ncu else None
         line = {
             "metric": METRIC, "value": acts * args.steps / (ms * 1e-3), "unit": "actions/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -295,12 +304,13 @@ def main():
                                              "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                                              "ms_per_step": e2e["ms"] / e2e["steps"]},
             "gpu_launches": launches,
-            "roofline": {"bound": "hbm", "kernel": dom[0] + (" (+ k_fill, which runs beside it)" if dom[0] == "k_stream" else ""), "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak,
-                         "traffic": (NCU_BYTES_PER_ACTION.get(w.name, {}).get(dom[0]) or 0) * S * N or None,
-                         "traffic_source": "ncu on 2048 scenarios of the same shape, scaled by actions", "peak_source": which,
-                         "longest_kernel": longest[0], "whole_step_achieved": step_gbs, "whole_step_frac": step_gbs / peak,
-                         "kernel_ms": {k: (v[0] / max(v[1], 1)) for k, v in ktimes.items() if v[1]}},
+            "roofline": {"bound": "hbm", "kernel": "whole step (%s)" % ", ".join(sorted(per_step)),
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "frac_nominal_8TBs": achieved / 8000.0,
+                         "traffic": traffic,
+                         "traffic_source": NCU_TRAFFIC_SOURCE if traffic else None,
+                         "peak_source": which, "longest_kernel": longest[0],
+                         "kernel_ms": per_step, "per_kernel": on_traffic},
             "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)

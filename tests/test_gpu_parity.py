@@ -142,3 +142,48 @@ def test_invalid_record_far_behind_the_prefix_matches_oracle(oracle):
     g = gpu_round(w.pools, a, depth=w.depth)
     assert_same(o, g)
     assert list(g["status"][[3, 7, 9]]) == [1, 1, 1] and g["n_selected"][3] == 0
+
+
+def test_saturating_objectives_match_oracle(oracle):
+    # queues of identical actions with s = p = 2^40: the completion times leave the 49 bits of the packed
+    # simulation keys, and the sums of the longer queues pass 2^63 and are clamped
+    pools = (Pool(POOL_CPU, 2, 2),)
+    S, N = 6, 6000
+    a = dict(pool=np.zeros((S, N), np.uint8), unit=np.ones((S, N), np.uint8),
+             level_mask=np.full((S, N), 3, np.uint32), s_us=np.full((S, N), 1 << 40, np.int64),
+             p_us=np.full((S, N), 1 << 40, np.int64), arrival_us=None,
+             n_actions=np.array([3500, 6000, 40, 2900, 3000, 4096], np.int32), gpu_busy=None)
+    a["s_us"][5, :] = 0                                # s < p / 2: the eviction pays while nothing saturates
+    a["n_actions"][5] = 3
+    for depth in (1, 2):
+        o = oracle.schedule_batch(pools, a, depth=depth)
+        g = gpu_round(pools, a, depth=depth)
+        assert_same(o, g)
+    assert list(o["alloc_units"][0][:2]) == [1, 1] and list(o["alloc_units"][5][:2]) == [2, 0]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_unnarrowed_random_rounds_match_oracle(oracle, seed):
+    # replica requests with up to 32 multiplicities, gang masks with unusable levels among usable ones,
+    # elastic quota actions, a few invalid records
+    pools = POOLSETS[seed % len(POOLSETS)]
+    w, a = random_round(800 + seed, 96, [60, 150][seed % 2], pools, narrow=False, max_mult=[32, 12, 6][seed % 3],
+                        small_durations=0.5 if seed % 2 else 0.0, busy_fraction=0.3 if seed % 3 == 0 else 0.0)
+    for depth in (2, 1):
+        o = oracle.schedule_batch(pools, a, depth=depth)
+        g = gpu_round(pools, a, depth=depth)
+        assert_same(o, g)
+    assert (o["status"] == 0).sum() > 10 and (o["status"] != 0).sum() > 0
+
+
+@pytest.mark.parametrize("seed,nodes", [(0, 32), (1, 40), (2, 64)])
+def test_fragmented_pool_with_elastic_gang_requests_matches_oracle(oracle, seed, nodes):
+    # gang requests (one chunk that grows with the level) couple the chunk sizes, so the per-size
+    # decomposition does not apply; mixed with replica requests on a fragmented pool of many nodes
+    pools = (Pool(POOL_GPU, 8 * nodes, 8),)
+    w, a = random_round(6100 + seed, 10, 260, pools, replicas=0.5, busy_fraction=0.35, inelastic=0.2,
+                        max_mult=8, small_durations=0.3 if seed == 1 else 0.0)
+    o = oracle.schedule_batch(pools, a)
+    g = gpu_round(pools, a)
+    assert_same(o, g)
+    assert np.all(g["status"] == 0) and o["n_selected"].max() > 30

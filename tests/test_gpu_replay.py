@@ -76,3 +76,40 @@ def test_replay_flags_bad_input(oracle):
     g = gpu_replay(pools, a, 2, 10_000, 200)
     assert_same(o, g)
     assert list(g["status"]) == [0, 2, 1, 0]
+
+
+def test_cfg2_full_size_sampled_scenarios_match_oracle(oracle):
+    # the whole 256 x 20000 trace on the GPU; eight scenarios recomputed by the oracle, everything compared
+    w = make_workload("cfg2")
+    a = generate(w)
+    g = gpu_replay(w.pools, a, w.depth, w.round_us, w.max_rounds)
+    assert np.all(g["status"] == 0) and np.all(g["n_selected"] == w.max_actions)
+    assert np.all(g["rounds_used"] < w.max_rounds)
+    rng = np.random.default_rng(3)
+    for sc in np.unique(np.concatenate([[0, w.n_scenarios - 1], rng.integers(0, w.n_scenarios, 6)])):
+        o = oracle.replay_trace(w.pools, a, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds,
+                                lo=int(sc), hi=int(sc) + 1)
+        for k in KEYS:
+            assert np.array_equal(o[k][0], g[k][sc]), f"scenario {sc}: {k} differs"
+    # conservation on every scenario: each action ran once, with a legal allocation
+    assert np.all(g["alloc_units"] > 0) and np.all(g["act_us"] >= 0)
+    assert np.array_equal(g["act_us"].sum(1), g["total_act_us"])
+
+
+def test_long_running_sets_match_oracle(oracle):
+    # a burst of long single-core actions on a pool of 600 cores: more than 448 actions run at once,
+    # so the completion heap of the estimates outgrows the warp's shared-memory tree
+    pools = (Pool(POOL_CPU, 600, 60),)
+    S, N = 4, 1400
+    rng = np.random.default_rng(17)
+    elastic = rng.random((S, N)) < 0.3
+    a = dict(pool=np.zeros((S, N), np.uint8), unit=np.ones((S, N), np.uint8),
+             level_mask=np.where(elastic, 0xB, 1).astype(np.uint32),
+             s_us=rng.integers(200_000, 900_000, (S, N)).astype(np.int64),
+             p_us=np.where(elastic, rng.integers(0, 2_000_000, (S, N)), 0).astype(np.int64),
+             arrival_us=np.cumsum(rng.integers(0, 600, (S, N)), axis=1).astype(np.int64),
+             n_actions=np.full(S, N, np.int32), gpu_busy=None)
+    o = oracle.replay_trace(pools, a, depth=2, round_us=10_000, max_rounds=600)
+    g = gpu_replay(pools, a, 2, 10_000, 600)
+    assert_same(o, g)
+    assert o["occupancy"][:, :, 0].max() > 448 and np.all(o["n_selected"] == N)

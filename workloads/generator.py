@@ -304,11 +304,13 @@ def generate(w: Workload, lo: int = 0, hi: Optional[int] = None) -> Dict[str, Op
 def random_round(seed: int, n_scenarios: int, max_actions: int, pools: Tuple[Pool, ...],
                  *, contiguous_levels: float = 0.3, max_mult: int = 8, inelastic: float = 0.25,
                  small_durations: float = 0.0, busy_fraction: float = 0.0, ragged: bool = True,
-                 replicas: float = 0.5) -> Tuple[Workload, Dict[str, Optional[np.ndarray]]]:
+                 replicas: float = 0.5, narrow: bool = True) -> Tuple[Workload, Dict[str, Optional[np.ndarray]]]:
     """Adversarial little rounds for parity and property tests: arbitrary level masks
     (power-of-two sets, contiguous ranges, random subsets), mixed gang/replica GPU
     requests, ragged action counts, optional tiny durations (forces ties) and
-    pre-occupied GPUs."""
+    pre-occupied GPUs.  With narrow=False the masks are left as drawn: replica requests with up
+    to max_mult multiplicities, gang requests whose masks hold unusable levels among usable
+    ones (and sometimes none, which makes the record invalid), elastic quota actions."""
     rng = np.random.Generator(np.random.PCG64(seed))
     S, N = n_scenarios, max_actions
     w = Workload(f"random{seed}", S, N, tuple(pools), "random", base_seed=seed,
@@ -331,12 +333,16 @@ def random_round(seed: int, n_scenarios: int, max_actions: int, pools: Tuple[Poo
     unit = np.where(rep, np.minimum(np.int64(1) << rng.integers(0, 4, size=(S, N)), grp), unit)
     unit = np.where(is_gpu & ~rep, 1 | GANG, unit)
     # gang requests need power-of-two levels <= GPUs per node; replicas keep few multiplicities
-    gang_ok = np.array([_pow2_mask(int(c)) for c in range(0, 33)], dtype=np.int64)[np.minimum(grp, 32)]
-    mask = np.where(is_gpu & ~rep, mask & gang_ok, mask)
-    mask = np.where(is_gpu & ~rep & (mask == 0), 1, mask)
-    mask = np.where(rep, mask & 0xF, mask)
-    mask = np.where(rep & (mask == 0), 1, mask)
-    mask = np.where(ptype == POOL_API, 1, mask)
+    if narrow:
+        gang_ok = np.array([_pow2_mask(int(c)) for c in range(0, 33)], dtype=np.int64)[np.minimum(grp, 32)]
+        mask = np.where(is_gpu & ~rep, mask & gang_ok, mask)
+        mask = np.where(is_gpu & ~rep & (mask == 0), 1, mask)
+        mask = np.where(rep, mask & 0xF, mask)
+        mask = np.where(rep & (mask == 0), 1, mask)
+        mask = np.where(ptype == POOL_API, 1, mask)
+    else:
+        # most gang records keep a usable level (one GPU); the few that do not are invalid records
+        mask = np.where(is_gpu & ~rep & (rng.random((S, N)) < 0.97), mask | 1, mask)
     if small_durations > 0.0:
         tiny = rng.random((S, N)) < small_durations
     else:
