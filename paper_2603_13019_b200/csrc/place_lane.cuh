@@ -68,7 +68,9 @@ __device__ __forceinline__ void kpl_store(const Params& P, KplWarp& W, size_t ro
   __syncwarp();
 }
 
-__global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ Params P, const HeadState* hst) {
+// phase 0: the pools that the head kernel certified (decided by k_easy); phase 1: all the others, and
+// the cleaning up behind scenarios with an invalid record.
+__global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ Params P, const HeadState* hst, int phase) {
   __shared__ KplWarp s_w[KPL_WARPS];
   const int lane = threadIdx.x & 31;
   KplWarp& W = s_w[threadIdx.x >> 5];
@@ -81,7 +83,7 @@ __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ P
   // where k_stream finds it while k_solve is already deciding the scenario's pools; so the last
   // kernel of the round takes back whatever was written for such a scenario.
   const bool bad = sc < P.S && (P.o_status[sc] & TG_ST_BAD_ACTION);
-  if (bad && gw / wps == 0) {
+  if (bad && gw / wps == 0 && phase == 1) {
     const size_t r0 = (size_t)sc * P.N;
     for (int i = 0; i < min(hst[sc].n, P.N); ++i) { P.o_alloc[r0 + i] = 0; P.o_node[r0 + i] = -1; P.o_off[r0 + i] = -1; P.o_act[r0 + i] = -1; }
     P.o_total[sc] = 0; P.o_nsel[sc] = 0; P.o_status[sc] = TG_ST_BAD_ACTION;
@@ -89,6 +91,7 @@ __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ P
   if (!pd.lane_place) return;
   int keep = (sc < P.S && !bad) ? P.keepn[(size_t)sc * P.P + j] : 0;
   if (keep < 0) keep = 0;
+  if (sc < P.S && (int)(((hst[sc].need >> j) & 1u) != 0u) != phase) keep = 0;   // the other phase's pool
   const int maxkeep = warp_max32(keep);
   if (maxkeep == 0) return;
   const size_t row = (size_t)(sc < P.S ? sc : 0) * P.N;

@@ -157,6 +157,14 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
     }
   }
   const u32 elw = __reduce_or_sync(TG_FULL, el);
+  if (hs == n_act && n_pref == n_act) {
+    // the whole queue is the candidate prefix: the same test tells which pools are certified
+    const u32 unfit = __ballot_sync(TG_FULL, lane < D && mxd > capreg);
+    for (int jj = 0; jj < P.P; ++jj) {
+      const u32 slots = ((1u << P.pool[jj].n_slots) - 1u) << P.pool[jj].slot0;
+      if (((elw >> jj) & 1u) && (unfit & slots)) need |= 1u << jj;
+    }
+  }
   const int anybad = __any_sync(TG_FULL, bad) ? 1 : 0;
   if (lane < P.P) {
     PoolMeta mt;

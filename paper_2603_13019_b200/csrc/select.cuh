@@ -876,11 +876,24 @@ __device__ bool estimate_rest(const Params& P, const PoolTask& T, int q, const u
   else { fs = T.ac_first.s; fp = T.ac_first.p; fm = T.ac_first.mask; }
   const int dmax = min(min(T.depth, __popc(fm)), 32);
   const int H = T.n_seeds + q;
-  if (H <= 128) {
-    // the whole warp on one simulation, one depth (the largest level tried is the best one)
+  if (H <= 256) {
+    // the whole warp on one simulation, one depth (the largest level tried is the best one):
+    // 32-bit times on a sorted array first, packed 64-bit keys if a time leaves 32 bits
     bool overflow;
     const i64 fd = duration(fs, fp, nth_level_of(fm, dmax - 1));
-    const i64 val = warp_sim<4>(
+    auto seed_of = [&](int i) { return i < T.n_seeds ? T.seeds[i]
+                                                     : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], alloc[i - T.n_seeds]); };
+    auto dur_of = [&](int k) { return k == 0 ? fd
+                                   : (k < n_ev ? duration(T.cs[q + k], T.cp[q + k], __ffs(T.cmask[q + k])) : T.ac_tmin[k - n_ev]); };
+    i64 fast;
+    if (H <= 32) fast = sorted_sim<1>(H, n_rest, seed_of, dur_of, lane, &overflow);
+    else if (H <= 64) fast = sorted_sim<2>(H, n_rest, seed_of, dur_of, lane, &overflow);
+    else if (H <= 96) fast = sorted_sim<3>(H, n_rest, seed_of, dur_of, lane, &overflow);
+    else if (H <= 128) fast = sorted_sim<4>(H, n_rest, seed_of, dur_of, lane, &overflow);
+    else if (H <= 192) fast = sorted_sim<6>(H, n_rest, seed_of, dur_of, lane, &overflow);
+    else fast = sorted_sim<8>(H, n_rest, seed_of, dur_of, lane, &overflow);
+    if (!overflow) { *est = fast; return true; }
+    const i64 val = warp_sim<8>(
         H, n_rest,
         [&](int i) { return i < T.n_seeds ? T.seeds[i]
                                           : duration(T.cs[i - T.n_seeds], T.cp[i - T.n_seeds], alloc[i - T.n_seeds]); },
@@ -1060,10 +1073,8 @@ __device__ __noinline__ int evict_batch(const Params& P, const PoolTask& T, Slab
 __device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int lane, i64 obj, int keep,
                             bool have_obj = true, i64 opt_keep = 0) {
   i64 opt, est;
-  if (have_obj && keep < T.m) {                          // an eviction has been accepted already: look further ahead
-    const int kb = evict_batch(P, PoolTask(T), slab, lane, obj, keep);
-    if (kb != -2) return kb;
-  }
+  // (most chains end with the step after the first accepted eviction: that step is taken alone,
+  // and only a chain that goes on looks several steps ahead)
   for (int t = T.m - keep + 1; t <= T.m - 1; ++t) {
     const int q = T.m - t;
     if (!solve_prefix(P, T, q, slab, lane, &opt)) return -1;

@@ -311,6 +311,75 @@ __device__ __forceinline__ i64 warp_sim(int H, int steps, SeedFn seed, DurFn dur
   return total;
 }
 
+// One simulation run by a whole warp on a SORTED array of completion times spread over the lanes:
+// position i lives in lane i & 31, register i >> 5 (H <= 32 * NS), unused positions hold
+// 0xffffffff.  "Pop the earliest, push earliest + T" removes position 0 and inserts the new time
+// where it belongs: every lane compares its elements with it, one vote per register counts the
+// smaller ones, and the elements in front of that place move down one position (a rotation by one
+// lane per register, which does not depend on the new time and is issued ahead).  The two earliest
+// times are also kept in every lane, so that the next completion is known a few instructions after
+// the step starts; no reduction sits on the path from step to step.
+// Keys are 32-bit completion times saturated at SORTED_SAT (about 71 minutes); the sum of
+// completions is exact: the popped keys are exact as long as none of them is saturated, and the
+// durations are summed apart, 32 at a time.  A saturated key that gets popped sets *overflow: the
+// caller then uses an exact 64-bit simulation.
+#define SORTED_SAT 0xfffffffeu
+template <int NS>
+__device__ __forceinline__ void sorted_replace_min(u32 (&key)[NS], u32 c, int lane) {
+  int lt = 0;
+#pragma unroll
+  for (int r = 0; r < NS; ++r) lt += __popc(__ballot_sync(TG_FULL, key[r] < c));
+  const int cnt = max(lt - 1, 0);                        // where c goes once position 0 is gone
+  u32 rot[NS + 1];
+#pragma unroll
+  for (int r = 0; r < NS; ++r) rot[r] = __shfl_sync(TG_FULL, key[r], (lane + 1) & 31);
+  rot[NS] = 0xffffffffu;
+#pragma unroll
+  for (int r = 0; r < NS; ++r) {
+    const int pos = r * 32 + lane;
+    const u32 next = lane < 31 ? rot[r] : rot[r + 1];    // the element one position behind
+    key[r] = pos < cnt ? next : (pos == cnt ? c : key[r]);
+  }
+}
+__device__ __forceinline__ u32 sorted_key(i64 v) { return v >= (i64)SORTED_SAT ? SORTED_SAT : (u32)v; }
+
+template <int NS, class SeedFn, class DurFn>
+__device__ __forceinline__ i64 sorted_sim(int H, int steps, SeedFn seed, DurFn dur, int lane, bool* overflow) {
+  u32 key[NS];
+  // start from H zeros (no seed is smaller) and replace them by the seeds one by one
+#pragma unroll
+  for (int r = 0; r < NS; ++r) key[r] = r * 32 + lane < H ? 0u : 0xffffffffu;
+  for (int i0 = 0; i0 < H; i0 += 32) {
+    const u32 mine = i0 + lane < H ? sorted_key(seed(i0 + lane)) : 0u;
+    const int nb = min(32, H - i0);
+    for (int b = 0; b < nb; ++b) sorted_replace_min<NS>(key, __shfl_sync(TG_FULL, mine, b), lane);
+  }
+  u32 t0 = __shfl_sync(TG_FULL, key[0], 0), t1 = __shfl_sync(TG_FULL, key[0], 1);
+  i64 total = 0;
+  bool ovf = false;
+  for (int k0 = 0; k0 < steps; k0 += 32) {
+    const i64 mine = k0 + lane < steps ? dur(k0 + lane) : 0;
+    const u32 mine32 = sorted_key(mine);
+    const int nb = min(32, steps - k0);
+    u64 pops = 0;                                        // 32 popped keys below 2^32 each
+    for (int b = 0; b < nb; ++b) {
+      const u32 d = __shfl_sync(TG_FULL, mine32, b);
+      const u32 b2 = __shfl_sync(TG_FULL, key[0], 2);    // the third earliest time
+      ovf |= t0 >= SORTED_SAT;                           // the popped key is not an exact time any more
+      pops += t0;
+      const u64 c64 = (u64)t0 + d;                       // pop the earliest completion ts, push ts + T
+      const u32 c = c64 >= SORTED_SAT ? SORTED_SAT : (u32)c64;
+      sorted_replace_min<NS>(key, c, lane);
+      const bool lt1 = t1 < c, lt2 = b2 < c;
+      t0 = lt1 ? t1 : c;
+      t1 = lt1 ? (lt2 ? b2 : c) : t1;
+    }
+    total = sat_add(total, (i64)pops + warp_sum64(mine));  // completions = popped times + durations
+  }
+  *overflow = ovf;
+  return total;
+}
+
 // One persistent warp per block, one lane per simulation (trees interleaved by lane: SS = 8).
 template <int MAXD>
 __global__ void __launch_bounds__(32) k_sims1(const __grid_constant__ Params P, TaskState* ts, const i64* seed2,

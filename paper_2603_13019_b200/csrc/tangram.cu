@@ -237,6 +237,44 @@ __global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ P
   }
 }
 
+// The pools that the head kernel certified (no elastic candidate, or every candidate's largest level
+// fits: then each takes the smallest level that reaches its lowest duration and no eviction can
+// pay) need no selection at all.  One warp per such (scenario, pool), nothing but registers: the
+// candidates' allocations and predicted completion times (Eq. 2) are written, their requests are
+// left for the placement kernel.  Runs beside the streaming kernel, on a stream of its own.
+__global__ void __launch_bounds__(256) k_easy(const __grid_constant__ Params P, const HeadState* hst) {
+  const int lane = threadIdx.x & 31;
+  const long long x = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (x >= (long long)P.S * P.P) return;
+  const int sc = (int)(x % P.S), j = P.pool_order[x / P.S], task = sc * P.P + j;
+  const PoolDev& pd = P.pool[j];
+  if (((hst[sc].need >> j) & 1u) || !pd.lane_place) return;
+  const PoolMeta mt = P.meta[task];
+  const int m = mt.m;
+  if (lane == 0) P.keepn[task] = m;
+  if (m == 0) return;
+  const size_t row = (size_t)sc * P.N;
+  const int* ord = P.order + row + mt.base;
+  unsigned short* rq = P.preq + row + mt.base;
+  i64 tot = 0; int cnt = 0;
+  for (int i = lane; i < m; i += 32) {
+    const size_t o = row + ord[i];
+    int g, gang; u32 eff;
+    decode_levels(pd, P.a_unit[o], P.a_mask[o], g, gang, eff);
+    const i64 s = clamp_param(P.a_s[o]), p = clamp_param(P.a_p[o]);
+    const int r = best_level(p, eff);
+    const i64 act = (P.now - (P.a_arrival ? P.a_arrival[o] : 0)) + duration(s, p, r);
+    P.o_alloc[o] = g * r; P.o_act[o] = act;
+    rq[i] = (unsigned short)((u32)g | ((u32)gang << 7) | ((u32)r << 8));
+    tot += act; ++cnt;
+  }
+  tot = warp_sum64(tot); cnt = warp_sum32(cnt);
+  if (lane == 0) {
+    atomicAdd((u64*)&P.o_total[sc], (u64)tot);
+    atomicAdd(&P.o_nsel[sc], cnt);
+  }
+}
+
 // workspace of the batched path, indexed like the partitioned arrays
 struct BatchWs {
   TaskState* ts;   // [S][P]
@@ -245,7 +283,7 @@ struct BatchWs {
   u8* rs2;         // [S][N] ... of the first m-1
 };
 
-__global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__ Params P, const BatchWs W) {
+__global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__ Params P, const BatchWs W, const HeadState* hst) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
   const int n_tasks = P.S * P.P;
@@ -253,8 +291,12 @@ __global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__
     const int x = next_task(P.arena_top + 1, lane);
     if (x >= n_tasks) break;
     const int sc = x % P.S, j = P.pool_order[x / P.S], task = sc * P.P + j;
-    const PoolMeta mt = P.meta[task];
     TaskState* st = W.ts + task;
+    if (!((hst[sc].need >> j) & 1u) && P.pool[j].lane_place) {   // certified by the head kernel: k_easy has it
+      if (lane == 0) st->flags = TS_DECIDED;
+      continue;
+    }
+    const PoolMeta mt = P.meta[task];
     if (lane == 0) P.keepn[task] = -1;                   // nothing for k_place unless a decision says so
     if (mt.m == 0) { if (lane == 0) st->flags = TS_DECIDED; continue; }
     Slab slab = warp_slab(P, gw);
@@ -409,6 +451,8 @@ struct tangram_round {
   // and a join event so that their partial waves overlap
   cudaStream_t sim_stream[TG_N_SIM_CLASSES + 1];
   cudaEvent_t sim_fork, sim_join[TG_N_SIM_CLASSES + 1];
+  // the certified pools (k_easy and their placement) run beside the kernels that follow k_solve
+  cudaStream_t side; cudaEvent_t side_fork, side_join;
   // staging for host-buffer mode
   char* d_stage; size_t stage_bytes;
   size_t in_off[8], out_off[9];
@@ -606,6 +650,13 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
       bad |= cudaStreamCreateWithFlags(&r->sim_stream[c], cudaStreamNonBlocking) != cudaSuccess;
     bad |= cudaEventCreateWithFlags(&r->sim_join[c], cudaEventDisableTiming) != cudaSuccess;
   }
+  {
+    int lo = 0, hi = 0;
+    bad |= cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess;
+    bad |= cudaStreamCreateWithPriority(&r->side, cudaStreamNonBlocking, lo) != cudaSuccess;
+    bad |= cudaEventCreateWithFlags(&r->side_fork, cudaEventDisableTiming) != cudaSuccess;
+    bad |= cudaEventCreateWithFlags(&r->side_join, cudaEventDisableTiming) != cudaSuccess;
+  }
   if (!bad && desc->host_buffers) {
     bad |= cudaStreamCreateWithFlags(&r->io_in, cudaStreamNonBlocking) != cudaSuccess;
     bad |= cudaStreamCreateWithFlags(&r->io_comp, cudaStreamNonBlocking) != cudaSuccess;
@@ -710,6 +761,9 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
     if (r->io_in_done[c]) cudaEventDestroy(r->io_in_done[c]);
     if (r->io_comp_done[c]) cudaEventDestroy(r->io_comp_done[c]);
   }
+  if (r->side) cudaStreamDestroy(r->side);
+  if (r->side_fork) cudaEventDestroy(r->side_fork);
+  if (r->side_join) cudaEventDestroy(r->side_join);
   if (r->sim_fork) cudaEventDestroy(r->sim_fork);
   for (int c = 0; c <= TG_N_SIM_CLASSES; ++c) {
     if (r->sim_stream[c]) cudaStreamDestroy(r->sim_stream[c]);
@@ -782,6 +836,7 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   if (ev) CK(cudaEventRecord(ev[0], st));
   k_head<<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[1], st));
+  const unsigned place_grid = ((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS;
   {                                                        // the output fill runs beside everything that follows
     cudaStream_t fs = r->sim_stream[TG_N_SIM_CLASSES];
     CK(cudaEventRecord(r->sim_fork, st));
@@ -795,7 +850,7 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   // other's way on the SMs (1.6 ms together against 0.65 + 0.70 one after the other), so they do not
   k_stream<<<P.S, KS_THREADS, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[2], st));
-  k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W);
+  k_solve<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W, r->hst);
   if (ev) CK(cudaEventRecord(ev[3], st));
   CK(cudaMemsetAsync(L.count, 0, 2 * 64 * sizeof(int), st));
   k_sim_classify<<<(L.n_groups + 7) / 8, 256, 0, st>>>(P, W.ts, L);
@@ -815,14 +870,23 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   }
   k_sims_big<<<(int)((n_sims + 31) / 32), 32, 0, st>>>(P, W.ts, W.seed2, g_sim_caps[TG_N_SIM_CLASSES - 1], L.count + 63);
   if (ev) CK(cudaEventRecord(ev[4], st));
+  {                                                        // the certified pools: decided and placed beside the continued evictions,
+                                                           // which are chains of dependent steps that leave most of the machine idle
+    CK(cudaEventRecord(r->side_fork, st));
+    CK(cudaStreamWaitEvent(r->side, r->side_fork, 0));
+    k_easy<<<(unsigned)(((size_t)P.S * P.P + 7) / 8), 256, 0, r->side>>>(P, r->hst);
+    k_place<<<place_grid, KPL_THREADS, 0, r->side>>>(P, r->hst, 0);
+    CK(cudaEventRecord(r->side_join, r->side));
+  }
   CK(cudaMemsetAsync(r->d_fl, 0, 2 * sizeof(int), st));
   k_finish_list<<<(P.S * P.P + 255) / 256, 256, 0, st>>>(P, W, r->d_fl);
   k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W, r->d_fl);
   if (ev) CK(cudaEventRecord(ev[5], st));
-  k_place<<<((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS, KPL_THREADS, 0, st>>>(P, r->hst);
+  k_place<<<place_grid, KPL_THREADS, 0, st>>>(P, r->hst, 1);
+  CK(cudaStreamWaitEvent(st, r->side_join, 0));
   CK(cudaStreamWaitEvent(st, r->sim_join[TG_N_SIM_CLASSES], 0));   // the fill is part of the round
   if (ev) CK(cudaEventRecord(ev[6], st));
-  r->launches += 9 + TG_N_SIM_CLASSES;
+  r->launches += 11 + TG_N_SIM_CLASSES;
   CK(cudaGetLastError());
   return TANGRAM_OK;
 }
