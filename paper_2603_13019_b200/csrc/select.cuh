@@ -359,6 +359,51 @@ __device__ u32 dp_small_multi(const PoolTask& T, int nrows, int ncell, const int
   return solved;
 }
 
+// ---- marginal gains of a class of rows whose steps all have the same size ------------------
+// A row with contiguous multiplicities r0 .. rmax offers the steps r0 -> r0+1 -> ... each worth one
+// chunk of the class's size; step k (1-based) gains T(r0+k-1) - T(r0+k) >= 0.  If every row's gains
+// are non-increasing (the floor in Eq. 1 can break that; such a class goes through its DP), the
+// least duration sum with exactly x extra chunks is the sum at the least levels minus the x
+// largest gains (separable convex resource allocation), and among allocations of equal value the
+// canonical order (a later queue position gets less) takes equal gains from the earliest rows
+// first.  So the steps are sorted by one key: gain descending, row ascending, step ascending, and
+// every x is served by a prefix of that order; an allocation is read back from the threshold
+// key at the cut.  All steps of a class have the same size, so comparing gains is comparing
+// densities; nothing is divided.
+#define MG_GAIN_BITS 41
+#define MG_ROW_BITS 18
+#define MG_GAIN_MAX ((1ull << MG_GAIN_BITS) - 1ull)
+__device__ __forceinline__ u64 mg_key(i64 gain, int row, int step) {     // step 1-based, at most 31
+  return ((MG_GAIN_MAX - (u64)gain) << (MG_ROW_BITS + 5)) | ((u64)row << 5) | (u64)(step - 1);
+}
+__device__ __forceinline__ i64 mg_gain(u64 key) { return (i64)(MG_GAIN_MAX - (key >> (MG_ROW_BITS + 5))); }
+// contiguous multiplicities and non-increasing gains
+__device__ __forceinline__ bool mg_row_ok(i64 s, i64 p, u32 mk) {
+  const int r0 = __ffs(mk), rmax = 32 - __clz(mk);
+  if (mk != ((rmax == 32 ? 0xffffffffu : ((1u << rmax) - 1u)) & ~((1u << (r0 - 1)) - 1u))) return false;
+  i64 before = duration(s, p, r0), last_gain = TG_INF;
+  for (int r = r0 + 1; r <= rmax; ++r) {
+    const i64 now = duration(s, p, r), gain = before - now;
+    if (gain > last_gain) return false;
+    last_gain = gain; before = now;
+  }
+  return true;
+}
+// ascending bitonic sort of n (a power of two) keys by the calling warp
+__device__ __forceinline__ void warp_sort_u64(u64* a, int n, int lane) {
+  for (int k = 2; k <= n; k <<= 1)
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = lane; i < n; i += 32) {
+        const int l = i ^ j;
+        if (l > i) {
+          const u64 x = a[i], y = a[l];
+          if ((x > y) == ((i & k) == 0)) { a[i] = y; a[l] = x; }
+        }
+      }
+      __syncwarp();
+    }
+}
+
 // DPArrange on a fragmented GPU pool (Algorithm 4) when no row is a gang request: a row of chunk
 // size 2^c only ever adds requests of that size, so the rows fall into four classes that
 // interact through nothing but the nested capacities (extra GPUs at sizes >= 2^l <= Y[l]).  Per
@@ -372,38 +417,48 @@ __device__ u32 dp_small_multi(const PoolTask& T, int nrows, int ncell, const int
 // loop (as it does when the scratch does not suffice).  Rows are T.rowcand[0..nrows).
 #define DPC_MAX_CELLS 4096
 __device__ __noinline__ int dp_classes(const PoolTask& T, int nrows, const int Y[4], const int maxex[4], Slab slab, int lane) {
-  // class sizes
+  // class sizes; which classes can go by their marginal gains
   int rows_c[4] = {0, 0, 0, 0}, mx_c[4] = {0, 0, 0, 0};  // rows and largest extra chunks per class
   bool gang_row = false;
+  u32 not_convex = 0;
+  i64 base_c[4] = {0, 0, 0, 0};                          // duration sum of the class at the least levels
   for (int t = lane; t < nrows; t += 32) {
     const int i = T.rowcand[t];
     const int g = T.cg[i] & 0x7f;
     if (T.cg[i] >> 7) gang_row = true;
     const u32 mk = T.cmask[i];
     const int c = ilog2(g), ex = (32 - __clz(mk)) - __ffs(mk);
+    const i64 s = T.cs[i], p = T.cp[i];
+    const i64 tl = duration(s, p, __ffs(mk));
+    if (!mg_row_ok(s, p, mk)) not_convex |= 1u << c;
 #pragma unroll
-    for (int l = 0; l < 4; ++l) if (l == c) { rows_c[l] += 1; mx_c[l] += ex; }
+    for (int l = 0; l < 4; ++l) if (l == c) { rows_c[l] += 1; mx_c[l] += ex; base_c[l] += tl; }
   }
   if (__any_sync(TG_FULL, gang_row)) return 0;
+  not_convex = __reduce_or_sync(TG_FULL, not_convex);
   int U[4];                                               // largest useful number of extra chunks per class
-  u64 need = 0;
+  bool by_gain[4];
 #pragma unroll
   for (int l = 0; l < 4; ++l) {
-    rows_c[l] = warp_sum32(rows_c[l]); mx_c[l] = warp_sum32(mx_c[l]);
+    rows_c[l] = warp_sum32(rows_c[l]); mx_c[l] = warp_sum32(mx_c[l]); base_c[l] = warp_sum64(base_c[l]);
     U[l] = min(max(Y[l], 0) >> l, mx_c[l]);
     if (U[l] + 1 > DPC_MAX_CELLS || (Y[l] >> l) + 1 > 2 * DPC_MAX_CELLS) return 0;
-    need += (u64)rows_c[l] * (U[l] + 1) + 3 * (u64)(U[l] + 1) * 8 + 16 * 4;
+    by_gain[l] = !((not_convex >> l) & 1u) && nrows < (1 << MG_ROW_BITS) && mx_c[l] >= 1;
   }
   (void)maxex;
-  // scratch: per class f (final values), two work rows, choices; merged tables
-  i64* f[4]; u8* ch[4];
+  // scratch: per class f (final values), two work rows, choices or sorted step keys; merged tables
+  i64* f[4]; u8* ch[4]; u64* keys[4]; int npad[4];
   i64* work = nullptr;
   int Umax = max(max(U[0], U[1]), max(U[2], U[3]));
   work = (i64*)slab.take(2 * (u64)(Umax + 1) * 8);
 #pragma unroll
   for (int l = 0; l < 4; ++l) {
     f[l] = (i64*)slab.take((u64)(U[l] + 1) * 8);
-    ch[l] = (u8*)slab.take((u64)max(rows_c[l], 1) * (U[l] + 1));
+    npad[l] = 1;
+    while (npad[l] < mx_c[l]) npad[l] <<= 1;
+    keys[l] = by_gain[l] ? (u64*)slab.take((u64)npad[l] * 8) : nullptr;
+    ch[l] = by_gain[l] ? (u8*)f[l] : (u8*)slab.take((u64)max(rows_c[l], 1) * (U[l] + 1));
+    if (by_gain[l] && !keys[l]) return 0;
   }
   // merged tables: E[l] cells in chunks of 2^l, value, chosen cell of the level above, tie flag
   int E[4];
@@ -419,11 +474,77 @@ __device__ __noinline__ int dp_classes(const PoolTask& T, int nrows, const int Y
 #pragma unroll
   for (int l = 0; l < 4; ++l) if (!f[l] || !ch[l] || !G[l] || !gsel[l] || !gtie[l]) return 0;
 
-  // ---- per class: one-dimensional DP over its rows, in queue order
+  // ---- step keys of the classes that go by their gains: every row writes its steps behind those
+  // ---- of the rows before it (one scan per class and block of 32 rows)
+  {
+    int fill[4] = {0, 0, 0, 0};
+    for (int t0 = 0; t0 < nrows; t0 += 32) {
+      const int t = t0 + lane;
+      int c = -1, ex = 0, r0 = 1; i64 s = 0, p = 0;
+      if (t < nrows) {
+        const int i = T.rowcand[t];
+        const u32 mk = T.cmask[i];
+        c = ilog2(T.cg[i] & 0x7f); r0 = __ffs(mk); ex = (32 - __clz(mk)) - r0;
+        s = T.cs[i]; p = T.cp[i];
+      }
+#pragma unroll
+      for (int l = 0; l < 4; ++l) {
+        if (!by_gain[l]) continue;
+        const int mine = c == l ? ex : 0;
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(TG_FULL, incl, o); if (lane >= o) incl += y; }
+        if (c == l) {
+          u64* dst = keys[l] + fill[l] + incl - mine;
+          i64 before = duration(s, p, r0);
+          for (int k = 1; k <= ex; ++k) {
+            const i64 now = duration(s, p, r0 + k);
+            dst[k - 1] = mg_key(before - now, t, k);
+            before = now;
+          }
+        }
+        fill[l] += __shfl_sync(TG_FULL, incl, 31);
+      }
+    }
+#pragma unroll
+    for (int l = 0; l < 4; ++l)
+      if (by_gain[l]) for (int x = mx_c[l] + lane; x < npad[l]; x += 32) keys[l][x] = ~0ull;
+    __syncwarp();
+  }
+
+  // ---- per class: f_c(x), least duration sum with exactly x extra chunks
 #pragma unroll 1
   for (int c = 0; c < 4; ++c) {
-    i64* prev = work; i64* cur = work + (Umax + 1);
     const int Uc = U[c];
+    if (by_gain[c]) {
+      // sorted steps (in the warp's shared memory when they fit), then f_c(x) = base - the x largest gains
+      u64* srt = keys[c];
+      const int n = npad[c];
+      if (T.sim_base && n * 8 <= T.sim_cap * 16) {
+        u64* sm = (u64*)__cvta_shared_to_generic((size_t)T.sim_base);
+        for (int x = lane; x < n; x += 32) sm[x] = srt[x];
+        __syncwarp();
+        warp_sort_u64(sm, n, lane);
+        for (int x = lane; x < n; x += 32) srt[x] = sm[x];
+        __syncwarp();
+      } else warp_sort_u64(srt, n, lane);
+      i64 run = base_c[c];                               // f_c at the start of the block of 32
+      for (int x0 = 0; x0 <= Uc; x0 += 32) {
+        // f_c(x0 + lane) = run - gains of the steps x0 .. x0+lane-1 (an exclusive scan)
+        const int x = x0 + lane;
+        i64 gsum = (x >= 1 && x <= Uc) ? mg_gain(srt[x - 1]) : 0;   // lane holds the gain of step x-1
+        if (x0 > 0 && lane == 0) gsum = 0;               // step x0-1 went into `run` already
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const i64 y = __shfl_up_sync(TG_FULL, gsum, o); if (lane >= o) gsum += y; }
+        if (x <= Uc) f[c][x] = run - gsum;
+        // carry: f_c(x0 + 32) needs the gain of step x0+31 as well
+        const i64 tail = (x0 + 32 <= Uc) ? mg_gain(srt[x0 + 31]) : 0;
+        run = run - __shfl_sync(TG_FULL, gsum, 31) - tail;
+      }
+      __syncwarp();
+      continue;
+    }
+    i64* prev = work; i64* cur = work + (Umax + 1);
     for (int u = lane; u <= Uc; u += 32) prev[u] = u == 0 ? 0 : TG_INF;
     __syncwarp();
     int tc = 0;
@@ -495,6 +616,28 @@ __device__ __noinline__ int dp_classes(const PoolTask& T, int nrows, const int Y
   for (int c = 0; c < 4; ++c) {
     int u = c < 3 ? cell[c] - 2 * cell[c + 1] : cell[3];
     const int Uc = U[c];
+    if (by_gain[c]) {
+      // the x steps in front of the sorted order are taken: a row gets its steps up to the threshold key
+      const u64 thr = u >= 1 ? keys[c][u - 1] : 0ull;
+      for (int t = lane; t < nrows; t += 32) {
+        const int i = T.rowcand[t];
+        if (ilog2(T.cg[i] & 0x7f) != c) continue;
+        const u32 mk = T.cmask[i];
+        const int r0 = __ffs(mk), ex = (32 - __clz(mk)) - r0;
+        const i64 s = T.cs[i], p = T.cp[i];
+        int take = 0;
+        if (u >= 1) {
+          i64 before = duration(s, p, r0);
+          for (int k = 1; k <= ex; ++k) {
+            const i64 now = duration(s, p, r0 + k);
+            if (mg_key(before - now, t, k) > thr) break;  // a row's keys ascend with the step
+            take = k; before = now;
+          }
+        }
+        T.rsel[i] = (u8)(r0 + take);
+      }
+      continue;
+    }
     int tc = rows_c[c];
     if (lane == 0) {
       for (int t = nrows - 1; t >= 0; --t) {
