@@ -2,7 +2,8 @@
 import numpy as np
 import pytest
 
-from workloads import POOL_API, POOL_CPU, POOL_GPU, Pool, generate, make_workload, random_round
+from workloads import (POOL_API, POOL_CPU, POOL_GPU, Pool, contiguous_replica_round, generate, make_workload,
+                       random_round)
 
 pytestmark = pytest.mark.gpu
 
@@ -187,3 +188,17 @@ def test_fragmented_pool_with_elastic_gang_requests_matches_oracle(oracle, seed,
     g = gpu_round(pools, a)
     assert_same(o, g)
     assert np.all(g["status"] == 0) and o["n_selected"].max() > 30
+
+
+@pytest.mark.parametrize("seed,nodes,N,max_mult,tiny", [(0, 128, 800, 8, 0.0), (1, 160, 1000, 12, 0.3),
+                                                         (2, 64, 500, 16, 0.0), (3, 96, 600, 31, 0.7)])
+def test_marginal_gain_classes_match_oracle(oracle, seed, nodes, N, max_mult, tiny):
+    # hundreds of candidates with contiguous multiplicities on a fragmented pool: the chunk-size classes
+    # are served from their sorted marginal gains (more than 512 steps in a class: sorted in global
+    # memory); tiny durations break the monotony of some rows' gains, whose classes keep their DP
+    w, a = contiguous_replica_round(7300 + seed, 5, N, nodes, max_mult, small_durations=tiny)
+    for depth in (2, 1):
+        o = oracle.schedule_batch(w.pools, a, depth=depth)
+        g = gpu_round(w.pools, a, depth=depth)
+        assert_same(o, g)
+    assert np.all(g["status"] == 0) and o["n_selected"].max() > 80

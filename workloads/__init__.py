@@ -21,4 +21,5 @@ from .generator import (  # noqa: F401
     make_workload,
     generate,
     random_round,
+    contiguous_replica_round,
 )

@@ -356,3 +356,27 @@ def random_round(seed: int, n_scenarios: int, max_actions: int, pools: Tuple[Poo
     for k in ("pool", "unit", "level_mask", "s_us", "p_us"):
         a[k] = np.ascontiguousarray(a[k])
     return w, a
+
+
+def contiguous_replica_round(seed: int, n_scenarios: int, max_actions: int, nodes: int, max_mult: int,
+                             *, small_durations: float = 0.0, busy_fraction: float = 0.3
+                             ) -> Tuple[Workload, Dict[str, Optional[np.ndarray]]]:
+    """Rounds on one fragmented GPU pool whose actions all ask for replicas (chunks of 1, 2, 4 or 8
+    GPUs with the probabilities of config 3) with CONTIGUOUS multiplicities lo..hi, hi up to
+    max_mult: many candidates with many upgrade steps each.  Tiny durations make the floor of the
+    duration model break the monotony of the gains and produce ties."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    S, N = n_scenarios, max_actions
+    pools = (Pool(POOL_GPU, 8 * nodes, 8),)
+    w = Workload(f"contig{seed}", S, N, pools, "random", base_seed=seed, params=dict(busy_fraction=busy_fraction))
+    unit = (1 << rng.choice(4, size=(S, N), p=[0.4, 0.3, 0.2, 0.1])).astype(np.uint8)
+    hi = rng.integers(1, max_mult + 1, size=(S, N))
+    lo = np.where(rng.random((S, N)) < 0.8, 1, np.minimum(2, hi))
+    mask = (((np.int64(1) << hi) - 1) & ~((np.int64(1) << (lo - 1)) - 1)).astype(np.uint32)
+    tiny = rng.random((S, N)) < small_durations
+    s = np.where(tiny, rng.integers(0, 4, (S, N)), rng.integers(0, 50_000, (S, N))).astype(np.int64)
+    p = np.where(tiny, rng.integers(0, 40, (S, N)), rng.integers(0, 500_000, (S, N))).astype(np.int64)
+    a = dict(pool=np.zeros((S, N), np.uint8), unit=unit, level_mask=mask, s_us=s, p_us=p, arrival_us=None,
+             n_actions=np.full(S, N, np.int32))
+    a["gpu_busy"] = _busy_masks(w, 0, S)
+    return w, a
