@@ -654,6 +654,182 @@ __device__ __noinline__ int dp_classes(const PoolTask& T, int nrows, const int Y
   return 1;
 }
 
+// The box DP on the REACHABLE cells only, for boxes whose dense table would not fit: Algorithm 4's
+// state space is the product of the four chunk-count ranges, but a row only moves a state by one of
+// a handful of demand vectors, so few cells are ever reached.  A state is the extra-demand vector
+// packed into one key (one bit field per kept dimension); the states of a row are built from those
+// of the row before through a hash table (open addressing; a cell keeps the least
+// duration sum << 6 | multiplicity, i.e. the lowest value and among equals the smallest level,
+// which is what the dense loop's ascending levels with strict '<' keep), compacted into the next
+// list, and their (key, multiplicity) pairs are kept per row for the walk back.  Same end-cell rule
+// as the dense loop: lowest value, then fewest extra units, then the allocations compared from the
+// last row down.  Everything lives in [mem, mem + bytes).  Returns 1 (T.rsel written), 0 if the
+// memory does not suffice or a value outgrows its field.
+#define SP_EMPTY 0xffffffffffffffffull
+__device__ __forceinline__ u64 sp_hash(u64 k) { k ^= k >> 29; k *= 0xbf58476d1ce4e5b9ull; k ^= k >> 32; return k; }
+__device__ __noinline__ int dp_sparse(const PoolTask& T, int nrows, const int ext[4], const bool kept[4],
+                                      char* mem, u64 bytes, int lane) {
+  // bit fields of a key
+  int shift[4], width[4], total_bits = 0;
+#pragma unroll
+  for (int l = 0; l < 4; ++l) {
+    width[l] = kept[l] ? 32 - __clz(max(ext[l] - 1, 1)) : 0;
+    shift[l] = total_bits; total_bits += width[l];
+  }
+  if (total_bits > 60) return 0;
+  // memory: two state lists and the hash table at the end, the rows' (key, multiplicity) pairs from the front
+  const u64 cap_states = bytes / 2 / (2 * 16 + 4 * 16);          // each list 16 B per state, table 4 slots of 16 B per state
+  if (cap_states < 64) return 0;
+  u64* lk[2]; i64* lv[2];
+  char* top = mem + bytes;
+  u64 tab_slots = 1; while (tab_slots < 4 * cap_states) tab_slots <<= 1; tab_slots >>= 1;   // largest power of two <= 4 cap
+  top -= tab_slots * 16; u64* tk = (u64*)top; u64* tv = tk + tab_slots;
+  for (int x = 0; x < 2; ++x) { top -= cap_states * 16; lk[x] = (u64*)top; lv[x] = (i64*)(lk[x] + cap_states); }
+  char* store = mem;                                             // grows towards `top`
+  // per row: where its pairs start and how many (kept in the store itself, in front of the pairs)
+  u64* row_dir = (u64*)store; store += (u64)nrows * 16;
+  if (store > top) return 0;
+  u64 n = 1;
+  if (lane == 0) { lk[0][0] = 0; lv[0][0] = 0; }
+  __syncwarp();
+  int cur = 0;
+  for (int t = 0; t < nrows; ++t) {
+    const int i = T.rowcand[t];
+    const int g = T.cg[i] & 0x7f, gang = T.cg[i] >> 7;
+    const u32 mk = T.cmask[i];
+    const int r0 = __ffs(mk), nlev = __popc(mk);
+    const i64 s = T.cs[i], p = T.cp[i];
+    // table of this row: a power of two of at least four slots per candidate state
+    u64 want = n * (u64)nlev * 2, slots = 64;
+    while (slots < want && slots < tab_slots) slots <<= 1;
+    for (u64 x = lane; x < slots; x += 32) { tk[x] = SP_EMPTY; tv[x] = ~0ull; }
+    __syncwarp();
+    u64 distinct = 0;
+    bool fail = false;
+    for (u64 x0 = 0; x0 < n; x0 += 32) {
+      const u64 x = x0 + lane;
+      const bool on = x < n;
+      const u64 key = on ? lk[cur][x] : 0;
+      const i64 val = on ? lv[cur][x] : 0;
+      u32 mm = mk;
+      while (mm) {
+        const int r = __ffs(mm); mm &= mm - 1;
+        int d[4];
+        extra_demand(T.type, g, gang, r0, r, d);
+        u64 nk = key; bool inside = on;
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+          if (kept[l]) {
+            const int dl = d[l] >> l;
+            const int e = (int)((key >> shift[l]) & ((1ull << width[l]) - 1ull));
+            inside &= e + dl < ext[l];
+            nk += (u64)dl << shift[l];
+          }
+        const i64 cand = val + duration(s, p, r);
+        if (inside && cand >= (1ll << 56)) { fail = true; inside = false; }
+        if (inside) {
+          const u64 packed = ((u64)cand << 6) | (u64)r;
+          u64 h = sp_hash(nk) & (slots - 1);
+          for (u64 probe = 0; probe < slots; ++probe) {
+            const u64 seen = atomicCAS((unsigned long long*)&tk[h], SP_EMPTY, nk);
+            if (seen == SP_EMPTY || seen == nk) { atomicMin((unsigned long long*)&tv[h], packed); if (seen == SP_EMPTY) ++distinct; break; }
+            h = (h + 1) & (slots - 1);
+            if (probe + 1 == slots) fail = true;
+          }
+        }
+      }
+    }
+    __syncwarp();
+    distinct = (u64)warp_sum64((i64)distinct);
+    if (__any_sync(TG_FULL, fail) || distinct > cap_states || distinct > slots / 2 + 32) return 0;
+    // compact the table into the next list and into the row's store
+    if (store + distinct * 16 > top) return 0;
+    u64* sk = (u64*)store; u64* sr = sk + distinct;
+    if (lane == 0) { row_dir[2 * t] = (u64)(store - mem); row_dir[2 * t + 1] = distinct; }
+    store += distinct * 16;
+    u64 filled = 0;
+    for (u64 x0 = 0; x0 < slots; x0 += 32) {
+      const u64 x = x0 + lane;
+      const u64 k = tk[x];
+      const bool has = k != SP_EMPTY;
+      const u32 b = __ballot_sync(TG_FULL, has);
+      if (has) {
+        const u64 at = filled + __popc(b & ((1u << lane) - 1u));
+        const u64 pv = tv[x];
+        lk[cur ^ 1][at] = k; lv[cur ^ 1][at] = (i64)(pv >> 6);
+        sk[at] = k; sr[at] = pv & 63ull;
+      }
+      filled += __popc(b);
+    }
+    __syncwarp();
+    n = distinct; cur ^= 1;
+  }
+  // best end state: lowest value, then fewest extra units (dimension 0)
+  const u64 m0 = (1ull << width[0]) - 1ull;
+  i64 bv = TG_INF;
+  for (u64 x = lane; x < n; x += 32) bv = min(bv, lv[cur][x]);
+  bv = warp_min64(bv);
+  if (bv == TG_INF) return 0;
+  int be = INT_MAX;
+  for (u64 x = lane; x < n; x += 32) if (lv[cur][x] == bv) be = min(be, (int)((lk[cur][x] >> shift[0]) & m0));
+  be = warp_min32(be);
+  // the tied end states walk back together; at each row (last first) those with the smallest multiplicity stay
+  const int TIE_CAP = 32;
+  u64 tied = SP_EMPTY;                                     // lane x holds the x-th tied key
+  int nt = 0;
+  for (u64 x0 = 0; x0 < n; x0 += 32) {
+    const u64 x = x0 + lane;
+    const bool hit = x < n && lv[cur][x] == bv && (int)((lk[cur][x] >> shift[0]) & m0) == be;
+    const u32 b = __ballot_sync(TG_FULL, hit);
+    if (nt + __popc(b) > TIE_CAP) return 0;
+    // hand the hits to lanes nt, nt+1, ...
+    for (u32 bb = b; bb; bb &= bb - 1) {
+      const int src = __ffs(bb) - 1;
+      const u64 k = __shfl_sync(TG_FULL, hit ? lk[cur][x] : 0ull, src);
+      if (lane == nt) tied = k;
+      ++nt;
+    }
+  }
+  for (int t = nrows - 1; t >= 0; --t) {
+    const int i = T.rowcand[t];
+    const u64* sk = (const u64*)(mem + row_dir[2 * t]);
+    const u64 cnt = row_dir[2 * t + 1];
+    const u64* sr = sk + cnt;
+    // every tied key looks up its multiplicity in this row (all lanes scan for one key at a time)
+    int myr = 255;
+    for (int y = 0; y < nt; ++y) {
+      const u64 k = __shfl_sync(TG_FULL, tied, y);
+      int found = 255;
+      for (u64 x = lane; x < cnt; x += 32) if (sk[x] == k) found = (int)sr[x];
+      found = warp_min32(found);
+      if (lane == y) myr = found;
+    }
+    const int rm = warp_min32(lane < nt ? myr : 255);
+    if (rm == 255) return 0;                               // cannot happen: every kept key was written by this row
+    if (lane == 0) T.rsel[i] = (u8)rm;
+    int d[4];
+    extra_demand(T.type, T.cg[i] & 0x7f, T.cg[i] >> 7, __ffs(T.cmask[i]), rm, d);
+    u64 delta = 0;
+#pragma unroll
+    for (int l = 0; l < 4; ++l) if (kept[l]) delta += (u64)(d[l] >> l) << shift[l];
+    // keep the keys whose multiplicity is the smallest, move them to the row before, drop duplicates
+    const bool stay = lane < nt && myr == rm;
+    const u64 prevk = tied - delta;
+    const u32 sb = __ballot_sync(TG_FULL, stay);
+    u64 next = SP_EMPTY;
+    int nn = 0;
+    for (u32 bb = sb; bb; bb &= bb - 1) {
+      const int src = __ffs(bb) - 1;
+      const u64 k = __shfl_sync(TG_FULL, prevk, src);
+      const bool dup = __any_sync(TG_FULL, lane < nn && next == k);
+      if (!dup) { if (lane == nn) next = k; ++nn; }
+    }
+    tied = next; nt = nn;
+  }
+  __syncwarp();
+  return 1;
+}
+
 // Optimal allocation of candidates [0, q) -> T.rsel[0..q), duration sum -> *opt.
 // *all_best tells that every candidate got its best level (then so does every shorter prefix).
 // Returns false if the workspace is too small.
@@ -740,7 +916,7 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
     *opt = warp_sum64(sum);
     return true;
   }
-  if (cells > (1ull << 30)) return false;
+  if (cells > (1ull << 30)) cells = (1ull << 30) + 1;       // (never dense: the reachable cells only, below)
   const int ncell = (int)cells;
   if (ncell <= 32 && T.sim_base && nrows * 4 <= T.sim_cap &&
       dp_small(T, nrows, ncell, ext, stride, kept, T.sim_base, lane)) {
@@ -751,12 +927,18 @@ __device__ bool solve_prefix(const Params& P, const PoolTask& T, int q, Slab sla
   }
   i64* val = (i64*)slab.take(2 * cells * sizeof(i64));
   u8* choice = val ? (u8*)slab.take((u64)nrows * cells) : nullptr;
-  int slot = -1;
+  const int slot = -1;
   if (!choice) {
-    slot = slot_acquire(P, 2 * cells * sizeof(i64) + (u64)nrows * cells, lane);
-    if (slot < 0) return false;
-    char* big = slot_ptr(P, slot);
-    val = (i64*)big; choice = (u8*)(big + 2 * cells * sizeof(i64));
+    // the dense table does not fit the warp's slab: only the reachable cells, in a borrowed slot of the arena
+    const int sl = slot_acquire(P, 1, lane);
+    if (sl < 0) return false;
+    const int done = dp_sparse(PoolTask(T), nrows, ext, kept, slot_ptr(P, sl), arena_slot_bytes(P), lane);
+    slot_release(P, sl, lane);
+    if (!done) return false;
+    i64 sum = 0;
+    for (int i = lane; i < q; i += 32) sum += duration(T.cs[i], T.cp[i], T.rsel[i]);
+    *opt = warp_sum64(sum);
+    return true;
   }
   i64* prev = val; i64* cur = val + cells;
   for (int c = lane; c < ncell; c += 32) prev[c] = c == 0 ? 0 : TG_INF;

@@ -202,3 +202,18 @@ def test_marginal_gain_classes_match_oracle(oracle, seed, nodes, N, max_mult, ti
         g = gpu_round(w.pools, a, depth=depth)
         assert_same(o, g)
     assert np.all(g["status"] == 0) and o["n_selected"].max() > 80
+
+
+@pytest.mark.parametrize("seed,nodes,N", [(0, 32, 24), (2, 64, 36), (3, 64, 48), (4, 128, 64)])
+def test_gang_requests_with_a_large_feasible_box_match_oracle(oracle, seed, nodes, N):
+    # short queues on a large fragmented pool: every action is a candidate, there is far more room than
+    # the least levels need but not enough for everybody's best level, and gang requests couple the
+    # chunk sizes: the dense table over the four chunk-count ranges has millions of cells, of which
+    # the rows reach a few thousand (Algorithm 4 on the reachable states only)
+    pools = (Pool(POOL_GPU, 8 * nodes, 8),)
+    w, a = random_round(6200 + seed, 6, N, pools, replicas=0.5, busy_fraction=0.35, inelastic=0.1, max_mult=8,
+                        ragged=False)
+    o = oracle.schedule_batch(pools, a)
+    g = gpu_round(pools, a)
+    assert_same(o, g)
+    assert np.all(g["status"] == 0) and o["n_selected"].min() >= N - 2
