@@ -85,8 +85,10 @@ typedef struct {
                            copies and kernels overlap; ordered after the work queued on the
                            given stream, which in turn waits for the results; use pinned
                            memory)                                                         */
-  int64_t workspace_bytes; /* scratch for large DP tables; 0 = default (8 GiB): 7/8 of it
-                              are 48 reusable slots (a DP table must fit one), the rest is bump-allocated             */
+  int64_t workspace_bytes; /* scratch for the rare large tables (reachable-state DP of fragmented GPU
+                              pools with gang requests, simulations beyond shared memory);
+                              0 = default (2 GiB): 7/8 of it are up to 48 reusable slots of at
+                              least 64 MiB (such a table must fit one), the rest is bump-allocated */
   const tangram_pool_desc* pools; /* host array of n_pools entries, copied                 */
 } tangram_round_desc;
 

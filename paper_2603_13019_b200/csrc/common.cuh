@@ -28,7 +28,8 @@ struct PoolDev {
 
 // per (scenario, pool) facts produced by the prefix kernel
 struct PoolMeta {
-  i64 base;       // the pool's positions in the partitioned arrays start at scenario * max_actions + base
+  i64 base;       // the pool's list in `tmin` starts at scenario * max_actions + base
+  i64 cbase;      // the pool's candidates in order / preq / the solver's arrays start at scenario * max_actions + cbase
   int count;      // actions of the pool in the queue (candidates only, if nobody will read its waiting list)
   int m;          // candidates of the pool (they occupy positions base .. base+m-1)
   int elastic;    // some candidate has more than one level
@@ -39,6 +40,9 @@ struct Params {
   int S, N, P, depth, n_nodes_total, V;
   PoolDev pool[TG_MAX_POOLS];
   int pool_order[TG_MAX_POOLS];   // pools in the order their tasks are handed out (longest tasks first)
+  // candidate arrays of the batched path: a pool has at most min(max_actions, capacity) candidates (each
+  // takes a unit at least), so a scenario's rows are cand_off[j] .. cand_off[j+1] of cand_stride entries
+  int cand_off[TG_MAX_POOLS + 1]; int cand_stride;
   i64 now;
   // inputs (device)
   const u8* a_pool; const u8* a_unit; const u32* a_mask;

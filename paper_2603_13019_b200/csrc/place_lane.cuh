@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ P
   const int maxkeep = warp_max32(keep);
   if (maxkeep == 0) return;
   const size_t row = (size_t)(sc < P.S ? sc : 0) * P.N;
-  const i64 base = sc < P.S ? P.meta[(size_t)sc * P.P + j].base : 0;
+  const i64 base = sc < P.S ? P.meta[(size_t)sc * P.P + j].cbase : 0;
   const unsigned short* rq = P.preq + row + base;
   const int* ord = P.order + row + base;
   u8* st = W.state + lane;

@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(K1_THREADS) k_prefix(const __grid_constant__ P
   }
   if (t < P.P) {
     PoolMeta mt;
-    mt.base = s_base[t]; mt.count = bad ? 0 : s_tot[t]; mt.m = bad ? 0 : s_m[t];
+    mt.base = s_base[t]; mt.cbase = s_base[t]; mt.count = bad ? 0 : s_tot[t]; mt.m = bad ? 0 : s_m[t];
     mt.elastic = (s_el >> t) & 1;
     // waiting actions of a pool whose selection runs recorded their index behind the candidates
     mt.first_wait = (!bad && mt.elastic && mt.count > mt.m) ? P.order[row + s_base[t] + s_m[t]] : -1;

@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
       if (lane == jj) { cnt += __popc(b); mreg += __popc(b & below_f); }
     }
     if (cand) {
-      P.order[prow + (size_t)j * P.N + pos] = i;
+      P.order[(size_t)sc * P.cand_stride + P.cand_off[j] + pos] = i;
       if (eff & (eff - 1)) el |= 1u << j;
     }
     for (int v = 0; v < D; ++v) {
@@ -169,6 +169,7 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
   if (lane < P.P) {
     PoolMeta mt;
     mt.base = (i64)sc * (P.P - 1) * P.N + (i64)lane * P.N;   // row + base = prow + lane * N
+    mt.cbase = (i64)sc * (P.cand_stride - P.N) + P.cand_off[lane];   // row + cbase = sc * cand_stride + cand_off
     // an invalid record among the actions seen here: nothing of the scenario is decided
     mt.count = anybad ? 0 : cnt; mt.m = anybad ? 0 : mreg; mt.elastic = anybad ? 0 : ((elw >> lane) & 1u);
     mt.first_wait = anybad ? -1 : fwreg;

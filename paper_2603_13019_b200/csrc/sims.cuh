@@ -87,14 +87,14 @@ __device__ __forceinline__ SimJob sim_job(const Params& P, TaskState* ts, const 
   const PoolDev& pd = P.pool[j];
   // first remaining action: the evicted last candidate (e = 1) or the first waiting one; it takes
   // the largest of its first `depth` levels (see the header for why that depth is the best)
-  const int idx = e ? P.order[row + mt.base + mt.m - 1] : mt.first_wait;
+  const int idx = e ? P.order[row + mt.cbase + mt.m - 1] : mt.first_wait;
   int g, gang; u32 fm;
   decode_levels(pd, P.a_unit[row + idx], P.a_mask[row + idx], g, gang, fm);
   const int d = min(P.depth, __popc(fm)) - 1;
   J.active = true;
   J.first_dur = duration(clamp_param(P.a_s[row + idx]), clamp_param(P.a_p[row + idx]), nth_level_of(fm, d));
   J.H = mt.m - e;
-  J.seeds = (e ? seed2 : P.tmin) + row + mt.base;
+  J.seeds = e ? seed2 + row + mt.cbase : P.tmin + row + mt.base;
   J.lst = P.tmin + row + mt.base + mt.m + (1 - e);
   J.n_list = n_ac - (1 - e);
   return J;

@@ -70,7 +70,7 @@ __device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta
   for (int i0 = lane; i0 < m; i0 += 128) {
     int idx[4]; u8 un[4]; u32 mk[4]; i64 sv[4], pv[4];
 #pragma unroll
-    for (int x = 0; x < 4; ++x) idx[x] = i0 + 32 * x < m ? P.order[row + mt.base + i0 + 32 * x] : 0;
+    for (int x = 0; x < 4; ++x) idx[x] = i0 + 32 * x < m ? P.order[row + mt.cbase + i0 + 32 * x] : 0;
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
       const bool on = i0 + 32 * x < m;
@@ -153,7 +153,7 @@ __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& 
   defer = defer && pd.lane_place;
   if (defer) {
     // k_place will place this pool: leave it the kept requests in queue order
-    unsigned short* rq = P.preq + row + mt.base;
+    unsigned short* rq = P.preq + row + mt.cbase;
     for (int i = lane; i < keep; i += 32) rq[i] = (unsigned short)(C.cg[i] | ((u32)C.rkeep[i] << 8));
     if (lane == 0) P.keepn[(size_t)sc * P.P + j] = keep;
   } else if (pd.type == TG_POOL_GPU) {
@@ -254,8 +254,8 @@ __global__ void __launch_bounds__(256) k_easy(const __grid_constant__ Params P, 
   if (lane == 0) P.keepn[task] = m;
   if (m == 0) return;
   const size_t row = (size_t)sc * P.N;
-  const int* ord = P.order + row + mt.base;
-  unsigned short* rq = P.preq + row + mt.base;
+  const int* ord = P.order + row + mt.cbase;
+  unsigned short* rq = P.preq + row + mt.cbase;
   i64 tot = 0; int cnt = 0;
   for (int i = lane; i < m; i += 32) {
     const size_t o = row + ord[i];
@@ -278,9 +278,9 @@ __global__ void __launch_bounds__(256) k_easy(const __grid_constant__ Params P, 
 // workspace of the batched path, indexed like the partitioned arrays
 struct BatchWs {
   TaskState* ts;   // [S][P]
-  i64* seed2;      // [S][N] durations of the first m-1 candidates under their optimal allocation
-  u8* rs1;         // [S][N] multiplicities of the optimal allocation of all m candidates
-  u8* rs2;         // [S][N] ... of the first m-1
+  i64* seed2;      // [S][cand_stride] durations of the first m-1 candidates under their optimal allocation
+  u8* rs1;         // [S][cand_stride] multiplicities of the optimal allocation of all m candidates
+  u8* rs2;         // [S][cand_stride] ... of the first m-1
 };
 
 __global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__ Params P, const BatchWs W, const HeadState* hst) {
@@ -322,13 +322,13 @@ __global__ void __launch_bounds__(K2_THREADS, 3) k_solve(const __grid_constant__
           ok = solve_prefix(P, T, mt.m - 1, slab, lane, &opt1);
           if (ok && !eviction_cannot_pay(T, mt.m - 1, C.rkeep, C.rsel, lane)) {
             decided = false;
-            const size_t pos = (size_t)sc * P.N + mt.base;
+            const size_t pos = (size_t)sc * P.N + mt.base, cpos = (size_t)sc * P.N + mt.cbase;
             for (int i = lane; i < mt.m; i += 32) {
-              W.rs1[pos + i] = C.rkeep[i];
+              W.rs1[cpos + i] = C.rkeep[i];
               P.tmin[pos + i] = duration(C.cs[i], C.cp[i], C.rkeep[i]);   // heap seeds of the full list
               if (i < mt.m - 1) {
-                W.rs2[pos + i] = C.rsel[i];
-                W.seed2[pos + i] = duration(C.cs[i], C.cp[i], C.rsel[i]);
+                W.rs2[cpos + i] = C.rsel[i];
+                W.seed2[cpos + i] = duration(C.cs[i], C.cp[i], C.rsel[i]);
               }
             }
             if (lane == 0) {
@@ -364,7 +364,7 @@ __device__ void finish_task(const Params& P, const BatchWs& W, int x, int gw, in
   int keep = mt.m;
   if (!(st.flags & TS_SOLVED) || (st.flags & TS_FAILED)) keep = -1;
   else {
-    const size_t pos = (size_t)sc * P.N + mt.base;
+    const size_t pos = (size_t)sc * P.N + mt.cbase;
     i64 obj = sat_add(st.opt[0], st.est[0]);
     for (int i = lane; i < mt.m; i += 32) C.rkeep[i] = W.rs1[pos + i];
     i64 nobj = sat_add(st.opt[1], st.est[1]);
@@ -581,6 +581,10 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.n_nodes_total = node0;
   P.V = slot0 + desc->n_pools;
   fill_pool_order(P);
+  P.cand_off[0] = 0;
+  for (int j = 0; j < desc->n_pools; ++j)
+    P.cand_off[j + 1] = P.cand_off[j] + (int)align_up((size_t)(P.pool[j].capacity < P.N ? P.pool[j].capacity : P.N), 8);
+  P.cand_stride = P.cand_off[desc->n_pools];
 
   cudaError_t e = cudaGetDevice(&r->device);
   cudaDeviceProp prop;
@@ -588,17 +592,17 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   if (e == cudaSuccess) e = fill_tables();
   if (e != cudaSuccess) { delete r; return cuda_fail(e, "device set-up"); }
 
-  const size_t SN = (size_t)P.S * P.N;
-  P.n_workers = prop.multiProcessorCount * 4 * (K2_THREADS / 32);
+  const size_t SN = (size_t)P.S * P.N, SC = (size_t)P.S * P.cand_stride;
+  P.n_workers = prop.multiProcessorCount * 3 * (K2_THREADS / 32);   // what k_solve keeps resident
   if ((int64_t)P.n_workers > (int64_t)P.S * P.P) P.n_workers = (int)align_up((size_t)P.S * P.P, K2_THREADS / 32);
   // every worker warp owns a slab that holds the candidate arrays, heaps and small DP tables of
   // the pool it is working on; larger DP tables come from the shared arena
   size_t per_cand = 8 + 8 + 4 + 4 + 4 + 4 + 4 + 3 + 16 * (size_t)desc->depth;
   size_t slab = align_up((size_t)P.N * per_cand + 64 * 1024 + (1 << 20) / 4 + 4096, 256);
   P.slab_bytes = slab;
-  P.arena_bytes = desc->workspace_bytes ? (u64)desc->workspace_bytes : (8ull << 30);
+  P.arena_bytes = desc->workspace_bytes ? (u64)desc->workspace_bytes : (2ull << 30);
   bool bad = false;
-  bad |= cudaMalloc(&r->d_order, SN * sizeof(int) * P.P) != cudaSuccess;
+  bad |= cudaMalloc(&r->d_order, SC * sizeof(int)) != cudaSuccess;
   bad |= cudaMalloc(&r->d_tmin, SN * sizeof(i64) * P.P) != cudaSuccess;
   bad |= cudaMalloc(&r->d_meta, (size_t)P.S * P.P * sizeof(PoolMeta)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->hst, (size_t)P.S * sizeof(HeadState)) != cudaSuccess;
@@ -606,10 +610,10 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc(&r->d_arena, P.arena_bytes) != cudaSuccess;
   bad |= cudaMalloc(&r->d_arena_top, 256) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->W.ts, (size_t)P.S * P.P * sizeof(TaskState)) != cudaSuccess;
-  bad |= cudaMalloc((void**)&r->W.seed2, SN * sizeof(i64) * P.P) != cudaSuccess;
-  bad |= cudaMalloc((void**)&r->W.rs1, SN * P.P) != cudaSuccess;
-  bad |= cudaMalloc((void**)&r->W.rs2, SN * P.P) != cudaSuccess;
-  bad |= cudaMalloc((void**)&r->d_preq, SN * P.P * sizeof(unsigned short)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.seed2, SC * sizeof(i64)) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.rs1, SC) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->W.rs2, SC) != cudaSuccess;
+  bad |= cudaMalloc((void**)&r->d_preq, SC * sizeof(unsigned short)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->d_keepn, (size_t)P.S * P.P * sizeof(int)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->d_fl, ((size_t)P.S * P.P + 2) * sizeof(int)) != cudaSuccess;
   const long long n_sims = (long long)P.P * P.S * 2;
