@@ -89,6 +89,10 @@ typedef struct {
                               pools with gang requests, simulations beyond shared memory);
                               0 = default (2 GiB): 7/8 of it are up to 48 reusable slots of at
                               least 64 MiB (such a table must fit one), the rest is bump-allocated */
+  int64_t slot_wait_us;    /* how long a warp that needs one of those slots waits for another warp to
+                              give one back before it gives up (the scenario then gets
+                              TANGRAM_STATUS_WORKSPACE); 0 = default (100 ms).  The holders of the
+                              slots never wait for anything, so a waiter cannot block them.        */
   const tangram_pool_desc* pools; /* host array of n_pools entries, copied                 */
 } tangram_round_desc;
 

@@ -30,7 +30,8 @@ class _PoolDesc(C.Structure):
 class _RoundDesc(C.Structure):
     _fields_ = [("n_scenarios", C.c_int32), ("max_actions", C.c_int32), ("n_pools", C.c_int32),
                 ("depth", C.c_int32), ("round_us", C.c_int64), ("max_rounds", C.c_int32),
-                ("host_buffers", C.c_int32), ("workspace_bytes", C.c_int64), ("pools", C.POINTER(_PoolDesc))]
+                ("host_buffers", C.c_int32), ("workspace_bytes", C.c_int64), ("slot_wait_us", C.c_int64),
+                ("pools", C.POINTER(_PoolDesc))]
 
 
 class _Actions(C.Structure):
@@ -119,14 +120,14 @@ class Round:
 
     def __init__(self, n_scenarios: int, max_actions: int, pools: Sequence, *, depth: int = 2,
                  round_us: int = 10_000, max_rounds: int = 0, host_buffers: bool = False,
-                 workspace_bytes: int = 0):
+                 workspace_bytes: int = 0, slot_wait_us: int = 0):
         self._lib = load_library()
         self._h = None
         self.n_scenarios, self.max_actions, self.pools = int(n_scenarios), int(max_actions), tuple(pools)
         self.max_rounds, self.host_buffers = int(max_rounds), bool(host_buffers)
         arr = (_PoolDesc * len(pools))(*[_PoolDesc(p.type, p.capacity, p.group, p.window_us) for p in pools])
         desc = _RoundDesc(n_scenarios, max_actions, len(pools), depth, round_us, max_rounds,
-                          1 if host_buffers else 0, workspace_bytes, arr)
+                          1 if host_buffers else 0, workspace_bytes, slot_wait_us, arr)
         h = C.c_void_p()
         _check(self._lib.tangram_round_create(C.byref(desc), C.byref(h)))
         self._h = h
@@ -264,7 +265,7 @@ def schedule_batch_static(pools: Sequence, actions: Dict, result: Dict, *, depth
     ins, outs = _dtypes()
     S, N = actions["pool"].shape
     arr = (_PoolDesc * len(pools))(*[_PoolDesc(p.type, p.capacity, p.group, p.window_us) for p in pools])
-    desc = _RoundDesc(S, N, len(pools), depth, 0, 0, 0, 0, arr)
+    desc = _RoundDesc(S, N, len(pools), depth, 0, 0, 0, 0, 0, arr)
 
     def ptr(t):
         return None if t is None else t.data_ptr()

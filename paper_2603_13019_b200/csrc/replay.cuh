@@ -113,7 +113,8 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
   C.cg = (u8*)slab.take(m); C.rsel = (u8*)slab.take(m); C.rkeep = (u8*)slab.take(m);
   i64* ac_tmin = (i64*)slab.take((u64)(n_ac + 1) * 8);
   i64* seeds = (i64*)slab.take((u64)(nr + 1) * 8);
-  if (!seeds) return false;
+  if (!C.cs || !C.cp || !C.cmask || !C.cidx || !C.pnode || !C.poff || !C.rowcand || !C.cg || !C.rsel || !C.rkeep ||
+      !ac_tmin || !seeds) return false;
   // fill them in queue order
   int cm = 0, ca = 0, first_ac = -1;
   bool elastic = false;

@@ -55,7 +55,7 @@ __device__ __forceinline__ int slot_acquire(const Params& P, u64 bytes, int lane
     int* flags = (int*)(P.arena_top + 8);
     const int ns = arena_n_slots(P);
     const int start = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5) % ns;
-    for (int tries = 0; tries < 2000000 && got < 0; ++tries) {   // gives up after some seconds
+    for (int tries = 0; tries < P.slot_tries && got < 0; ++tries) {   // gives up after the round's slot_wait_us
       for (int k = 0; k < ns && got < 0; ++k) {
         const int s = (start + k) % ns;
         if (atomicCAS(&flags[s], 0, 1) == 0) got = s;

@@ -64,7 +64,7 @@ __device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta
   C.cidx = (int*)slab.take((u64)m * 4);
   C.pnode = (int*)slab.take((u64)m * 4);
   C.poff = (int*)slab.take((u64)m * 4);
-  if (!C.cg || !C.rkeep || !C.rsel || !C.cmask || !C.rowcand || !C.cp || !C.cs || !C.poff) return false;
+  if (!C.cg || !C.rkeep || !C.rsel || !C.cmask || !C.rowcand || !C.cp || !C.cs || !C.cidx || !C.pnode || !C.poff) return false;
   // four candidates per lane at a time: first all their indices, then all their records, so that a
   // pool of up to 128 candidates costs two rounds of loads instead of two per 32 candidates
   for (int i0 = lane; i0 < m; i0 += 128) {
@@ -549,7 +549,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   if (!desc || !out || !desc->pools) return TANGRAM_EINVAL;
   if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
       desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->max_rounds < 0 ||
-      desc->round_us < 0 || desc->workspace_bytes < 0)
+      desc->round_us < 0 || desc->workspace_bytes < 0 || desc->slot_wait_us < 0)
     return TANGRAM_EINVAL;
   if ((int64_t)desc->n_scenarios * desc->max_actions > (int64_t)1 << 31) return TANGRAM_EINVAL;
   tangram_round* r = new (std::nothrow) tangram_round();
@@ -601,6 +601,10 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   size_t slab = align_up((size_t)P.N * per_cand + 64 * 1024 + (1 << 20) / 4 + 4096, 256);
   P.slab_bytes = slab;
   P.arena_bytes = desc->workspace_bytes ? (u64)desc->workspace_bytes : (2ull << 30);
+  {
+    const int64_t us = desc->slot_wait_us ? desc->slot_wait_us : 100000;
+    P.slot_tries = (int)(us / 2 > 0x3fffffff ? 0x3fffffff : (us / 2 < 1 ? 1 : us / 2));
+  }
   bool bad = false;
   bad |= cudaMalloc(&r->d_order, SC * sizeof(int)) != cudaSuccess;
   bad |= cudaMalloc(&r->d_tmin, SN * sizeof(i64) * P.P) != cudaSuccess;
@@ -1077,6 +1081,7 @@ extern "C" int tangram_schedule_batch_static(const tangram_round_desc* desc, con
   P.order = (int*)(base + o_order); P.tmin = (i64*)(base + o_tmin);
   P.slabs = (char*)(base + o_slabs); P.slab_bytes = slab; P.n_workers = (int)workers;
   P.arena = (char*)(base + o_arena); P.arena_bytes = budget - o_arena;
+  P.slot_tries = 50000;
   bind_device_io(P, a, res);
 
   cudaStream_t st = (cudaStream_t)cuda_stream;

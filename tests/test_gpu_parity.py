@@ -217,3 +217,49 @@ def test_gang_requests_with_a_large_feasible_box_match_oracle(oracle, seed, node
     g = gpu_round(pools, a)
     assert_same(o, g)
     assert np.all(g["status"] == 0) and o["n_selected"].min() >= N - 2
+
+
+def _large_box_round(seed, S):
+    pools = (Pool(POOL_GPU, 8 * 64, 8),)
+    w, a = random_round(6200 + seed, S, 48, pools, replicas=0.5, busy_fraction=0.35, inelastic=0.1, max_mult=8,
+                        ragged=False)
+    return pools, a
+
+
+def _gpu_round_ws(pools, a, **kw):
+    import torch
+    from paper_2603_13019_b200 import binding
+    S, N = a["pool"].shape
+    rnd = binding.Round(S, N, pools, **kw)
+    out = rnd.schedule_batch(binding.to_device(a))
+    torch.cuda.synchronize()
+    res = {k: v.cpu().numpy() for k, v in out.items()}
+    rnd.destroy()
+    return res
+
+
+def test_table_that_fits_no_slot_is_reported_per_scenario(oracle):
+    # one MiB of scratch: the reachable-state tables of the large boxes do not fit a slot; those
+    # scenarios get TANGRAM_STATUS_WORKSPACE, the call returns, the others are unaffected
+    pools, a = _large_box_round(3, 6)
+    o = oracle.schedule_batch(pools, a)
+    g = _gpu_round_ws(pools, a, workspace_bytes=1 << 20)
+    assert set(np.unique(g["status"])) <= {0, 4} and (g["status"] == 4).any()
+    for sc in np.flatnonzero(g["status"] == 0):
+        for k in OUT_KEYS:
+            assert np.array_equal(o[k][sc], g[k][sc]), (sc, k)
+    assert_same(o, _gpu_round_ws(pools, a))                      # the default scratch holds them all
+
+
+def test_waiting_for_a_slot_ends(oracle):
+    # four slots for 40 scenarios whose tables all need one: with a wait of one millisecond some warps
+    # give up (status word, nothing else), with the default wait every warp gets its turn
+    pools, a = _large_box_round(3, 40)
+    o = oracle.schedule_batch(pools, a)
+    short = _gpu_round_ws(pools, a, workspace_bytes=320 << 20, slot_wait_us=1000)
+    assert set(np.unique(short["status"])) <= {0, 4}
+    for sc in np.flatnonzero(short["status"] == 0):
+        for k in OUT_KEYS:
+            assert np.array_equal(o[k][sc], short[k][sc]), (sc, k)
+    patient = _gpu_round_ws(pools, a, workspace_bytes=320 << 20, slot_wait_us=5_000_000)
+    assert_same(o, patient)
