@@ -93,7 +93,7 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
 // actions that sit on pool j), placement on the pool's live state, start of what was selected.
 // Appends the started actions to run[] (nr updated).  Returns false if the scratch ran out.
 __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, const int* wait, int nw, int n,
-                            int* run, int& nr, i64 now, Slab slab, int lane) {
+                            int* run, int& nr, i64 now, Slab slab, int lane, int& busy_units) {
   const size_t row = (size_t)sc * P.N;
   const PoolDev& pd = P.pool[j];
   // members of the pool among the candidates (m) and behind them (n_ac)
@@ -199,25 +199,32 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
   __syncwarp();
   // start what was selected (Eq. 2: completion - arrival = waited so far + execution)
   i64 tot = 0;
+  int started = 0;
   for (int i = lane; i < keep; i += 32) {
     const size_t o = row + C.cidx[i];
     const int r = C.rkeep[i];
+    started += (C.cg[i] & 0x7f) * r;
     const i64 act = (now - (P.a_arrival ? P.a_arrival[o] : 0)) + duration(C.cs[i], C.cp[i], r);
     P.o_alloc[o] = (C.cg[i] & 0x7f) * r; P.o_node[o] = C.pnode[i]; P.o_off[o] = C.poff[i]; P.o_act[o] = act;
     run[nr + i] = C.cidx[i];
     tot += act;
   }
   tot = warp_sum64(tot);
+  busy_units += warp_sum32(started);
   if (lane == 0) { P.o_total[sc] += tot; P.o_nsel[sc] += keep; }
   nr += keep;
   __syncwarp();
   return true;
 }
 
-__global__ void __launch_bounds__(K2_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
+// Blocks of KR_THREADS threads: a scenario is a long chain of dependent steps on one warp, so the warps
+// are spread over as many SMs (and schedulers) as possible instead of sharing one.
+#define KR_THREADS 64
+#define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 256) + 16)
+__global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
   const int lane = threadIdx.x & 31;
-  const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
-  const int nw_warps = (gridDim.x * K2_THREADS) >> 5;
+  const int gw = (blockIdx.x * KR_THREADS + threadIdx.x) >> 5;
+  const int nw_warps = (gridDim.x * KR_THREADS) >> 5;
   for (int sc = gw; sc < P.S; sc += nw_warps) {
     const size_t row = (size_t)sc * P.N;
     const int n_act = min(max(P.n_actions[sc], 0), P.N);
@@ -257,10 +264,13 @@ __global__ void __launch_bounds__(K2_THREADS, 1) k_replay(const __grid_constant_
     int rounds = 0;
     if (status == 0) {
       extern __shared__ __align__(16) unsigned char k2_smem[];
-      int* dem = (int*)(k2_smem + K2_DYN_SMEM_TREES) + (threadIdx.x >> 5) * 64;   // 4 ints per pool: demand, capacity
+      int* dem = (int*)(k2_smem + (KR_THREADS / 32) * WARP_SMEM_BYTES + 16) + (threadIdx.x >> 5) * 64;   // 4 ints per pool: demand, capacity
       int* cap = dem + 32;
       int next = 0, nw = 0, nr = 0, r = 0;
       bool drained = false;
+      // units in use per core / GPU pool, kept up to date by what starts and what is released
+      int busy[TG_MAX_POOLS];
+      for (int j = 0; j < P.P; ++j) busy[j] = P.pool[j].type == TG_POOL_API ? 0 : pool_busy_units(P, R, sc, j, lane);
       while (r < R.max_rounds) {
         const i64 now = (i64)r * R.round_us;
         // 1. quota refill
@@ -291,6 +301,9 @@ __global__ void __launch_bounds__(K2_THREADS, 1) k_replay(const __grid_constant_
             const PoolDev& pd = P.pool[j];
             if (pd.type == TG_POOL_API) { if (pd.window_us == 0 && lane == 0) R.pst[((size_t)sc * P.P + j) * 2 + 1] -= P.o_alloc[row + fa]; }
             else {
+              const int freed = P.o_alloc[row + fa];
+#pragma unroll
+              for (int jj = 0; jj < TG_MAX_POOLS; ++jj) if (jj == j) busy[jj] -= freed;
               for (int c = lane; c < pd.capacity; c += 32) {
                 if (owner[R.unit0[j] + c] != fa) continue;
                 owner[R.unit0[j] + c] = -1;
@@ -331,7 +344,12 @@ __global__ void __launch_bounds__(K2_THREADS, 1) k_replay(const __grid_constant_
           const int nr0 = nr;
           bool ok = true;
           if (n > 0)
-            for (int j = 0; j < P.P && ok; ++j) ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane);
+            for (int j = 0; j < P.P && ok; ++j) {
+              int add = 0;
+              ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add);
+#pragma unroll
+              for (int jj = 0; jj < TG_MAX_POOLS; ++jj) if (jj == j) busy[jj] += add;
+            }
           if (!ok) { if (lane == 0) P.o_status[sc] |= TG_ST_WORKSPACE; break; }
           if (nr > nr0) {                                   // drop the started actions from the queue
             int kw = 0;
@@ -349,8 +367,7 @@ __global__ void __launch_bounds__(K2_THREADS, 1) k_replay(const __grid_constant_
           }
         }
         // 5. occupancy of this round
-        int busy[TG_MAX_POOLS];
-        for (int j = 0; j < P.P; ++j) busy[j] = pool_busy_units(P, R, sc, j, lane);
+        for (int j = 0; j < P.P; ++j) if (P.pool[j].type == TG_POOL_API) busy[j] = pool_busy_units(P, R, sc, j, lane);
         if (occ && lane == 0) for (int j = 0; j < P.P; ++j) occ[(size_t)r * P.P + j] = busy[j];
         ++r;
         if (next == n_act && nw == 0 && nr == 0) { drained = true; break; }

@@ -124,8 +124,6 @@ __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, co
 #define WARP_FAST_BYTES 2048
 #define WARP_SMEM_BYTES (WARP_TREE_BYTES + WARP_FAST_BYTES)
 #define K2_DYN_SMEM ((K2_THREADS / 32) * WARP_SMEM_BYTES + 16)
-#define K2_DYN_SMEM_TREES K2_DYN_SMEM                       // the replay kernel keeps 256 more bytes per warp behind the trees
-#define K2_DYN_SMEM_REPLAY (K2_DYN_SMEM + (K2_THREADS / 32) * 256)
 __device__ __forceinline__ void attach_warp_tree(PoolTask& T) {
   extern __shared__ __align__(16) unsigned char k2_smem[];
   const u32 start = ((u32)__cvta_generic_to_shared(k2_smem) + 15u) & ~15u;
@@ -691,7 +689,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM_REPLAY);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay, cudaFuncAttributeMaxDynamicSharedMemorySize, KR_DYN_SMEM);
   for (int c = 0; c < TG_N_SIM_CLASSES && e == cudaSuccess; ++c)
     e = cudaFuncSetAttribute(sim_kernel(g_sim_caps[c]), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TG_SMEM_PER_BLOCK - 1024);
@@ -977,7 +975,7 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
   int warps = P.n_workers < P.S ? P.n_workers : (int)align_up((size_t)P.S, K2_THREADS / 32);
   cudaEvent_t* ev = prof_begin(r, 2, -1, -1, -1);
   if (ev) CK(cudaEventRecord(ev[0], st));
-  k_replay<<<warps / (K2_THREADS / 32), K2_THREADS, K2_DYN_SMEM_REPLAY, st>>>(P, R);
+  k_replay<<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM, st>>>(P, R);
   if (ev) CK(cudaEventRecord(ev[1], st));
   r->launches += 1;
   CK(cudaGetLastError());
