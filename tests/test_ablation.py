@@ -42,3 +42,24 @@ def test_ablation_replay_matches_oracle(oracle, name):
               "rounds_used", "occupancy"):
         assert np.array_equal(o[k], out[k].cpu().numpy()), k
     rnd.destroy()
+
+
+@pytest.mark.gpu
+def test_sweep_points_match_oracle(oracle):
+    # two corners of the capacity / load sweeps (half the cores; twice the arrival rate), all policies
+    import torch
+    from dataclasses import replace
+    from paper_2603_13019_b200 import binding
+    from workloads import ablation_sweep
+    for cores, rate, pol, w in ablation_sweep():
+        if (cores, rate) not in ((128, 110.0), (256, 220.0)):
+            continue
+        w = replace(w, n_scenarios=3, max_actions=1200)
+        a = generate(w)
+        o = oracle.replay_trace(w.pools, a, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds)
+        rnd = binding.Round(3, 1200, w.pools, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds)
+        out = rnd.replay_trace(binding.to_device(a))
+        torch.cuda.synchronize()
+        for k in ("status", "n_selected", "total_act_us", "alloc_units", "act_us", "rounds_used", "occupancy"):
+            assert np.array_equal(o[k], out[k].cpu().numpy()), (w.name, k)
+        rnd.destroy()

@@ -22,4 +22,5 @@ from .generator import (  # noqa: F401
     generate,
     random_round,
     contiguous_replica_round,
+    ablation_sweep,
 )

@@ -256,11 +256,22 @@ CONFIGS: Dict[str, Workload] = {
 }
 
 
-def _ablation(dop: int) -> Workload:
-    return Workload("abl_dop%d" % dop if dop else "abl_elastic", 64, 4000, (Pool(POOL_CPU, 256, _CPU_NUMA),),
+def _ablation(dop: int, cores: int = 256, rate_per_s: float = 110.0, name: Optional[str] = None) -> Workload:
+    return Workload(name or ("abl_dop%d" % dop if dop else "abl_elastic"), 64, 4000, (Pool(POOL_CPU, cores, _CPU_NUMA),),
                     "ablation", replay=True, max_rounds=12_000,
-                    params=dict(rate_per_s=110.0, reward_fraction=0.20, pareto_alpha=1.3, pareto_min_us=5_000.0,
+                    params=dict(rate_per_s=rate_per_s, reward_fraction=0.20, pareto_alpha=1.3, pareto_min_us=5_000.0,
                                 reward_median_us=4_000_000.0, reward_sigma=1.0, dop=dop))
+
+
+def ablation_sweep():
+    """The capacity and load sweeps of the scheduling ablation: the same trace recipe at 0.5x, 1x and
+    2x the cores and at 0.5x, 1x and 2x the arrival rate (the rate stands in for the batch size of
+    the paper's sweep: more trajectories in flight submit more actions per second), each for the
+    elastic policy and the two fixed degrees of parallelism.  Yields (cores, rate, policy, workload)."""
+    for cores, rate in ((128, 110.0), (256, 110.0), (512, 110.0), (256, 55.0), (256, 220.0)):
+        for dop in (0, 4, 16):
+            pol = "dop%d" % dop if dop else "elastic"
+            yield cores, rate, pol, _ablation(dop, cores, rate, "abl_%s_c%d_r%d" % (pol, cores, int(rate)))
 
 
 # scheduling ablation on a synthetic coding-like trace: elastic 1..32 against fixed DoP 4 and 16
