@@ -59,6 +59,7 @@ struct Params {
   char* slabs; u64 slab_bytes; int n_workers;
   char* arena; u64 arena_bytes; u64* arena_top;
   int slot_tries;    // rounds of looking for a free arena slot (2 us apart) before a warp gives up
+  const u32* ok_table;   // [TG_MAX_POOLS][256]: multiplicities a record with that unit byte may use on that pool (0: none)
 };
 
 // ceil(2^64 / r) for r = 2..32: floor(p / r) == umul64hi(p, c_recip[r]) for 0 <= p <= 2^40,

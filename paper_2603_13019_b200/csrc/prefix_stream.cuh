@@ -199,7 +199,9 @@ __device__ __forceinline__ int ks_block_scan(int x, int* wsum, int t, int* total
 __global__ void __launch_bounds__(KS_THREADS, 5) k_stream(const __grid_constant__ Params P, const HeadState* hst) {
   __shared__ int s_m[TG_MAX_POOLS], s_first[TG_MAX_POOLS], s_cur[TG_MAX_POOLS], s_scan[KS_THREADS / 32];
   __shared__ int s_bad;
-  __shared__ u32 s_pinfo[TG_MAX_POOLS];             // type | GPUs per node << 4, 0xf for "no such pool"
+  // usable multiplicities by (pool, unit byte): a record's usable levels are its mask ANDed with the
+  // entry, and a record with none is invalid (decode_levels, tabulated once per round description)
+  __shared__ __align__(16) u32 s_ok[TG_MAX_POOLS * 256];
 
   const int sc = blockIdx.x, t = threadIdx.x;
   const size_t row = (size_t)sc * P.N;
@@ -211,8 +213,8 @@ __global__ void __launch_bounds__(KS_THREADS, 5) k_stream(const __grid_constant_
   if (t < TG_MAX_POOLS) {
     s_m[t] = t < P.P ? P.meta[(size_t)sc * P.P + t].m : 0;
     s_first[t] = INT_MAX;
-    s_pinfo[t] = t < P.P ? (u32)P.pool[t].type | ((u32)(P.pool[t].type == TG_POOL_GPU ? P.pool[t].group : 0) << 4) : 0xfu;
   }
+  for (int x = t; x < TG_MAX_POOLS * 256 / 4; x += KS_THREADS) ((uint4*)s_ok)[x] = ((const uint4*)P.ok_table)[x];
   if (t == 0) s_bad = H.bad;
   __syncthreads();
 
@@ -247,13 +249,9 @@ __global__ void __launch_bounds__(KS_THREADS, 5) k_stream(const __grid_constant_
       for (int k = 0; k < KS_ITEMS; ++k) {
         if (!full && i_first + k >= n_act) continue;
         const int j = rp[k];
-        const u32 pi = s_pinfo[j & (TG_MAX_POOLS - 1)];
-        PoolDev pd;
-        pd.type = pi & 15; pd.group = (pi >> 4) & 15;
-        int g, gang; u32 eff;
-        const bool ok = j < P.P && decode_levels(pd, ru[k], rm[k], g, gang, eff);
-        bad |= !ok;
-        if (ok && ((need >> j) & 1u)) rmin4[k >> 2] |= (u32)__ffs(eff) << (8 * (k & 3));
+        const u32 eff = j < TG_MAX_POOLS ? rm[k] & s_ok[j * 256 + ru[k]] : 0u;   // pools beyond the description hold zeros
+        bad |= eff == 0;
+        if ((need >> j) & 1u) rmin4[k >> 2] |= (u32)__ffs(eff) << (8 * (k & 3));
       }
     }
     if (bad) s_bad = 1;

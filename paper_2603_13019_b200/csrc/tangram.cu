@@ -439,7 +439,7 @@ struct tangram_round {
   int64_t launches;
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
-  HeadState* hst; void* d_preq; void* d_keepn; int* d_fl;
+  HeadState* hst; void* d_preq; void* d_keepn; int* d_fl; u32* d_ok_table;
   BatchWs W; int sim_blocks; SimLists L; int n_sm;
   ReplayWs R;
   // host-buffer mode: copy-in, kernels and copy-out of successive chunks on streams of their own
@@ -684,6 +684,37 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
     bad |= cudaMalloc((void**)&r->d_stage, off) != cudaSuccess;
   }
   if (bad) { cudaGetLastError(); tangram_round_destroy(r); return TANGRAM_ENOMEM; }
+  {
+    // usable multiplicities by (pool, unit byte), as decode_levels computes them
+    static_assert(sizeof(u32) == 4, "");
+    u32* tab = new (std::nothrow) u32[TG_MAX_POOLS * 256]();
+    cudaError_t ce = tab ? cudaMalloc((void**)&r->d_ok_table, TG_MAX_POOLS * 256 * sizeof(u32)) : cudaErrorMemoryAllocation;
+    if (ce == cudaSuccess) {
+      for (int j = 0; j < P.P; ++j)
+        for (int un = 0; un < 256; ++un) {
+          const int g = un & 0x7f;
+          const bool gpu = P.pool[j].type == TG_POOL_GPU, gang = (un >> 7) && gpu;
+          u32 ok = g == 0 ? 0u : 0xffffffffu;
+          if (g != 0 && gpu) {
+            const bool p2 = (g & (g - 1)) == 0;
+            if (gang) {
+              ok = 0;
+              if (p2) {
+                if (g <= P.pool[j].group) ok |= 1u;
+                if (2 * g <= P.pool[j].group) ok |= 2u;
+                if (4 * g <= P.pool[j].group) ok |= 8u;
+                if (8 * g <= P.pool[j].group) ok |= 128u;
+              }
+            } else if (!(p2 && g <= P.pool[j].group)) ok = 0;
+          }
+          tab[j * 256 + un] = ok;
+        }
+      ce = cudaMemcpy(r->d_ok_table, tab, TG_MAX_POOLS * 256 * sizeof(u32), cudaMemcpyHostToDevice);
+    }
+    delete[] tab;
+    if (ce != cudaSuccess) { cudaGetLastError(); tangram_round_destroy(r); return TANGRAM_ENOMEM; }
+    P.ok_table = r->d_ok_table;
+  }
   P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
   P.preq = (unsigned short*)r->d_preq; P.keepn = (int*)r->d_keepn;
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
@@ -753,7 +784,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
-  cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl);
+  cudaFree(r->d_ok_table); cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
