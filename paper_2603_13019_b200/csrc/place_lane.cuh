@@ -70,7 +70,83 @@ __device__ __forceinline__ void kpl_store(const Params& P, KplWarp& W, size_t ro
 
 // phase 0: the pools that the head kernel certified (decided by k_easy); phase 1: all the others, and
 // the cleaning up behind scenarios with an invalid record.
-__global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ Params P, const HeadState* hst, int phase) {
+// GPU pools of at most 128 nodes whose selection went through the solver: one WARP per (scenario, pool).
+// The node masks live in lane registers and "lowest node with a free block of this size" is one warp
+// reduction (place_gpu_reg's rule, Section 5.3), so a pool's placement is a short chain on a warp of
+// its own instead of the longest per-thread loop of a warp that holds 32 pools.  Requests and indices
+// are read from the kept-request rows, results go straight to place_node / place_off.
+__global__ void __launch_bounds__(256) k_place_gpu(const __grid_constant__ Params P, const HeadState* hst) {
+  const int lane = threadIdx.x & 31;
+  const long long x = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (x >= (long long)P.S * P.P) return;
+  const int sc = (int)(x % P.S), j = P.pool_order[x / P.S];
+  const PoolDev& pd = P.pool[j];
+  if (pd.type != TG_POOL_GPU || !pd.lane_place || pd.n_nodes > 128 || !((hst[sc].need >> j) & 1u)) return;
+  if (P.o_status[sc] & TG_ST_BAD_ACTION) return;
+  const int keep = P.keepn[(size_t)sc * P.P + j];
+  if (keep <= 0) return;
+  const size_t row = (size_t)sc * P.N;
+  const i64 base = P.meta[(size_t)sc * P.P + j].cbase;
+  const unsigned short* rq = P.preq + row + base;
+  const int* ord = P.order + row + base;
+  // Section 5.3: requests by size descending, then queue position; each takes the smallest
+  // sufficient maximal free block, lowest (node, start), and the low end of a split block.
+  const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total + pd.node0 : nullptr;
+  const int top = ilog2(pd.group), n_nodes = pd.n_nodes;
+  const u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;
+  u32 nm[4], lev[4];
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const int v = lane + 32 * s;
+    nm[s] = v < n_nodes ? ((busy_row ? busy_row[v] : 0u) | pad) : 0xffu;
+    lev[s] = node_levels(nm[s]);
+  }
+  for (int lz = top; lz >= 0; --lz) {
+    const int z = 1 << lz;
+    for (int i0 = 0; i0 < keep; i0 += 32) {
+      const int i = i0 + lane;
+      int nreq = 0;
+      if (i < keep) {
+        const u32 v = rq[i];
+        const int g = v & 0x7f, gang = (v >> 7) & 1, ri = v >> 8;
+        nreq = gang ? (g * ri == z ? 1 : 0) : (g == z ? ri : 0);
+      }
+      int myn = -1, myo = -1;
+      u32 bm = __ballot_sync(TG_FULL, nreq > 0);
+      while (bm) {
+        const int b = __ffs(bm) - 1; bm &= bm - 1;
+        const int cnt = __shfl_sync(TG_FULL, nreq, b);
+        for (int rep = 0; rep < cnt; ++rep) {
+          u32 node = 0xffffffffu; int bl = lz;
+          for (; bl <= top; ++bl) {                     // smallest sufficient block level, lowest node
+            u32 key = 0xffffffffu;
+#pragma unroll
+            for (int s = 3; s >= 0; --s) if ((lev[s] >> bl) & 1u) key = (u32)(lane + 32 * s);
+            node = __reduce_min_sync(TG_FULL, key);
+            if (node != 0xffffffffu) break;
+          }
+          if (node == 0xffffffffu) continue;            // cannot happen: the selection fits
+          int start = 0;
+          if (lane == (int)(node & 31u)) {
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+              if (s == (int)(node >> 5)) {
+                start = node_block_start(nm[s], bl);
+                nm[s] |= ((1u << z) - 1u) << start;
+                lev[s] = node_levels(nm[s]);
+              }
+          }
+          start = __shfl_sync(TG_FULL, start, node & 31u);
+          if (rep == 0 && lane == b) { myn = (int)node; myo = start; }
+        }
+      }
+      if (i < keep && myn >= 0) { const size_t o = row + ord[i]; P.o_node[o] = myn; P.o_off[o] = myo; }
+    }
+  }
+}
+
+// gpu_apart: the solver-side GPU pools are left to k_place_gpu.
+__global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ Params P, const HeadState* hst, int phase, int gpu_apart) {
   __shared__ KplWarp s_w[KPL_WARPS];
   const int lane = threadIdx.x & 31;
   KplWarp& W = s_w[threadIdx.x >> 5];
@@ -92,6 +168,7 @@ __global__ void __launch_bounds__(KPL_THREADS) k_place(const __grid_constant__ P
   int keep = (sc < P.S && !bad) ? P.keepn[(size_t)sc * P.P + j] : 0;
   if (keep < 0) keep = 0;
   if (sc < P.S && (int)(((hst[sc].need >> j) & 1u) != 0u) != phase) keep = 0;   // the other phase's pool
+  if (phase == 1 && gpu_apart && pd.type == TG_POOL_GPU) keep = 0;             // k_place_gpu has them
   const int maxkeep = warp_max32(keep);
   if (maxkeep == 0) return;
   const size_t row = (size_t)(sc < P.S ? sc : 0) * P.N;

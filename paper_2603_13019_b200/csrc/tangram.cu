@@ -912,18 +912,22 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
     CK(cudaEventRecord(r->side_fork, st));
     CK(cudaStreamWaitEvent(r->side, r->side_fork, 0));
     k_easy<<<(unsigned)(((size_t)P.S * P.P + 7) / 8), 256, 0, r->side>>>(P, r->hst);
-    k_place<<<place_grid, KPL_THREADS, 0, r->side>>>(P, r->hst, 0);
+    k_place<<<place_grid, KPL_THREADS, 0, r->side>>>(P, r->hst, 0, 0);
     CK(cudaEventRecord(r->side_join, r->side));
   }
   CK(cudaMemsetAsync(r->d_fl, 0, 2 * sizeof(int), st));
   k_finish_list<<<(P.S * P.P + 255) / 256, 256, 0, st>>>(P, W, r->d_fl);
   k_finish<<<wblocks, K2_THREADS, K2_DYN_SMEM, st>>>(P, W, r->d_fl);
   if (ev) CK(cudaEventRecord(ev[5], st));
-  k_place<<<place_grid, KPL_THREADS, 0, st>>>(P, r->hst, 1);
+  // A warp per GPU pool is the shorter chain as long as all those warps are resident at once; beyond
+  // that a thread per pool (32 pools per warp instruction) gets through the batch sooner.
+  const int gpu_apart = (long long)P.S * P.P <= (long long)r->n_sm * 64 * 2 ? 1 : 0;
+  k_place<<<place_grid, KPL_THREADS, 0, st>>>(P, r->hst, 1, gpu_apart);
+  if (gpu_apart) k_place_gpu<<<(unsigned)(((size_t)P.S * P.P + 7) / 8), 256, 0, st>>>(P, r->hst);
   CK(cudaStreamWaitEvent(st, r->side_join, 0));
   CK(cudaStreamWaitEvent(st, r->sim_join[TG_N_SIM_CLASSES], 0));   // the fill is part of the round
   if (ev) CK(cudaEventRecord(ev[6], st));
-  r->launches += 11 + TG_N_SIM_CLASSES;
+  r->launches += 11 + TG_N_SIM_CLASSES + gpu_apart;
   CK(cudaGetLastError());
   return TANGRAM_OK;
 }
