@@ -37,8 +37,10 @@ METRIC = "actions scheduled/sec (1xB200)"
 # DRAM bytes per pending action (dram__bytes_read.sum + dram__bytes_write.sum of one launch / actions of the
 # launch) from the ncu capture summarised under profiles/ (cfg4 shape, 2048
 # scenarios); traffic grows in proportion to the actions, so a launch's traffic is this times its actions.
-# The k_stream interval of the per-kernel timing holds k_fill as well (it runs beside it).
-NCU_BYTES_PER_ACTION = {"cfg4": {"k_stream": 35.0, "k_head": 1.72, "k_solve": 2.07, "k_finish": 1.89, "k_place": 0.59}}
+# The k_stream interval of the per-kernel timing holds k_fill as well (it runs beside it), the k_finish interval
+# k_easy and the certified pools' k_place (beside it), the k_place interval the solver-side pools' placement.
+NCU_BYTES_PER_ACTION = {"cfg4": {"k_head": 1.72, "k_stream": 34.1, "k_solve": 1.54, "k_sims": 2.40,
+                                 "k_finish": 1.88 + 1.91 + 0.53, "k_place": 0.05 + 0.22}}
 NCU_TRAFFIC_SOURCE = "ncu on 2048 scenarios of the same shape, scaled by actions (profiles/)"
 
 
