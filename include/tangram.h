@@ -160,16 +160,18 @@ int tangram_replay_trace(tangram_round* round, const tangram_actions* actions,
  * All scratch lives in one array of TANGRAM_STATIC_SCRATCH_BYTES that is part of the library
  * image: every GPU that loads the library holds those bytes until the process exits, whether
  * or not this entry point is ever called.  A batch whose scratch does not fit is refused with
- * TANGRAM_ETOOBIG and nothing is launched; roughly, 12 bytes per action of
- * n_scenarios * max_actions plus eight worker areas of about 63 * max_actions + 330 KiB plus
- * 4 MiB for large DP tables must fit.  At most 32 worker warps run, so this call is slower on
- * big batches; results are identical.  A scenario whose DP tables outgrow what is left of the
+ * TANGRAM_ETOOBIG and nothing is launched: 12 bytes per action of n_scenarios * max_actions,
+ * plus (39 + 16 * depth) * max_actions + 324 KiB for each of 8 to 32 worker warps (as many as
+ * fit, at least 8), plus at least 4 MiB for large DP tables must fit.  At most 32 worker warps
+ * run, so this call is slower on big batches; results are identical.  A scenario whose DP tables outgrow what is left of the
  * array is marked TANGRAM_STATUS_WORKSPACE in `status`, exactly as with a round whose
  * workspace_bytes is too small; the other scenarios of the batch are unaffected.
  *
  * The first call on each device (with that device current) looks up the array's device
  * address and loads two small constant tables; make that first call outside any stream
- * capture.  Every call uses the same array and leaves its contents behind: two calls whose
+ * capture, and from one host thread: the look-up is remembered in plain process-wide
+ * variables, so two threads making the FIRST call on a device at the same time race on them
+ * (later calls only read them).  Every call uses the same array and leaves its contents behind: two calls whose
  * kernels can overlap on the GPU (different streams, or different host threads on one
  * device) race on it and must be serialised by the caller; calls on one stream are safe.
  * Asynchronous on `cuda_stream`. */

@@ -51,9 +51,12 @@
 //   R14 Objective sums saturate at INT64_MAX.
 //   R17 Quota pools refill to capacity at multiples of their window.
 //
-// Parity unpinned by the paper: the value of estimate() and the eviction stopping point
-// are heuristics with no printed example; they are pinned by closed-form special cases
-// and invariants only (see tests).
+// The paper prints no worked example of a schedule.  estimate() and the eviction loop are
+// heuristics; they are pinned by closed forms, by an independent list-scheduling statement
+// and by cases worked by hand in the tests (two accepted evictions and a refused third,
+// evicted candidates ahead of the waiting list, a running action of the same pool in the
+// heap, saturating sums), DPArrange by exhaustive enumeration, the chunk test by brute-force
+// packing, placement by worked examples.
 #include <algorithm>
 #include <climits>
 #include <cstdint>
