@@ -93,8 +93,7 @@ __device__ bool gather_candidates(const Params& P, int sc, int j, const PoolMeta
   return true;
 }
 
-// with_waiting = false leaves out what is known about the pool's waiting actions (k_solve runs
-// beside k_stream, which is still counting them).
+// with_waiting = false leaves out the pool's waiting actions (k_solve estimates nothing itself).
 __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, const CandArrays& C, int lane,
                           PoolTask& T, bool with_waiting = true) {
   const PoolDev& pd = P.pool[j];
@@ -224,10 +223,8 @@ __device__ void run_pool_task(const Params& P, int sc, int j, Slab slab, int lan
 __global__ void __launch_bounds__(K2_THREADS) k_select(const __grid_constant__ Params P) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * K2_THREADS + threadIdx.x) >> 5;
-  const int nw = (gridDim.x * K2_THREADS) >> 5;
   const Slab slab = warp_slab(P, gw);
   const int n_tasks = P.S * P.P;
-  (void)nw;
   for (;;) {
     const int x = next_task(P.arena_top + 3, lane);
     if (x >= n_tasks) break;
