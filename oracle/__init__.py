@@ -56,9 +56,25 @@ def _c(a, dt):
     return None if a is None else np.ascontiguousarray(a, dtype=dt)
 
 
+def _cache_args(arrays, sl, S, pools, cache_slots):
+    """service / restore_us / cache state of scenarios `sl` (copies: the oracle updates the state in place)."""
+    service = _c(arrays["service"][sl], np.uint16) if arrays.get("service") is not None else None
+    restore = _c(arrays["restore_us"][sl], np.int64) if arrays.get("restore_us") is not None else None
+    tag = use = None
+    if cache_slots > 0:
+        n = _n_nodes(pools) * 8 * cache_slots
+        tag = (np.array(arrays["cache_tag"][sl], dtype=np.uint32, order="C", copy=True).reshape(S, n)
+               if arrays.get("cache_tag") is not None else np.zeros((S, n), np.uint32))
+        use = (np.array(arrays["cache_use"][sl], dtype=np.int64, order="C", copy=True).reshape(S, n)
+               if arrays.get("cache_use") is not None else np.zeros((S, n), np.int64))
+    return service, restore, tag, use
+
+
 def schedule_batch(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, depth: int = 2,
-                   now_us: int = 0, lo: int = 0, hi: Optional[int] = None) -> Dict[str, np.ndarray]:
-    """One scheduling round for scenarios [lo, hi) of the given input arrays."""
+                   now_us: int = 0, lo: int = 0, hi: Optional[int] = None, cache_slots: int = 0) -> Dict[str, np.ndarray]:
+    """One scheduling round for scenarios [lo, hi) of the given input arrays.  With cache_slots > 0 the
+    GPU pools keep a service cache (arrays "service", "restore_us", "cache_tag", "cache_use"); the
+    updated cache state comes back as "cache_tag" / "cache_use"."""
     S_all, N = arrays["pool"].shape
     hi = S_all if hi is None else hi
     S = hi - lo
@@ -77,21 +93,26 @@ def schedule_batch(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, 
         total_act_us=np.empty(S, np.int64), n_selected=np.empty(S, np.int32),
         status=np.empty(S, np.int32))
     pf = _pools_flat(pools)
-    rc = lib().oracle_schedule_batch(
+    service, restore, tag, use = _cache_args(arrays, sl, S, pools, cache_slots)
+    rc = lib().oracle_schedule_batch_cache(
         C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), C.c_int(depth),
         C.c_int(_n_nodes(pools)), _p(n_act, C.c_int), _p(pool, C.c_uint8), _p(unit, C.c_uint8),
         _p(mask, C.c_uint32), _p(s, C.c_longlong), _p(p, C.c_longlong), _p(arr, C.c_longlong),
         _p(busy, C.c_uint8), C.c_longlong(now_us),
         _p(out["alloc_units"], C.c_int), _p(out["place_node"], C.c_int), _p(out["place_off"], C.c_int),
         _p(out["act_us"], C.c_longlong), _p(out["total_act_us"], C.c_longlong),
-        _p(out["n_selected"], C.c_int), _p(out["status"], C.c_int))
+        _p(out["n_selected"], C.c_int), _p(out["status"], C.c_int),
+        _p(service, C.c_uint16), _p(restore, C.c_longlong), C.c_int(cache_slots), _p(tag, C.c_uint32),
+        _p(use, C.c_longlong))
     assert rc == 0
+    if cache_slots > 0:
+        out["cache_tag"], out["cache_use"] = tag, use
     return out
 
 
 def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, depth: int = 2,
                  round_us: int = 10_000, max_rounds: int, lo: int = 0, hi: Optional[int] = None,
-                 want_occupancy: bool = True) -> Dict[str, np.ndarray]:
+                 want_occupancy: bool = True, cache_slots: int = 0) -> Dict[str, np.ndarray]:
     """Trace replay of scenarios [lo, hi)."""
     S_all, N = arrays["pool"].shape
     hi = S_all if hi is None else hi
@@ -112,7 +133,8 @@ def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, de
         status=np.empty(S, np.int32), rounds_used=np.empty(S, np.int32),
         occupancy=np.empty((S, max_rounds, len(pools)), np.int32) if want_occupancy else None)
     pf = _pools_flat(pools)
-    rc = lib().oracle_replay_trace(
+    service, restore, tag, use = _cache_args(arrays, sl, S, pools, cache_slots)
+    rc = lib().oracle_replay_trace_cache(
         C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), C.c_int(depth),
         C.c_int(_n_nodes(pools)), C.c_longlong(round_us), C.c_int(max_rounds),
         _p(n_act, C.c_int), _p(pool, C.c_uint8), _p(unit, C.c_uint8), _p(mask, C.c_uint32),
@@ -120,8 +142,12 @@ def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, de
         _p(out["alloc_units"], C.c_int), _p(out["place_node"], C.c_int), _p(out["place_off"], C.c_int),
         _p(out["act_us"], C.c_longlong), _p(out["total_act_us"], C.c_longlong),
         _p(out["n_selected"], C.c_int), _p(out["status"], C.c_int), _p(out["occupancy"], C.c_int),
-        _p(out["rounds_used"], C.c_int))
+        _p(out["rounds_used"], C.c_int),
+        _p(service, C.c_uint16), _p(restore, C.c_longlong), C.c_int(cache_slots), _p(tag, C.c_uint32),
+        _p(use, C.c_longlong))
     assert rc == 0
+    if cache_slots > 0:
+        out["cache_tag"], out["cache_use"] = tag, use
     return out
 
 

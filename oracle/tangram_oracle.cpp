@@ -50,6 +50,19 @@
 //       ascending domains.  API pools report the units consumed before the grant.
 //   R14 Objective sums saturate at INT64_MAX.
 //   R17 Quota pools refill to capacity at multiples of their window.
+//   R19 Service cache (Section 5.3, evict on execution): every GPU remembers up to K service
+//       instances, an instance being (service id, chunk size) since different degrees of
+//       parallelism of a service count as distinct services; a chunk caches an instance iff
+//       every GPU of the chunk remembers it.
+//   R20 Among the free blocks of the level that the allocation rule picks (smallest
+//       sufficient), one whose granted chunk (its low end) caches the requested instance is
+//       preferred; then lowest (node, start).
+//   R21 A grant refreshes the instance's last use on every GPU of the chunk; on a miss each
+//       GPU first overwrites an empty entry (lowest index), else its least recently used one
+//       (lowest index among equals).
+//   R22 An action one of whose chunks missed runs restore_us longer (restoration from host
+//       memory precedes execution).  The scheduler's duration model does not see this: it
+//       decides before the placement.
 //
 // The paper prints no worked example of a schedule.  estimate() and the eviction loop are
 // heuristics; they are pinned by closed forms, by an independent list-scheduling statement
@@ -81,6 +94,8 @@ struct Action {
   bool gang = false, valid = true;
   std::vector<int> r;       // allowed multiplicities, ascending
   i64 s = 0, p = 0, arrival = 0;
+  int service = -1;         // requested service (GPU pools), -1: none
+  i64 restore = 0;          // restoration time if the granted chunk does not cache the instance
   bool elastic() const { return r.size() > 1; }
 };
 
@@ -329,6 +344,9 @@ struct PoolRuntime {
   PoolDesc d;
   std::vector<int> core_owner;       // CPU: action id or -1
   std::vector<uint8_t> node_busy;    // GPU: bit b = GPU b busy
+  int cache_slots = 0;               // GPU: instances a GPU remembers (0: no service cache)
+  std::vector<unsigned> cache_tag;   // GPU: [gpu][slot] instance tag, 0 = empty
+  std::vector<i64> cache_use;        // GPU: [gpu][slot] time of last use
   int api_used = 0;                  // quota pools: tokens used in the current window
   i64 window = 0;
   int in_use = 0;                    // concurrency pools: units held
@@ -342,7 +360,7 @@ struct PoolRuntime {
 
 struct Chunk { int node, start, size; };
 struct Running { i64 finish; int action, pool, units; std::vector<Chunk> chunks; };
-struct Grant { int action, r, units, node, off; std::vector<Chunk> chunks; };
+struct Grant { int action, r, units, node, off; std::vector<Chunk> chunks; bool missed = false; };
 
 // what DPArrange needs to know about the pool: free units, or free chunk counts
 struct PoolRoom { bool gpu; int free_units; int F[4]; };
@@ -369,8 +387,33 @@ i64 approx_objective(const std::vector<const Action*>& Cj, int q, const PoolRoom
 }
 
 // ------------------------------------------------------------- placement (R13)
+// instance tag of (service, chunk size); 0 is "empty"
+unsigned instance_tag(int service, int size) { return ((unsigned)service << 3 | (unsigned)log2i(size)) + 1u; }
+
+bool chunk_caches(const PoolRuntime& pr, int node, int start, int size, unsigned tag) {
+  for (int b = start; b < start + size; ++b) {
+    bool has = false;
+    for (int k = 0; k < pr.cache_slots; ++k) has |= pr.cache_tag[(size_t)(node * pr.d.group + b) * pr.cache_slots + k] == tag;
+    if (!has) return false;
+  }
+  return true;
+}
+
+// R21: the instance becomes the most recently used one on every GPU of the chunk
+void cache_touch(PoolRuntime& pr, int node, int start, int size, unsigned tag, i64 now) {
+  for (int b = start; b < start + size; ++b) {
+    unsigned* tg = &pr.cache_tag[(size_t)(node * pr.d.group + b) * pr.cache_slots];
+    i64* us = &pr.cache_use[(size_t)(node * pr.d.group + b) * pr.cache_slots];
+    int at = -1;
+    for (int k = 0; k < pr.cache_slots && at < 0; ++k) if (tg[k] == tag) at = k;
+    for (int k = 0; k < pr.cache_slots && at < 0; ++k) if (tg[k] == 0) at = k;
+    if (at < 0) { at = 0; for (int k = 1; k < pr.cache_slots; ++k) if (us[k] < us[at]) at = k; }
+    tg[at] = tag; us[at] = now;
+  }
+}
+
 void place_gpu(PoolRuntime& pr, const std::vector<Action>& acts, std::vector<Grant>& grants,
-               const std::vector<int>& which) {
+               const std::vector<int>& which, i64 now = 0) {
   struct Req { int size, rank, rep, grant; };
   std::vector<Req> reqs;
   for (int gi : which) {
@@ -384,13 +427,21 @@ void place_gpu(PoolRuntime& pr, const std::vector<Action>& acts, std::vector<Gra
     return x.rep < y.rep;
   });
   for (const Req& rq : reqs) {
+    const Action& a = acts[grants[rq.grant].action];
+    const bool cached_pool = pr.cache_slots > 0 && a.service >= 0;
+    const unsigned tag = cached_pool ? instance_tag(a.service, rq.size) : 0u;
     int best_size = INT_MAX, best_node = -1, best_start = -1;
+    bool best_hit = false;
     for (int node = 0; node < (int)pr.node_busy.size(); ++node) {
-      // maximal free aligned blocks of this node, smallest sufficient one
+      // maximal free aligned blocks of this node: smallest sufficient one, a caching one first (R20)
       std::function<void(int, int)> walk = [&](int start, int size) {
         int bits = ((1 << size) - 1) << start;
         if ((pr.node_busy[node] & bits) == 0) {
-          if (size >= rq.size && size < best_size) { best_size = size; best_node = node; best_start = start; }
+          if (size < rq.size) return;
+          const bool hit = cached_pool && chunk_caches(pr, node, start, rq.size, tag);
+          if (size < best_size || (size == best_size && hit && !best_hit)) {
+            best_size = size; best_node = node; best_start = start; best_hit = hit;
+          }
           return;
         }
         if (size == 1) return;
@@ -403,6 +454,10 @@ void place_gpu(PoolRuntime& pr, const std::vector<Action>& acts, std::vector<Gra
     Grant& g = grants[rq.grant];
     g.chunks.push_back(Chunk{best_node, best_start, rq.size});
     if (rq.rep == 0) { g.node = best_node; g.off = best_start; }
+    if (cached_pool) {
+      if (!best_hit) g.missed = true;                              // R22
+      cache_touch(pr, best_node, best_start, rq.size, tag, now);
+    }
   }
 }
 
@@ -500,14 +555,17 @@ std::vector<Grant> schedule_round(std::vector<PoolRuntime>& pools, const std::ve
       which.push_back((int)grants.size());
       grants.push_back(g);
     }
-    if (pools[j].d.type == POOL_GPU) place_gpu(pools[j], acts, grants, which);
+    if (pools[j].d.type == POOL_GPU) place_gpu(pools[j], acts, grants, which, now);
     else if (pools[j].d.type == POOL_CPU) place_cpu(pools[j], grants, which);
     else place_api(pools[j], grants, which);
   }
   return grants;
 }
 
-std::vector<PoolRuntime> fresh_pools(const std::vector<PoolDesc>& pd, const uint8_t* gpu_busy) {
+struct CacheIo { int slots; unsigned* tag; i64* use; };   // per scenario: [node][8][slots], in and out
+
+std::vector<PoolRuntime> fresh_pools(const std::vector<PoolDesc>& pd, const uint8_t* gpu_busy,
+                                     const CacheIo* cache = nullptr) {
   std::vector<PoolRuntime> pools(pd.size());
   int node0 = 0;
   for (size_t j = 0; j < pd.size(); ++j) {
@@ -518,6 +576,18 @@ std::vector<PoolRuntime> fresh_pools(const std::vector<PoolDesc>& pd, const uint
       pools[j].node_busy.assign(nodes, 0);
       if (gpu_busy)
         for (int v = 0; v < nodes; ++v) pools[j].node_busy[v] = gpu_busy[node0 + v] & (uint8_t)((1 << pd[j].group) - 1);
+      if (cache && cache->slots > 0) {
+        pools[j].cache_slots = cache->slots;
+        pools[j].cache_tag.assign((size_t)nodes * pd[j].group * cache->slots, 0u);
+        pools[j].cache_use.assign((size_t)nodes * pd[j].group * cache->slots, 0);
+        for (int v = 0; v < nodes; ++v)
+          for (int b = 0; b < pd[j].group; ++b)
+            for (int k = 0; k < cache->slots; ++k) {
+              const size_t src = ((size_t)(node0 + v) * 8 + b) * cache->slots + k;
+              const size_t dst = ((size_t)v * pd[j].group + b) * cache->slots + k;
+              pools[j].cache_tag[dst] = cache->tag[src]; pools[j].cache_use[dst] = cache->use[src];
+            }
+      }
       node0 += nodes;
     }
   }
@@ -526,14 +596,35 @@ std::vector<PoolRuntime> fresh_pools(const std::vector<PoolDesc>& pd, const uint
 
 bool load_actions(std::vector<Action>& acts, int n, const std::vector<PoolDesc>& pd,
                   const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
-                  const i64* s, const i64* p, const i64* arrival) {
+                  const i64* s, const i64* p, const i64* arrival,
+                  const uint16_t* service = nullptr, const i64* restore = nullptr) {
   acts.resize(n);
   bool ok = true;
   for (int i = 0; i < n; ++i) {
     acts[i] = decode_action(pool[i], unit[i], mask[i], s[i], p[i], arrival ? arrival[i] : 0, pd);
+    if (service && service[i] != 0xffff) acts[i].service = service[i];
+    if (restore) acts[i].restore = clamp_param(restore[i]);
     ok &= acts[i].valid;
   }
   return ok;
+}
+
+// the pools' cache state back to the caller's arrays
+void store_cache(const std::vector<PoolRuntime>& pools, const CacheIo* cache) {
+  if (!cache || cache->slots <= 0) return;
+  int node0 = 0;
+  for (const PoolRuntime& pr : pools) {
+    if (pr.d.type != POOL_GPU) continue;
+    const int nodes = pr.d.capacity / pr.d.group;
+    for (int v = 0; v < nodes; ++v)
+      for (int b = 0; b < pr.d.group; ++b)
+        for (int k = 0; k < cache->slots; ++k) {
+          const size_t dst = ((size_t)(node0 + v) * 8 + b) * cache->slots + k;
+          const size_t src = ((size_t)v * pr.d.group + b) * cache->slots + k;
+          cache->tag[dst] = pr.cache_tag[src]; cache->use[dst] = pr.cache_use[src];
+        }
+    node0 += nodes;
+  }
 }
 
 }  // namespace
@@ -544,12 +635,16 @@ extern "C" {
 // Whole batched round.  Arrays are host memory, scenario-major with row stride max_actions;
 // pools = n_pools x {type, capacity, group, window_us}; gpu_busy has row stride n_nodes
 // (may be null); arrival may be null.  Outputs as documented for the product's result.
-int oracle_schedule_batch(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+// service (0xffff: none), restore_us, cache_slots, cache_tag / cache_use ([scenario][node][8][slots],
+// updated in place) describe the service cache of the GPU pools (Section 5.3); all may be null / 0.
+int oracle_schedule_batch_cache(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
                           int depth, int n_nodes, const int* n_actions, const uint8_t* pool,
                           const uint8_t* unit, const uint32_t* mask, const i64* s, const i64* p,
                           const i64* arrival, const uint8_t* gpu_busy, i64 now,
                           int* alloc_units, int* place_node, int* place_off, i64* act_us,
-                          i64* total_act_us, int* n_selected, int* status) {
+                          i64* total_act_us, int* n_selected, int* status,
+                          const uint16_t* service, const i64* restore, int cache_slots,
+                          unsigned* cache_tag, i64* cache_use) {
   std::vector<PoolDesc> pd(n_pools);
   for (int j = 0; j < n_pools; ++j)
     pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
@@ -562,11 +657,15 @@ int oracle_schedule_batch(int n_scenarios, int max_actions, int n_pools, const i
     total_act_us[sc] = 0; n_selected[sc] = 0; status[sc] = STATUS_OK;
     std::vector<Action> acts;
     if (!load_actions(acts, n, pd, pool + base, unit + base, mask + base, s + base, p + base,
-                      arrival ? arrival + base : nullptr)) {
+                      arrival ? arrival + base : nullptr, service ? service + base : nullptr,
+                      restore ? restore + base : nullptr)) {
       status[sc] = STATUS_BAD_ACTION;
       continue;
     }
-    std::vector<PoolRuntime> pools = fresh_pools(pd, gpu_busy ? gpu_busy + (size_t)sc * n_nodes : nullptr);
+    const size_t cstride = (size_t)n_nodes * 8 * (cache_slots > 0 ? cache_slots : 0);
+    CacheIo cio{cache_slots, cache_tag ? cache_tag + sc * cstride : nullptr, cache_use ? cache_use + sc * cstride : nullptr};
+    const CacheIo* cache = (cache_slots > 0 && cache_tag && cache_use) ? &cio : nullptr;
+    std::vector<PoolRuntime> pools = fresh_pools(pd, gpu_busy ? gpu_busy + (size_t)sc * n_nodes : nullptr, cache);
     std::vector<int> W(n);
     for (int i = 0; i < n; ++i) W[i] = i;
     std::vector<Running> E;
@@ -577,25 +676,40 @@ int oracle_schedule_batch(int n_scenarios, int max_actions, int n_pools, const i
       place_node[base + g.action] = g.node;
       place_off[base + g.action] = g.off;
       i64 act = (now - a.arrival) + duration(a, g.r);              // Eq. 2: queueing + execution
+      if (g.missed) act += a.restore;                              // R22: restoration precedes execution
       act_us[base + g.action] = act;
       total_act_us[sc] = sat_add(total_act_us[sc], act);
       n_selected[sc]++;
     }
+    store_cache(pools, cache);
   }
   return 0;
+}
+
+int oracle_schedule_batch(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+                          int depth, int n_nodes, const int* n_actions, const uint8_t* pool,
+                          const uint8_t* unit, const uint32_t* mask, const i64* s, const i64* p,
+                          const i64* arrival, const uint8_t* gpu_busy, i64 now,
+                          int* alloc_units, int* place_node, int* place_off, i64* act_us,
+                          i64* total_act_us, int* n_selected, int* status) {
+  return oracle_schedule_batch_cache(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, n_actions, pool,
+                                     unit, mask, s, p, arrival, gpu_busy, now, alloc_units, place_node, place_off,
+                                     act_us, total_act_us, n_selected, status, nullptr, nullptr, 0, nullptr, nullptr);
 }
 
 // Trace replay: rounds at now = r * round_us, r = 0 .. max_rounds-1.  Each round releases
 // what has finished, admits what has arrived, runs the scheduler, starts what it selects.
 // occupancy: [scenario][round][pool] units in use after the round's scheduling (zero after
 // the scenario has drained); rounds_used: rounds until drained (max_rounds if never).
-int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+int oracle_replay_trace_cache(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
                         int depth, int n_nodes, i64 round_us, int max_rounds, const int* n_actions,
                         const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
                         const i64* s, const i64* p, const i64* arrival, const uint8_t* gpu_busy,
                         int* alloc_units, int* place_node, int* place_off, i64* act_us,
                         i64* total_act_us, int* n_selected, int* status, int* occupancy,
-                        int* rounds_used) {
+                        int* rounds_used,
+                        const uint16_t* service, const i64* restore, int cache_slots,
+                        unsigned* cache_tag, i64* cache_use) {
   std::vector<PoolDesc> pd(n_pools);
   for (int j = 0; j < n_pools; ++j)
     pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
@@ -610,14 +724,18 @@ int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int
       std::memset(occupancy + (size_t)sc * max_rounds * n_pools, 0, sizeof(int) * (size_t)max_rounds * n_pools);
     std::vector<Action> acts;
     if (!load_actions(acts, n, pd, pool + base, unit + base, mask + base, s + base, p + base,
-                      arrival ? arrival + base : nullptr)) {
+                      arrival ? arrival + base : nullptr, service ? service + base : nullptr,
+                      restore ? restore + base : nullptr)) {
       status[sc] = STATUS_BAD_ACTION;
       continue;
     }
     bool sorted = true;
     for (int i = 1; i < n; ++i) sorted &= acts[i - 1].arrival <= acts[i].arrival;
     if (!sorted) { status[sc] = STATUS_UNSORTED; continue; }
-    std::vector<PoolRuntime> pools = fresh_pools(pd, gpu_busy ? gpu_busy + (size_t)sc * n_nodes : nullptr);
+    const size_t cstride = (size_t)n_nodes * 8 * (cache_slots > 0 ? cache_slots : 0);
+    CacheIo cio{cache_slots, cache_tag ? cache_tag + sc * cstride : nullptr, cache_use ? cache_use + sc * cstride : nullptr};
+    const CacheIo* cache = (cache_slots > 0 && cache_tag && cache_use) ? &cio : nullptr;
+    std::vector<PoolRuntime> pools = fresh_pools(pd, gpu_busy ? gpu_busy + (size_t)sc * n_nodes : nullptr, cache);
     std::vector<int> W;
     std::vector<Running> E;
     int next = 0, r = 0;
@@ -641,6 +759,7 @@ int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int
       for (const Grant& g : grants) {                               // start selected actions
         const Action& a = acts[g.action];
         i64 T = duration(a, g.r);
+        if (g.missed) T += a.restore;                               // R22
         E.push_back(Running{now + T, g.action, a.pool, g.units, g.chunks});
         alloc_units[base + g.action] = g.units;
         place_node[base + g.action] = g.node;
@@ -657,8 +776,22 @@ int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int
       if (next == n && W.empty() && E.empty()) { ++r; break; }
     }
     rounds_used[sc] = r;
+    store_cache(pools, cache);
   }
   return 0;
+}
+
+int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+                        int depth, int n_nodes, i64 round_us, int max_rounds, const int* n_actions,
+                        const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
+                        const i64* s, const i64* p, const i64* arrival, const uint8_t* gpu_busy,
+                        int* alloc_units, int* place_node, int* place_off, i64* act_us,
+                        i64* total_act_us, int* n_selected, int* status, int* occupancy,
+                        int* rounds_used) {
+  return oracle_replay_trace_cache(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, round_us, max_rounds,
+                                   n_actions, pool, unit, mask, s, p, arrival, gpu_busy, alloc_units, place_node,
+                                   place_off, act_us, total_act_us, n_selected, status, occupancy, rounds_used,
+                                   nullptr, nullptr, 0, nullptr, nullptr);
 }
 
 // ---- single pieces, exported so that tests can pin each of them on its own ----------
