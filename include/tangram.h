@@ -93,6 +93,11 @@ typedef struct {
                               give one back before it gives up (the scenario then gets
                               TANGRAM_STATUS_WORKSPACE); 0 = default (100 ms).  The holders of the
                               slots never wait for anything, so a waiter cannot block them.        */
+  int32_t cache_slots;     /* service cache of the GPU pools (Section 5.3, evict on execution): service
+                              instances every GPU remembers, 0 .. 4; 0 = no cache (then `service`,
+                              `restore_us` and the cache arrays of tangram_actions are ignored).
+                              Not available with host_buffers = 1.                                 */
+  int32_t reserved;        /* 0                                                                    */
   const tangram_pool_desc* pools; /* host array of n_pools entries, copied                 */
 } tangram_round_desc;
 
@@ -110,6 +115,16 @@ typedef struct {
   const uint8_t* gpu_busy;    /* may be null.  Per scenario, one byte per node of every GPU
                                  pool (pools in index order, row stride = total nodes): bit b
                                  set <=> GPU b of the node is occupied before the round       */
+  /* Service cache (only read when cache_slots > 0; Section 5.3).  An action on a GPU pool asks for a
+   * service; the instance it needs is (service, chunk size), different degrees of parallelism of a
+   * service being distinct instances.  Among the free chunks of the level that the allocation rule
+   * picks, one that caches the instance is preferred; an action one of whose chunks does not cache
+   * it runs restore_us longer.  Every GPU remembers cache_slots instances, least recently used out. */
+  const uint16_t* service;    /* per action, may be null; 0xffff = no service                    */
+  const int64_t* restore_us;  /* per action, may be null (0); clamped to [0, 2^40]               */
+  uint32_t* gpu_cache_tag;    /* per scenario [node][8][cache_slots], IN and OUT: instance tag
+                                 (service * 8 + log2(chunk size)) + 1, 0 = empty entry           */
+  int64_t* gpu_cache_use;     /* same shape, IN and OUT: time of the entry's last use             */
 } tangram_actions;
 
 /* Results, caller-owned, fully overwritten by a call (rows up to max_actions). */

@@ -48,6 +48,8 @@ struct Params {
   const u8* a_pool; const u8* a_unit; const u32* a_mask;
   const i64* a_s; const i64* a_p; const i64* a_arrival;
   const int* n_actions; const u8* gpu_busy;
+  // service cache of the GPU pools (cache_slots = 0: none)
+  const unsigned short* a_service; const i64* a_restore; u32* cache_tag; i64* cache_use; int cache_slots;
   // outputs (device)
   int* o_alloc; int* o_node; int* o_off; i64* o_act; i64* o_total; int* o_nsel; int* o_status;
   // workspace

@@ -192,6 +192,76 @@ __device__ __forceinline__ int node_block_start(u32 busy, int bl) {
   return __ffs(m) - 1;
 }
 
+// GPU placement with a service cache (Section 5.3, evict on execution).  The rule of place_gpu, and among
+// the free blocks of the level it picks, one whose granted chunk (the block's low end) caches the
+// request's instance goes first, then the lowest (node, start).  An instance is (service, chunk size);
+// a chunk caches it iff every GPU of the chunk remembers its tag.  ctag / cuse: the pool's entries,
+// [node][8][K] (tag 0 = empty, time of last use).  A grant makes the instance the most recently used
+// one on every GPU of the chunk; on a miss a GPU overwrites an empty entry (lowest index), else its
+// least recently used one (lowest index among equals), and miss[i] is set: candidate i then runs its
+// restoration time longer.  svc: the scenario's service column (may be null), ids: action indices.
+__device__ void place_gpu_cache(const PoolDev& pd, u8* nm, int keep, const u8* cg, const u8* r, const int* ids,
+                                int* pnode, int* poff, u8* miss, const unsigned short* svc, u32* ctag, i64* cuse,
+                                int K, i64 now, int lane, int* owner = nullptr) {
+  const int top = ilog2(pd.group);
+  const u32 pad = (~((1u << pd.group) - 1u)) & 0xffu;
+  for (int i = lane; i < keep; i += 32) miss[i] = 0;
+  __syncwarp();
+  for (int lz = top; lz >= 0; --lz) {
+    const int z = 1 << lz;
+    for (int i = 0; i < keep; ++i) {
+      const int g = cg[i] & 0x7f, gang = cg[i] >> 7, ri = r[i];
+      const int nreq = gang ? (g * ri == z ? 1 : 0) : (g == z ? ri : 0);
+      if (nreq == 0) continue;
+      const u32 sv = svc ? svc[ids[i]] : 0xffffu;
+      const u32 tag = sv == 0xffffu ? 0u : ((sv << 3) | (u32)lz) + 1u;
+      for (int rep = 0; rep < nreq; ++rep) {
+        u32 kmin = 0xffffffffu;
+        for (int bl = lz; bl <= top && kmin == 0xffffffffu; ++bl) {
+          u32 key = 0xffffffffu;
+          for (int v = lane; v < pd.n_nodes; v += 32) {
+            const NodeBlocks nb = node_blocks(nm[v] | pad);
+            u32 starts = bl == 0 ? nb.s1 : (bl == 1 ? nb.s2 : (bl == 2 ? nb.s4 : nb.s8));
+            while (starts) {
+              const int st = __ffs(starts) - 1; starts &= starts - 1;
+              bool hit = tag != 0;
+              for (int b = st; b < st + z && hit; ++b) {
+                bool has = false;
+                for (int k = 0; k < K; ++k) has |= ctag[(size_t)(v * 8 + b) * K + k] == tag;
+                hit = has;
+              }
+              key = min(key, (hit ? 0u : 1u << 30) | ((u32)v << 4) | (u32)st);
+            }
+          }
+          kmin = __reduce_min_sync(TG_FULL, key);
+        }
+        if (kmin == 0xffffffffu) continue;              // cannot happen: the selection fits
+        const int node = (int)((kmin >> 4) & 0x3ffffffu), start = (int)(kmin & 15u);
+        const bool hit = (kmin >> 30) == 0;
+        __syncwarp();
+        if (lane == 0) {
+          nm[node] |= (u8)(((1u << z) - 1u) << start);
+          if (rep == 0) { pnode[i] = node; poff[i] = start; }
+          if (owner) for (int b = 0; b < z; ++b) owner[node * pd.group + start + b] = ids[i];
+          if (tag) {
+            if (!hit) miss[i] = 1;
+            for (int b = start; b < start + z; ++b) {
+              u32* tg = ctag + (size_t)(node * 8 + b) * K;
+              i64* us = cuse + (size_t)(node * 8 + b) * K;
+              int at = -1;
+              for (int k = 0; k < K && at < 0; ++k) if (tg[k] == tag) at = k;
+              for (int k = 0; k < K && at < 0; ++k) if (tg[k] == 0) at = k;
+              if (at < 0) { at = 0; for (int k = 1; k < K; ++k) if (us[k] < us[at]) at = k; }
+              tg[at] = tag; us[at] = now;
+            }
+          }
+        }
+        __syncwarp();
+      }
+    }
+  }
+}
+
 // Same placement rule as place_gpu; requires pd.n_nodes <= 128.  busy_row: the pool's node
 // masks before the round (may be null).
 __device__ void place_gpu_reg(const PoolDev& pd, const u8* busy_row, int keep, const u8* cg, const u8* r,

@@ -184,7 +184,14 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
     if (keep < 0) return false;
   }
   // placement on the pool's live state
-  if (pd.type == TG_POOL_GPU) {
+  const u8* missed = nullptr;                            // candidates whose chunk did not cache their service
+  if (pd.type == TG_POOL_GPU && P.cache_slots > 0) {
+    const size_t cbase = ((size_t)sc * P.n_nodes_total + pd.node0) * 8 * P.cache_slots;
+    place_gpu_cache(pd, R.nm + (size_t)sc * P.n_nodes_total + pd.node0, keep, C.cg, C.rkeep, C.cidx, C.pnode, C.poff,
+                    C.rsel, P.a_service ? P.a_service + row : nullptr, P.cache_tag + cbase, P.cache_use + cbase,
+                    P.cache_slots, now, lane, R.owner + (size_t)sc * R.U + R.unit0[j]);
+    missed = C.rsel;
+  } else if (pd.type == TG_POOL_GPU) {
     place_gpu(pd, R.nm + (size_t)sc * P.n_nodes_total + pd.node0, keep, C.cg, C.rkeep, C.pnode, C.poff, lane,
               R.owner + (size_t)sc * R.U + R.unit0[j], C.cidx);
   } else if (pd.type == TG_POOL_CPU) {
@@ -204,7 +211,8 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
     const size_t o = row + C.cidx[i];
     const int r = C.rkeep[i];
     started += (C.cg[i] & 0x7f) * r;
-    const i64 act = (now - (P.a_arrival ? P.a_arrival[o] : 0)) + duration(C.cs[i], C.cp[i], r);
+    i64 act = (now - (P.a_arrival ? P.a_arrival[o] : 0)) + duration(C.cs[i], C.cp[i], r);
+    if (missed && missed[i] && P.a_restore) act += clamp_param(P.a_restore[o]);   // restoration precedes execution
     P.o_alloc[o] = (C.cg[i] & 0x7f) * r; P.o_node[o] = C.pnode[i]; P.o_off[o] = C.poff[i]; P.o_act[o] = act;
     run[nr + i] = C.cidx[i];
     tot += act;

@@ -147,12 +147,26 @@ __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& 
   const PoolDev& pd = P.pool[j];
   const size_t row = (size_t)sc * P.N;
   const u8* busy_row = P.gpu_busy ? P.gpu_busy + (size_t)sc * P.n_nodes_total : nullptr;
+  const u8* missed = nullptr;                            // candidates whose chunk did not cache their service
   defer = defer && pd.lane_place;
   if (defer) {
     // k_place will place this pool: leave it the kept requests in queue order
     unsigned short* rq = P.preq + row + mt.cbase;
     for (int i = lane; i < keep; i += 32) rq[i] = (unsigned short)(C.cg[i] | ((u32)C.rkeep[i] << 8));
     if (lane == 0) P.keepn[(size_t)sc * P.P + j] = keep;
+  } else if (pd.type == TG_POOL_GPU && P.cache_slots > 0) {
+    // with a service cache: the chunk that caches the instance first, entries updated, misses noted in C.rsel
+    u8* nm = (u8*)slab.take_fast(pd.n_nodes);
+    if (!nm) { if (lane == 0) atomicOr(&P.o_status[sc], TG_ST_WORKSPACE); keep = 0; }
+    else {
+      for (int v = lane; v < pd.n_nodes; v += 32) nm[v] = busy_row ? busy_row[pd.node0 + v] : 0;
+      __syncwarp();
+      const size_t cbase = ((size_t)sc * P.n_nodes_total + pd.node0) * 8 * P.cache_slots;
+      place_gpu_cache(pd, nm, keep, C.cg, C.rkeep, C.cidx, C.pnode, C.poff, C.rsel,
+                      P.a_service ? P.a_service + row : nullptr, P.cache_tag + cbase, P.cache_use + cbase,
+                      P.cache_slots, P.now, lane);
+      missed = C.rsel;
+    }
   } else if (pd.type == TG_POOL_GPU) {
     if (pd.n_nodes <= 128) place_gpu_reg(pd, busy_row ? busy_row + pd.node0 : nullptr, keep, C.cg, C.rkeep, C.pnode, C.poff, lane);
     else {
@@ -187,6 +201,7 @@ __device__ void place_and_write(const Params& P, int sc, int j, const PoolMeta& 
       int r = C.rkeep[i];
       i64 arr = P.a_arrival ? P.a_arrival[o] : 0;
       i64 act = (P.now - arr) + duration(C.cs[i], C.cp[i], r);
+      if (missed && missed[i] && P.a_restore) act += clamp_param(P.a_restore[o]);   // restoration precedes execution
       P.o_alloc[o] = (C.cg[i] & 0x7f) * r; P.o_act[o] = act;
       if (!defer) { P.o_node[o] = C.pnode[i]; P.o_off[o] = C.poff[i]; }
       tot += act; ++cnt;
@@ -544,7 +559,8 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   if (!desc || !out || !desc->pools) return TANGRAM_EINVAL;
   if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
       desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->max_rounds < 0 ||
-      desc->round_us < 0 || desc->workspace_bytes < 0 || desc->slot_wait_us < 0)
+      desc->round_us < 0 || desc->workspace_bytes < 0 || desc->slot_wait_us < 0 || desc->cache_slots < 0 ||
+      desc->cache_slots > 4 || (desc->cache_slots > 0 && desc->host_buffers))
     return TANGRAM_EINVAL;
   if ((int64_t)desc->n_scenarios * desc->max_actions > (int64_t)1 << 31) return TANGRAM_EINVAL;
   tangram_round* r = new (std::nothrow) tangram_round();
@@ -553,6 +569,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   r->desc = *desc;
   Params& P = r->P;
   P.S = desc->n_scenarios; P.N = desc->max_actions; P.P = desc->n_pools; P.depth = desc->depth;
+  P.cache_slots = desc->cache_slots;
   int node0 = 0, slot0 = 0;
   for (int j = 0; j < desc->n_pools; ++j) {
     const tangram_pool_desc& pd = desc->pools[j];
@@ -571,6 +588,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
     d.slot0 = slot0; d.n_slots = pd.type == TANGRAM_POOL_GPU ? 4 : 1;
     slot0 += d.n_slots;
     d.lane_place = lane_place_ok(d);
+    if (desc->cache_slots > 0 && pd.type == TANGRAM_POOL_GPU) d.lane_place = 0;   // placed by the warp that decides the pool
   }
   r->desc.pools = r->pools;
   P.n_nodes_total = node0;
@@ -856,6 +874,8 @@ static void bind_device_io(Params& P, const tangram_actions* a, const tangram_re
   P.a_s = (const i64*)a->s_us; P.a_p = (const i64*)a->p_us; P.a_arrival = (const i64*)a->arrival_us;
   P.n_actions = a->n_actions;
   P.gpu_busy = P.n_nodes_total ? a->gpu_busy : nullptr;
+  P.a_service = a->service; P.a_restore = (const i64*)a->restore_us;
+  P.cache_tag = a->gpu_cache_tag; P.cache_use = (i64*)a->gpu_cache_use;
   P.o_alloc = res->alloc_units; P.o_node = res->place_node; P.o_off = res->place_off;
   P.o_act = (i64*)res->act_us; P.o_total = (i64*)res->total_act_us;
   P.o_nsel = res->n_selected; P.o_status = res->status;
@@ -932,6 +952,7 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
 extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a, int64_t now_us,
                                       tangram_result* res, void* cuda_stream) {
   if (!r || !check_io(a, res)) return TANGRAM_EINVAL;
+  if (r->desc.cache_slots > 0 && r->P.n_nodes_total > 0 && (!a->gpu_cache_tag || !a->gpu_cache_use)) return TANGRAM_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   Params P = r->P;
   P.now = now_us;
@@ -989,6 +1010,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
 extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, tangram_result* res,
                                     void* cuda_stream) {
   if (!r || !check_io(a, res) || r->desc.max_rounds <= 0 || !a->arrival_us) return TANGRAM_EINVAL;
+  if (r->desc.cache_slots > 0 && r->P.n_nodes_total > 0 && (!a->gpu_cache_tag || !a->gpu_cache_use)) return TANGRAM_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   Params P = r->P;
   P.now = 0;
@@ -1056,7 +1078,8 @@ extern "C" int tangram_schedule_batch_static(const tangram_round_desc* desc, con
                                              int64_t now_us, tangram_result* res, void* cuda_stream) {
   if (!desc || !desc->pools || !check_io(a, res)) return TANGRAM_EINVAL;
   if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
-      desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->host_buffers)
+      desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->host_buffers ||
+      desc->cache_slots != 0)
     return TANGRAM_EINVAL;
   if ((int64_t)desc->n_scenarios * desc->max_actions > (int64_t)1 << 31) return TANGRAM_ETOOBIG;
   Params P;

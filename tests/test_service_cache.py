@@ -112,3 +112,75 @@ def test_replay_keeps_the_instance_cached_after_the_action(oracle):
     assert list(o["cache_tag"][0, :8]) == [tag(5, 4)] * 4 + [tag(6, 4)] * 4
     assert list(o["cache_use"][0, :8]) == [3000] * 8
     assert o["rounds_used"][0] == 7                               # z finishes at 3000 + 2300 = 5300 -> round 6 is the last busy one
+
+
+# ------------------------------------------------------------------ CUDA path against the oracle
+def _with_services(seed, a, pools, slots, n_services=5):
+    """Adds services, restoration times and a random cache state to a round's arrays (input generator only)."""
+    rng = np.random.default_rng(seed)
+    S, N = a["pool"].shape
+    nodes = sum(p.capacity // p.group for p in pools if p.type == POOL_GPU)
+    a = dict(a)
+    a["service"] = np.where(rng.random((S, N)) < 0.85, rng.integers(0, n_services, (S, N)), NONE).astype(np.uint16)
+    a["restore_us"] = rng.integers(0, 300_000, (S, N)).astype(np.int64)
+    sv = rng.integers(0, n_services, (S, nodes * 8 * slots))
+    sz = rng.integers(0, 4, (S, nodes * 8 * slots))
+    a["cache_tag"] = np.where(rng.random((S, nodes * 8 * slots)) < 0.7, (sv << 3 | sz) + 1, 0).astype(np.uint32)
+    a["cache_use"] = rng.integers(-50, 50, (S, nodes * 8 * slots)).astype(np.int64)
+    return a
+
+
+CACHE_KEYS = ("status", "n_selected", "total_act_us", "alloc_units", "place_node", "place_off", "act_us",
+              "cache_tag", "cache_use")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed,slots", [(0, 1), (1, 2), (2, 4), (3, 2)])
+def test_rounds_with_a_service_cache_match_oracle(oracle, seed, slots):
+    import torch
+    from paper_2603_13019_b200 import binding
+    pools = [(Pool(POOL_CPU, 16, 4), Pool(POOL_GPU, 32, 8)), (Pool(POOL_GPU, 64, 8),),
+             (Pool(POOL_GPU, 16, 4), Pool(POOL_GPU, 24, 8)), (Pool(POOL_GPU, 8 * 70, 8),)][seed]
+    w, a = random_round(9100 + seed, 48, [60, 90, 40, 700][seed], pools, busy_fraction=0.3, max_mult=4,
+                        replicas=0.5, small_durations=0.3 if seed == 1 else 0.0)
+    a = _with_services(seed, a, pools, slots)
+    o = oracle.schedule_batch(pools, a, cache_slots=slots, now_us=100)
+    S, N = a["pool"].shape
+    rnd = binding.Round(S, N, pools, cache_slots=slots)
+    dev = binding.to_device(a)
+    out = rnd.schedule_batch(dev, now_us=100)
+    torch.cuda.synchronize()
+    g = {k: v.cpu().numpy() for k, v in out.items()}
+    g["cache_tag"] = dev["cache_tag"].cpu().numpy().view(np.uint32)
+    g["cache_use"] = dev["cache_use"].cpu().numpy()
+    rnd.destroy()
+    for k in CACHE_KEYS:
+        assert np.array_equal(o[k], g[k]), k
+    sel = o["alloc_units"] > 0
+    assert sel.sum() > 50
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(3))
+def test_traces_with_a_service_cache_match_oracle(oracle, seed):
+    import torch
+    from paper_2603_13019_b200 import binding
+    pools = [(Pool(POOL_CPU, 16, 4), Pool(POOL_GPU, 32, 8)), (Pool(POOL_GPU, 40, 8),),
+             (Pool(POOL_GPU, 16, 4), Pool(POOL_GPU, 32, 8))][seed]
+    slots = [1, 2, 3][seed]
+    w, a = random_round(9200 + seed, 12, 150, pools, max_mult=4, replicas=0.5, busy_fraction=0.0)
+    rng = np.random.default_rng(seed)
+    a["arrival_us"] = np.cumsum(rng.integers(0, 6000, a["pool"].shape), axis=1).astype(np.int64)
+    a = _with_services(seed, a, pools, slots, n_services=3)
+    o = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=6000, cache_slots=slots)
+    rnd = binding.Round(12, 150, pools, round_us=10_000, max_rounds=6000, cache_slots=slots)
+    dev = binding.to_device(a)
+    out = rnd.replay_trace(dev)
+    torch.cuda.synchronize()
+    g = {k: v.cpu().numpy() for k, v in out.items()}
+    g["cache_tag"] = dev["cache_tag"].cpu().numpy().view(np.uint32)
+    g["cache_use"] = dev["cache_use"].cpu().numpy()
+    rnd.destroy()
+    for k in CACHE_KEYS + ("rounds_used", "occupancy"):
+        assert np.array_equal(o[k], g[k]), k
+    assert (o["alloc_units"] > 0).sum() > 800 and np.all(o["status"] == 0)

@@ -75,7 +75,7 @@ def test_static_entry_point_refuses_what_does_not_fit():
     import ctypes as C
     arr = (binding._PoolDesc * len(w.pools))(*[binding._PoolDesc(p.type, p.capacity, p.group, p.window_us)
                                                  for p in w.pools])
-    desc = binding._RoundDesc(S, N, len(w.pools), 2, 0, 0, 0, 0, 0, arr)
+    desc = binding._RoundDesc(S, N, len(w.pools), 2, 0, 0, 0, 0, 0, 0, 0, arr)
     a = binding._Actions(z8.data_ptr(), z8.data_ptr(), z32.data_ptr(), z64.data_ptr(), z64.data_ptr(), None,
                          z32.data_ptr(), None)
     r = binding._Result(z32.data_ptr(), z32.data_ptr(), z32.data_ptr(), z64.data_ptr(), z64.data_ptr(),
