@@ -70,6 +70,15 @@ def _cache_args(arrays, sl, S, pools, cache_slots):
     return service, restore, tag, use
 
 
+def _side_args(arrays, sl):
+    """Further entries of the cost vectors, [n_side][scenario][action] (pool 0xff: none)."""
+    if arrays.get("side_pool") is None:
+        return 0, None, None
+    sp = _c(arrays["side_pool"][:, sl], np.uint8)
+    su = _c(arrays["side_units"][:, sl], np.uint16)
+    return sp.shape[0], sp, su
+
+
 def schedule_batch(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, depth: int = 2,
                    now_us: int = 0, lo: int = 0, hi: Optional[int] = None, cache_slots: int = 0) -> Dict[str, np.ndarray]:
     """One scheduling round for scenarios [lo, hi) of the given input arrays.  With cache_slots > 0 the
@@ -94,7 +103,8 @@ def schedule_batch(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, 
         status=np.empty(S, np.int32))
     pf = _pools_flat(pools)
     service, restore, tag, use = _cache_args(arrays, sl, S, pools, cache_slots)
-    rc = lib().oracle_schedule_batch_cache(
+    n_side, side_pool, side_units = _side_args(arrays, sl)
+    rc = lib().oracle_schedule_batch_ext(
         C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), C.c_int(depth),
         C.c_int(_n_nodes(pools)), _p(n_act, C.c_int), _p(pool, C.c_uint8), _p(unit, C.c_uint8),
         _p(mask, C.c_uint32), _p(s, C.c_longlong), _p(p, C.c_longlong), _p(arr, C.c_longlong),
@@ -103,7 +113,7 @@ def schedule_batch(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, 
         _p(out["act_us"], C.c_longlong), _p(out["total_act_us"], C.c_longlong),
         _p(out["n_selected"], C.c_int), _p(out["status"], C.c_int),
         _p(service, C.c_uint16), _p(restore, C.c_longlong), C.c_int(cache_slots), _p(tag, C.c_uint32),
-        _p(use, C.c_longlong))
+        _p(use, C.c_longlong), C.c_int(n_side), _p(side_pool, C.c_uint8), _p(side_units, C.c_uint16))
     assert rc == 0
     if cache_slots > 0:
         out["cache_tag"], out["cache_use"] = tag, use
@@ -134,7 +144,8 @@ def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, de
         occupancy=np.empty((S, max_rounds, len(pools)), np.int32) if want_occupancy else None)
     pf = _pools_flat(pools)
     service, restore, tag, use = _cache_args(arrays, sl, S, pools, cache_slots)
-    rc = lib().oracle_replay_trace_cache(
+    n_side, side_pool, side_units = _side_args(arrays, sl)
+    rc = lib().oracle_replay_trace_ext(
         C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), C.c_int(depth),
         C.c_int(_n_nodes(pools)), C.c_longlong(round_us), C.c_int(max_rounds),
         _p(n_act, C.c_int), _p(pool, C.c_uint8), _p(unit, C.c_uint8), _p(mask, C.c_uint32),
@@ -144,7 +155,7 @@ def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, de
         _p(out["n_selected"], C.c_int), _p(out["status"], C.c_int), _p(out["occupancy"], C.c_int),
         _p(out["rounds_used"], C.c_int),
         _p(service, C.c_uint16), _p(restore, C.c_longlong), C.c_int(cache_slots), _p(tag, C.c_uint32),
-        _p(use, C.c_longlong))
+        _p(use, C.c_longlong), C.c_int(n_side), _p(side_pool, C.c_uint8), _p(side_units, C.c_uint16))
     assert rc == 0
     if cache_slots > 0:
         out["cache_tag"], out["cache_use"] = tag, use

@@ -63,6 +63,21 @@
 //   R22 An action one of whose chunks missed runs restore_us longer (restoration from host
 //       memory precedes execution).  The scheduler's duration model does not see this: it
 //       decides before the placement.
+//   R23 Cost vectors (Section 4.1, vectorized resource cost): besides its key resource an
+//       action may name up to two further pools with a fixed amount each (memory beside the
+//       cores, quotas of other sites).  Such a pool is a quota or concurrency pool other than
+//       the key pool and the amount lies in 1 .. its capacity; anything else is a bad record.
+//       Only the key resource is elastic (the paper's assumption), durations follow it alone.
+//   R24 accommodate (Algorithm 1, candidate prefix): an action fits if its least key level
+//       and every further amount fit on top of what the actions before it in the queue ask.
+//   R25 R_k handed to DPArrange for pool k is what is free minus the further amounts that ALL
+//       candidates of the prefix ask of k, whatever their key pool; an evicted candidate's
+//       amounts are not handed back within the round.
+//   R26 A started action consumes its further amounts (a quota pool counts them in the
+//       window, a concurrency pool holds them until the action finishes); an evicted one
+//       consumes nothing.  They are booked after all pools have placed their key grants, so
+//       a quota pool's place_off counts what was used before the round plus the key grants
+//       ahead in queue order.
 //
 // The paper prints no worked example of a schedule.  estimate() and the eviction loop are
 // heuristics; they are pinned by closed forms, by an independent list-scheduling statement
@@ -96,6 +111,7 @@ struct Action {
   i64 s = 0, p = 0, arrival = 0;
   int service = -1;         // requested service (GPU pools), -1: none
   i64 restore = 0;          // restoration time if the granted chunk does not cache the instance
+  std::vector<std::pair<int, int> > side;   // further (pool, amount) entries of the cost vector (R23)
   bool elastic() const { return r.size() > 1; }
 };
 
@@ -515,9 +531,22 @@ std::vector<Grant> schedule_round(std::vector<PoolRuntime>& pools, const std::ve
       for (int l = 0; l < 4; ++l) req[j][l] = nn[l];
     } else {
       if (used[j] + a.g * a.r.front() > freeu[j]) break;
-      used[j] += a.g * a.r.front();
     }
+    // R24: the further amounts of the cost vector have to fit as well
+    std::vector<int> extra(k, 0);
+    bool fits = true;
+    for (const std::pair<int, int>& c : a.side) {
+      extra[c.first] += c.second;
+      fits &= used[c.first] + extra[c.first] <= freeu[c.first];
+    }
+    if (!fits) break;
+    if (pools[j].d.type != POOL_GPU) used[j] += a.g * a.r.front();
+    for (int q = 0; q < k; ++q) used[q] += extra[q];
   }
+  // R25: what the candidates ask of a pool beside their key resource is set aside
+  std::vector<int> aside(k, 0);
+  for (size_t i = 0; i < n; ++i)
+    for (const std::pair<int, int>& c : acts[W[i]].side) aside[c.first] += c.second;
   std::vector<Grant> grants;
   for (int j = 0; j < k; ++j) {                                    // line 3
     std::vector<const Action*> Cj, ACj;
@@ -538,7 +567,7 @@ std::vector<Grant> schedule_round(std::vector<PoolRuntime>& pools, const std::ve
       std::vector<i64> running_rel;
       for (const Running& e : E) if (e.pool == j) running_rel.push_back(std::max<i64>(0, e.finish - now));
       PoolRoom room;
-      room.gpu = pools[j].d.type == POOL_GPU; room.free_units = freeu[j];
+      room.gpu = pools[j].d.type == POOL_GPU; room.free_units = freeu[j] - aside[j];
       for (int l = 0; l < 4; ++l) room.F[l] = F[j][l];
       i64 obj = approx_objective(Cj, m, room, ACj, running_rel, depth, &alloc);   // line 8
       for (int tt = 1; tt <= m - 1; ++tt) {                        // lines 9-14 (R6)
@@ -559,6 +588,11 @@ std::vector<Grant> schedule_round(std::vector<PoolRuntime>& pools, const std::ve
     else if (pools[j].d.type == POOL_CPU) place_cpu(pools[j], grants, which);
     else place_api(pools[j], grants, which);
   }
+  for (const Grant& g : grants)                                    // R26
+    for (const std::pair<int, int>& c : acts[g.action].side) {
+      PoolRuntime& pr = pools[c.first];
+      if (pr.d.window_us > 0) pr.api_used += c.second; else pr.in_use += c.second;
+    }
   return grants;
 }
 
@@ -597,13 +631,22 @@ std::vector<PoolRuntime> fresh_pools(const std::vector<PoolDesc>& pd, const uint
 bool load_actions(std::vector<Action>& acts, int n, const std::vector<PoolDesc>& pd,
                   const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
                   const i64* s, const i64* p, const i64* arrival,
-                  const uint16_t* service = nullptr, const i64* restore = nullptr) {
+                  const uint16_t* service = nullptr, const i64* restore = nullptr,
+                  int n_side = 0, const uint8_t* side_pool = nullptr, const uint16_t* side_units = nullptr,
+                  size_t plane = 0) {
   acts.resize(n);
   bool ok = true;
   for (int i = 0; i < n; ++i) {
     acts[i] = decode_action(pool[i], unit[i], mask[i], s[i], p[i], arrival ? arrival[i] : 0, pd);
     if (service && service[i] != 0xffff) acts[i].service = service[i];
     if (restore) acts[i].restore = clamp_param(restore[i]);
+    for (int e = 0; e < n_side && side_pool && side_units; ++e) {    // R23
+      const int k = side_pool[e * plane + i], c = side_units[e * plane + i];
+      if (k == 0xff) continue;
+      if (k >= (int)pd.size() || pd[k].type != POOL_API || k == acts[i].pool || c < 1 || c > pd[k].capacity)
+        acts[i].valid = false;
+      else acts[i].side.push_back(std::make_pair(k, c));
+    }
     ok &= acts[i].valid;
   }
   return ok;
@@ -637,14 +680,17 @@ extern "C" {
 // (may be null); arrival may be null.  Outputs as documented for the product's result.
 // service (0xffff: none), restore_us, cache_slots, cache_tag / cache_use ([scenario][node][8][slots],
 // updated in place) describe the service cache of the GPU pools (Section 5.3); all may be null / 0.
-int oracle_schedule_batch_cache(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+// side_pool (0xff: none) / side_units, [n_side][scenario][action], are the further entries of the
+// actions' cost vectors (Section 4.1, R23-R26); may be null / 0.
+int oracle_schedule_batch_ext(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
                           int depth, int n_nodes, const int* n_actions, const uint8_t* pool,
                           const uint8_t* unit, const uint32_t* mask, const i64* s, const i64* p,
                           const i64* arrival, const uint8_t* gpu_busy, i64 now,
                           int* alloc_units, int* place_node, int* place_off, i64* act_us,
                           i64* total_act_us, int* n_selected, int* status,
                           const uint16_t* service, const i64* restore, int cache_slots,
-                          unsigned* cache_tag, i64* cache_use) {
+                          unsigned* cache_tag, i64* cache_use,
+                          int n_side, const uint8_t* side_pool, const uint16_t* side_units) {
   std::vector<PoolDesc> pd(n_pools);
   for (int j = 0; j < n_pools; ++j)
     pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
@@ -658,7 +704,8 @@ int oracle_schedule_batch_cache(int n_scenarios, int max_actions, int n_pools, c
     std::vector<Action> acts;
     if (!load_actions(acts, n, pd, pool + base, unit + base, mask + base, s + base, p + base,
                       arrival ? arrival + base : nullptr, service ? service + base : nullptr,
-                      restore ? restore + base : nullptr)) {
+                      restore ? restore + base : nullptr, n_side, side_pool ? side_pool + base : nullptr,
+                      side_units ? side_units + base : nullptr, (size_t)n_scenarios * max_actions)) {
       status[sc] = STATUS_BAD_ACTION;
       continue;
     }
@@ -692,16 +739,16 @@ int oracle_schedule_batch(int n_scenarios, int max_actions, int n_pools, const i
                           const i64* arrival, const uint8_t* gpu_busy, i64 now,
                           int* alloc_units, int* place_node, int* place_off, i64* act_us,
                           i64* total_act_us, int* n_selected, int* status) {
-  return oracle_schedule_batch_cache(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, n_actions, pool,
+  return oracle_schedule_batch_ext(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, n_actions, pool,
                                      unit, mask, s, p, arrival, gpu_busy, now, alloc_units, place_node, place_off,
-                                     act_us, total_act_us, n_selected, status, nullptr, nullptr, 0, nullptr, nullptr);
+                                     act_us, total_act_us, n_selected, status, nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr);
 }
 
 // Trace replay: rounds at now = r * round_us, r = 0 .. max_rounds-1.  Each round releases
 // what has finished, admits what has arrived, runs the scheduler, starts what it selects.
 // occupancy: [scenario][round][pool] units in use after the round's scheduling (zero after
 // the scenario has drained); rounds_used: rounds until drained (max_rounds if never).
-int oracle_replay_trace_cache(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
                         int depth, int n_nodes, i64 round_us, int max_rounds, const int* n_actions,
                         const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
                         const i64* s, const i64* p, const i64* arrival, const uint8_t* gpu_busy,
@@ -709,7 +756,8 @@ int oracle_replay_trace_cache(int n_scenarios, int max_actions, int n_pools, con
                         i64* total_act_us, int* n_selected, int* status, int* occupancy,
                         int* rounds_used,
                         const uint16_t* service, const i64* restore, int cache_slots,
-                        unsigned* cache_tag, i64* cache_use) {
+                        unsigned* cache_tag, i64* cache_use,
+                        int n_side, const uint8_t* side_pool, const uint16_t* side_units) {
   std::vector<PoolDesc> pd(n_pools);
   for (int j = 0; j < n_pools; ++j)
     pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
@@ -725,7 +773,8 @@ int oracle_replay_trace_cache(int n_scenarios, int max_actions, int n_pools, con
     std::vector<Action> acts;
     if (!load_actions(acts, n, pd, pool + base, unit + base, mask + base, s + base, p + base,
                       arrival ? arrival + base : nullptr, service ? service + base : nullptr,
-                      restore ? restore + base : nullptr)) {
+                      restore ? restore + base : nullptr, n_side, side_pool ? side_pool + base : nullptr,
+                      side_units ? side_units + base : nullptr, (size_t)n_scenarios * max_actions)) {
       status[sc] = STATUS_BAD_ACTION;
       continue;
     }
@@ -752,6 +801,8 @@ int oracle_replay_trace_cache(int n_scenarios, int max_actions, int n_pools, con
         else if (pr.d.type == POOL_GPU) {
           for (const Chunk& c : E[e].chunks) pr.node_busy[c.node] &= (uint8_t)~(((1 << c.size) - 1) << c.start);
         } else if (pr.d.window_us == 0) pr.in_use -= E[e].units;
+        for (const std::pair<int, int>& c : acts[E[e].action].side)  // R26: held until the action ends
+          if (pools[c.first].d.window_us == 0) pools[c.first].in_use -= c.second;
         E.erase(E.begin() + e);
       }
       while (next < n && acts[next].arrival <= now) W.push_back(next++);   // admit arrivals
@@ -788,10 +839,10 @@ int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int
                         int* alloc_units, int* place_node, int* place_off, i64* act_us,
                         i64* total_act_us, int* n_selected, int* status, int* occupancy,
                         int* rounds_used) {
-  return oracle_replay_trace_cache(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, round_us, max_rounds,
+  return oracle_replay_trace_ext(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, round_us, max_rounds,
                                    n_actions, pool, unit, mask, s, p, arrival, gpu_busy, alloc_units, place_node,
                                    place_off, act_us, total_act_us, n_selected, status, occupancy, rounds_used,
-                                   nullptr, nullptr, 0, nullptr, nullptr);
+                                   nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr);
 }
 
 // ---- single pieces, exported so that tests can pin each of them on its own ----------

@@ -22,5 +22,6 @@ from .generator import (  # noqa: F401
     generate,
     random_round,
     contiguous_replica_round,
+    add_side_costs,
     ablation_sweep,
 )

@@ -369,6 +369,34 @@ def random_round(seed: int, n_scenarios: int, max_actions: int, pools: Tuple[Poo
     return w, a
 
 
+def add_side_costs(seed: int, arrays: Dict[str, Optional[np.ndarray]], pools: Tuple[Pool, ...], n_side: int = 2,
+                   fraction: float = 0.5, max_share: float = 0.2, invalid: float = 0.0) -> Dict[str, Optional[np.ndarray]]:
+    """Further entries of the actions' cost vectors (Section 4.1): returns a copy of `arrays` with
+    "side_pool" (uint8, 0xff = none) and "side_units" (uint16), both [n_side][scenario][action].  An entry
+    names a quota / concurrency pool other than the action's own with an amount of up to max_share of its
+    capacity; `invalid` is the probability of an entry being drawn without these restrictions."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    S, N = arrays["pool"].shape
+    api = [j for j, p in enumerate(pools) if p.type == POOL_API]
+    sp = np.full((n_side, S, N), 0xFF, np.uint8)
+    su = np.zeros((n_side, S, N), np.uint16)
+    caps = np.array([p.capacity for p in pools], dtype=np.int64)
+    for e in range(n_side):
+        if not api:
+            break
+        k = np.array(api, dtype=np.int64)[rng.integers(0, len(api), size=(S, N))]
+        on = (rng.random((S, N)) < fraction) & (k != arrays["pool"])
+        amount = 1 + (rng.random((S, N)) * np.maximum(caps[k] * max_share - 1, 0)).astype(np.int64)
+        wild = rng.random((S, N)) < invalid
+        k = np.where(wild, rng.integers(0, len(pools) + 1, size=(S, N)), k)
+        amount = np.where(wild, rng.integers(0, 3, size=(S, N)) * caps[np.minimum(k, len(pools) - 1)], amount)
+        sp[e] = np.where(on | wild, k, 0xFF).astype(np.uint8)
+        su[e] = np.where(on | wild, np.minimum(amount, 65535), 0).astype(np.uint16)
+    out = dict(arrays)
+    out["side_pool"], out["side_units"] = sp, su
+    return out
+
+
 def contiguous_replica_round(seed: int, n_scenarios: int, max_actions: int, nodes: int, max_mult: int,
                              *, small_durations: float = 0.0, busy_fraction: float = 0.3
                              ) -> Tuple[Workload, Dict[str, Optional[np.ndarray]]]:
