@@ -97,7 +97,9 @@ typedef struct {
                               instances every GPU remembers, 0 .. 4; 0 = no cache (then `service`,
                               `restore_us` and the cache arrays of tangram_actions are ignored).
                               Not available with host_buffers = 1.                                 */
-  int32_t reserved;        /* 0                                                                    */
+  int32_t side_costs;      /* further entries of an action's cost vector (Section 4.1, vectorized resource
+                              cost): 0 .. 2; 0 = the key resource only (then `side_pool` / `side_units`
+                              of tangram_actions are ignored).  Not available with host_buffers = 1. */
   const tangram_pool_desc* pools; /* host array of n_pools entries, copied                 */
 } tangram_round_desc;
 
@@ -125,6 +127,17 @@ typedef struct {
   uint32_t* gpu_cache_tag;    /* per scenario [node][8][cache_slots], IN and OUT: instance tag
                                  (service * 8 + log2(chunk size)) + 1, 0 = empty entry           */
   int64_t* gpu_cache_use;     /* same shape, IN and OUT: time of the entry's last use             */
+  /* Cost vector (only read when side_costs > 0; Section 4.1).  Beside its key resource, which alone is
+   * elastic, an action may ask fixed amounts of up to side_costs further pools (memory beside the cores,
+   * the quotas of other sites).  Entry e of action (sc, i) is at [(e * n_scenarios + sc) * max_actions + i].
+   * Such a pool is a quota / concurrency pool (TANGRAM_POOL_API) other than the key pool and the amount
+   * lies in 1 .. its capacity, else the record is bad (TANGRAM_STATUS_BAD_ACTION).  The candidate prefix
+   * (Algorithm 1) ends at the first action whose key request at its least level or one of whose amounts
+   * does not fit on top of the actions before it; what the candidates ask of a pool this way is set aside
+   * before the pool's own actions share it; a started action consumes its amounts (a quota pool counts them
+   * in its window, a concurrency pool holds them until the action ends).                                */
+  const uint8_t* side_pool;   /* [side_costs][scenario][action], may be null (none); 0xff = no entry     */
+  const uint16_t* side_units; /* same shape; ignored where side_pool is 0xff                             */
 } tangram_actions;
 
 /* Results, caller-owned, fully overwritten by a call (rows up to max_actions). */

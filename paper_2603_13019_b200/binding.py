@@ -31,14 +31,15 @@ class _RoundDesc(C.Structure):
     _fields_ = [("n_scenarios", C.c_int32), ("max_actions", C.c_int32), ("n_pools", C.c_int32),
                 ("depth", C.c_int32), ("round_us", C.c_int64), ("max_rounds", C.c_int32),
                 ("host_buffers", C.c_int32), ("workspace_bytes", C.c_int64), ("slot_wait_us", C.c_int64),
-                ("cache_slots", C.c_int32), ("reserved", C.c_int32), ("pools", C.POINTER(_PoolDesc))]
+                ("cache_slots", C.c_int32), ("side_costs", C.c_int32), ("pools", C.POINTER(_PoolDesc))]
 
 
 class _Actions(C.Structure):
     _fields_ = [("pool", C.c_void_p), ("unit", C.c_void_p), ("level_mask", C.c_void_p), ("s_us", C.c_void_p),
                 ("p_us", C.c_void_p), ("arrival_us", C.c_void_p), ("n_actions", C.c_void_p),
                 ("gpu_busy", C.c_void_p), ("service", C.c_void_p), ("restore_us", C.c_void_p),
-                ("gpu_cache_tag", C.c_void_p), ("gpu_cache_use", C.c_void_p)]
+                ("gpu_cache_tag", C.c_void_p), ("gpu_cache_use", C.c_void_p),
+                ("side_pool", C.c_void_p), ("side_units", C.c_void_p)]
 
 
 class _Result(C.Structure):
@@ -102,7 +103,8 @@ def _dtypes():
     import torch
     ins = dict(pool=torch.uint8, unit=torch.uint8, level_mask=torch.int32, s_us=torch.int64,
                p_us=torch.int64, arrival_us=torch.int64, n_actions=torch.int32, gpu_busy=torch.uint8,
-               service=torch.int16, restore_us=torch.int64, cache_tag=torch.int32, cache_use=torch.int64)
+               service=torch.int16, restore_us=torch.int64, cache_tag=torch.int32, cache_use=torch.int64,
+               side_pool=torch.uint8, side_units=torch.int16)
     outs = dict(alloc_units=torch.int32, place_node=torch.int32, place_off=torch.int32,
                 act_us=torch.int64, total_act_us=torch.int64, n_selected=torch.int32,
                 status=torch.int32, occupancy=torch.int32, rounds_used=torch.int32)
@@ -122,15 +124,16 @@ class Round:
 
     def __init__(self, n_scenarios: int, max_actions: int, pools: Sequence, *, depth: int = 2,
                  round_us: int = 10_000, max_rounds: int = 0, host_buffers: bool = False,
-                 workspace_bytes: int = 0, slot_wait_us: int = 0, cache_slots: int = 0):
+                 workspace_bytes: int = 0, slot_wait_us: int = 0, cache_slots: int = 0, side_costs: int = 0):
         self._lib = load_library()
         self._h = None
         self.n_scenarios, self.max_actions, self.pools = int(n_scenarios), int(max_actions), tuple(pools)
         self.max_rounds, self.host_buffers = int(max_rounds), bool(host_buffers)
         self.cache_slots = int(cache_slots)
+        self.side_costs = int(side_costs)
         arr = (_PoolDesc * len(pools))(*[_PoolDesc(p.type, p.capacity, p.group, p.window_us) for p in pools])
         desc = _RoundDesc(n_scenarios, max_actions, len(pools), depth, round_us, max_rounds,
-                          1 if host_buffers else 0, workspace_bytes, slot_wait_us, cache_slots, 0, arr)
+                          1 if host_buffers else 0, workspace_bytes, slot_wait_us, cache_slots, side_costs, arr)
         h = C.c_void_p()
         _check(self._lib.tangram_round_create(C.byref(desc), C.byref(h)))
         self._h = h
@@ -156,12 +159,17 @@ class Round:
         ncache = self.n_scenarios * nodes * 8 * self.cache_slots
         sizes = dict(pool=SN, unit=SN, level_mask=SN, s_us=SN, p_us=SN, arrival_us=SN,
                      n_actions=self.n_scenarios, gpu_busy=self.n_scenarios * nodes,
-                     service=SN, restore_us=SN, cache_tag=ncache, cache_use=ncache)
-        on = self.cache_slots > 0                         # the cache columns are only handed over when a cache exists
-        return _Actions(*[self._ptr(k, a.get(k) if (on or k not in ("service", "restore_us", "cache_tag", "cache_use")) else None,
-                                    ins[k], sizes[k]) for k in
+                     service=SN, restore_us=SN, cache_tag=ncache, cache_use=ncache,
+                     side_pool=SN * self.side_costs, side_units=SN * self.side_costs)
+        # the cache and cost-vector columns are only handed over when the round was created with them
+        off = set()
+        if self.cache_slots == 0:
+            off |= {"service", "restore_us", "cache_tag", "cache_use"}
+        if self.side_costs == 0:
+            off |= {"side_pool", "side_units"}
+        return _Actions(*[self._ptr(k, None if k in off else a.get(k), ins[k], sizes[k]) for k in
                           ("pool", "unit", "level_mask", "s_us", "p_us", "arrival_us", "n_actions", "gpu_busy",
-                           "service", "restore_us", "cache_tag", "cache_use")])
+                           "service", "restore_us", "cache_tag", "cache_use", "side_pool", "side_units")])
 
     def new_result(self, replay: bool = False) -> Dict:
         """Output tensors of the right shapes (device, or pinned host in host-buffer mode)."""
@@ -284,7 +292,7 @@ def schedule_batch_static(pools: Sequence, actions: Dict, result: Dict, *, depth
         if t is not None and not (t.is_cuda and t.is_contiguous()):
             raise TangramError(f"{k}: a contiguous device tensor is required")
     a = _Actions(*([ptr(actions.get(k)) for k in
-                    ("pool", "unit", "level_mask", "s_us", "p_us", "arrival_us", "n_actions", "gpu_busy")] + [None] * 4))
+                    ("pool", "unit", "level_mask", "s_us", "p_us", "arrival_us", "n_actions", "gpu_busy")] + [None] * 6))
     r = _Result(*[ptr(result.get(k)) for k in
                   ("alloc_units", "place_node", "place_off", "act_us", "total_act_us", "n_selected", "status",
                    "occupancy", "rounds_used")])

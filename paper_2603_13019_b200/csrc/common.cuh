@@ -50,6 +50,10 @@ struct Params {
   const int* n_actions; const u8* gpu_busy;
   // service cache of the GPU pools (cache_slots = 0: none)
   const unsigned short* a_service; const i64* a_restore; u32* cache_tag; i64* cache_use; int cache_slots;
+  // further entries of the cost vectors (n_side = 0: none): entry e of (scenario, action) at e * side_plane + row + i
+  int n_side; const u8* a_side_pool; const unsigned short* a_side_units; u64 side_plane;
+  int* side_bad;     // [S] an entry of the scenario names no usable pool or amount
+  int* side_res;     // [S][P] what the candidates ask of a pool beside their key resource
   // outputs (device)
   int* o_alloc; int* o_node; int* o_off; i64* o_act; i64* o_total; int* o_nsel; int* o_status;
   // workspace

@@ -44,6 +44,26 @@ __device__ __forceinline__ int warp_incl_scan32(int x, int lane) {
   return x;
 }
 
+// Further entries of the cost vectors (Section 4.1): an entry has to name a quota / concurrency pool other
+// than the action's key pool and an amount of 1 .. its capacity.  One thread per action; a scenario with
+// a bad entry is flagged for k_head, which then decides nothing of it.
+__global__ void __launch_bounds__(256) k_side_check(const __grid_constant__ Params P) {
+  const size_t total = (size_t)P.S * P.N;
+  for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (size_t)gridDim.x * blockDim.x) {
+    const int sc = (int)(o / P.N), i = (int)(o - (size_t)sc * P.N);
+    if (i >= min(max(P.n_actions[sc], 0), P.N)) continue;
+    bool bad = false;
+    for (int e = 0; e < P.n_side; ++e) {
+      const int k = P.a_side_pool[e * P.side_plane + o];
+      if (k == 0xff) continue;
+      const int c = P.a_side_units[e * P.side_plane + o];
+      bad |= k >= P.P || P.pool[k < P.P ? k : 0].type != TG_POOL_API || k == P.a_pool[o] || c < 1 ||
+             c > P.pool[k < P.P ? k : 0].capacity;
+    }
+    if (bad) P.side_bad[sc] = 1;
+  }
+}
+
 __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, HeadState* hst) {
   const int lane = threadIdx.x & 31;
   const int sc = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
@@ -56,6 +76,7 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
   // lane v < D: capacity, running least-level demand and candidates' largest-level demand of slot v
   // lane j < P: actions / candidates / first waiting action of pool j, and the pool's description
   int capreg = 0, run = 0, mxd = 0, cnt = 0, mreg = 0, fwreg = -1;
+  int sres = 0;                                     // lane v: what the candidates ask of slot v beside their key resource
   u32 pinfo = 0;                                    // type | GPUs per node << 4 | slot0 << 8
   for (int j = 0; j < P.P; ++j) {
     const PoolDev& pd = P.pool[j];
@@ -96,19 +117,31 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
     const int rmin = __ffs(eff), rmax = 32 - __clz(eff);
     const int units = g * rmin, mxu = g * rmax;
     const int lz = gpu ? level_of(g, gang, rmin) : 0, lzx = gpu ? level_of(g, gang, rmax) : 0;
+    // further entries of the cost vector: the slot they charge and the amount (slot -1: none)
+    int ss0 = -1, su0 = 0, ss1 = -1, su1 = 0;
+    if (P.n_side > 0) {
+      int k0 = 0xff, k1 = 0xff;
+      if (present) {
+        k0 = P.a_side_pool[row + i]; su0 = P.a_side_units[row + i];
+        if (P.n_side > 1) { k1 = P.a_side_pool[P.side_plane + row + i]; su1 = P.a_side_units[P.side_plane + row + i]; }
+      }
+      const u32 p0 = __shfl_sync(TG_FULL, pinfo, k0 < P.P ? k0 : 0), p1 = __shfl_sync(TG_FULL, pinfo, k1 < P.P ? k1 : 0);
+      if (valid && k0 < P.P) ss0 = p0 >> 8;
+      if (valid && k1 < P.P) ss1 = p1 >> 8;
+    }
     // least-level demand: one scan per slot; the first action that overflows a slot ends the prefix
     // First the chunk's total per slot (one warp reduction each): only the chunk in which a slot
     // overflows needs the scans that tell which action does it.
     int tot_mine = 0;                                  // lane v: the chunk's demand on slot v
     for (int v = 0; v < D; ++v) {
-      const int c = (valid && v >= slot0 && v <= slot0 + lz) ? units : 0;
+      const int c = ((valid && v >= slot0 && v <= slot0 + lz) ? units : 0) + (ss0 == v ? su0 : 0) + (ss1 == v ? su1 : 0);
       const int tot = __reduce_add_sync(TG_FULL, c);
       if (lane == v) tot_mine = tot;
     }
     bool over = false;
     if (__any_sync(TG_FULL, lane < D && run + tot_mine > capreg)) {
       for (int v = 0; v < D; ++v) {
-        const int c = (valid && v >= slot0 && v <= slot0 + lz) ? units : 0;
+        const int c = ((valid && v >= slot0 && v <= slot0 + lz) ? units : 0) + (ss0 == v ? su0 : 0) + (ss1 == v ? su1 : 0);
         const int incl = warp_incl_scan32(c, lane);
         const int rv = __shfl_sync(TG_FULL, run, v), cv = __shfl_sync(TG_FULL, capreg, v);
         over |= c > 0 && rv + incl > cv;
@@ -131,9 +164,11 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
       if (eff & (eff - 1)) el |= 1u << j;
     }
     for (int v = 0; v < D; ++v) {
-      const int c = (cand && v >= slot0 && v <= slot0 + lzx) ? mxu : 0;
+      const int sd = cand ? (ss0 == v ? su0 : 0) + (ss1 == v ? su1 : 0) : 0;
+      const int c = ((cand && v >= slot0 && v <= slot0 + lzx) ? mxu : 0) + sd;
       const int tot = __reduce_add_sync(TG_FULL, c);
       if (lane == v) mxd += tot;
+      if (P.n_side > 0) { const int st = __reduce_add_sync(TG_FULL, sd); if (lane == v) sres += st; }
     }
     if (ob) {
       // The prefix is complete.  A pool may need its waiting list only if one of its candidates
@@ -165,7 +200,11 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
       if (((elw >> jj) & 1u) && (unfit & slots)) need |= 1u << jj;
     }
   }
-  const int anybad = __any_sync(TG_FULL, bad) ? 1 : 0;
+  const int anybad = (__any_sync(TG_FULL, bad) || (P.n_side > 0 && P.side_bad[sc])) ? 1 : 0;
+  if (P.n_side > 0) {
+    const int sr = __shfl_sync(TG_FULL, sres, lane < P.P ? P.pool[lane].slot0 : 0);
+    if (lane < P.P) P.side_res[(size_t)sc * P.P + lane] = sr;
+  }
   if (lane < P.P) {
     PoolMeta mt;
     mt.base = (i64)sc * (P.P - 1) * P.N + (i64)lane * P.N;   // row + base = prow + lane * N

@@ -42,8 +42,9 @@ __device__ __forceinline__ int pool_busy_units(const Params& P, const ReplayWs& 
 
 // Candidate prefix of the waiting queue (Algorithm 1, line 2) against the pools' current state.
 // dem / cap: 4 ints per pool in the warp's scratch.  Warp-uniform result.
+// aside: per pool, what the candidates ask of it beside their key resource (cost vectors).
 __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const int* wait, int nw,
-                             int* dem, int* cap, int lane) {
+                             int* dem, int* cap, int* aside, int lane) {
   const size_t row = (size_t)sc * P.N;
   for (int j = 0; j < P.P; ++j) {
     const PoolDev& pd = P.pool[j];
@@ -59,14 +60,20 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
     }
     if (lane < 4) { cap[j * 4 + lane] = c[lane]; dem[j * 4 + lane] = 0; }
   }
+  if (lane < TG_MAX_POOLS) aside[lane] = 0;
   __syncwarp();
   int n = 0;
   bool stop = false;
   for (int i0 = 0; i0 < nw && !stop; i0 += 32) {
     // every lane decodes one waiting action, then the 32 are admitted one after the other
     int j = 0, lz = 0, units = 0;
+    int k0 = 0xff, u0 = 0, k1 = 0xff, u1 = 0;            // further entries of the cost vector
     if (i0 + lane < nw) {
       const int a = wait[i0 + lane];
+      if (P.n_side > 0) {
+        k0 = P.a_side_pool[row + a]; u0 = P.a_side_units[row + a];
+        if (P.n_side > 1) { k1 = P.a_side_pool[P.side_plane + row + a]; u1 = P.a_side_units[P.side_plane + row + a]; }
+      }
       j = P.a_pool[row + a];
       int g, gang; u32 eff;
       decode_levels(P.pool[j], P.a_unit[row + a], P.a_mask[row + a], g, gang, eff);
@@ -79,9 +86,20 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
       const int bj = __shfl_sync(TG_FULL, j, b), bl = __shfl_sync(TG_FULL, lz, b), bu = __shfl_sync(TG_FULL, units, b);
       bool over = false;
       for (int l = 0; l <= bl; ++l) over |= dem[bj * 4 + l] + bu > cap[bj * 4 + l];
+      int a0 = 0xff, c0 = 0, a1 = 0xff, c1 = 0;
+      if (P.n_side > 0) {
+        a0 = __shfl_sync(TG_FULL, k0, b); c0 = __shfl_sync(TG_FULL, u0, b);
+        a1 = __shfl_sync(TG_FULL, k1, b); c1 = __shfl_sync(TG_FULL, u1, b);
+        if (a0 != 0xff) over |= dem[a0 * 4] + c0 > cap[a0 * 4];
+        if (a1 != 0xff) over |= dem[a1 * 4] + c1 + (a1 == a0 ? c0 : 0) > cap[a1 * 4];
+      }
       if (over) { stop = true; break; }
       __syncwarp();
       if (lane <= bl) dem[bj * 4 + lane] += bu;
+      if (lane == 0) {
+        if (a0 != 0xff) { dem[a0 * 4] += c0; aside[a0] += c0; }
+        if (a1 != 0xff) { dem[a1 * 4] += c1; aside[a1] += c1; }
+      }
       __syncwarp();
       ++n;
     }
@@ -93,7 +111,7 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
 // actions that sit on pool j), placement on the pool's live state, start of what was selected.
 // Appends the started actions to run[] (nr updated).  Returns false if the scratch ran out.
 __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, const int* wait, int nw, int n,
-                            int* run, int& nr, i64 now, Slab slab, int lane, int& busy_units) {
+                            int* run, int& nr, i64 now, Slab slab, int lane, int& busy_units, int aside_j) {
   const size_t row = (size_t)sc * P.N;
   const PoolDev& pd = P.pool[j];
   // members of the pool among the candidates (m) and behind them (n_ac)
@@ -166,7 +184,7 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
       T.cap[0] = warp_sum32(f);
     } else {
       const int* ps = R.pst + ((size_t)sc * P.P + j) * 2;
-      T.cap[0] = pd.capacity - (pd.window_us > 0 ? ps[0] : ps[1]);
+      T.cap[0] = pd.capacity - (pd.window_us > 0 ? ps[0] : ps[1]) - aside_j;   // set aside for the other pools' candidates
     }
     T.m = m; T.cs = C.cs; T.cp = C.cp; T.cmask = C.cmask; T.cg = C.cg;
     T.n_ac = n_ac; T.ac_tmin = ac_tmin;
@@ -228,7 +246,7 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
 // Blocks of KR_THREADS threads: a scenario is a long chain of dependent steps on one warp, so the warps
 // are spread over as many SMs (and schedulers) as possible instead of sharing one.
 #define KR_THREADS 64
-#define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 256) + 16)
+#define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 288) + 16)
 __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * KR_THREADS + threadIdx.x) >> 5;
@@ -248,6 +266,13 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
       const int j = P.a_pool[row + i];
       int g, gang; u32 eff;
       if (j >= P.P || !decode_levels(P.pool[j], P.a_unit[row + i], P.a_mask[row + i], g, gang, eff)) status |= TG_ST_BAD_ACTION;
+      for (int e = 0; e < P.n_side; ++e) {                  // further entries: a quota / concurrency pool other than j, 1 .. capacity
+        const int k = P.a_side_pool[e * P.side_plane + row + i];
+        if (k == 0xff) continue;
+        const int c = P.a_side_units[e * P.side_plane + row + i];
+        if (k >= P.P || P.pool[k < P.P ? k : 0].type != TG_POOL_API || k == j || c < 1 || c > P.pool[k < P.P ? k : 0].capacity)
+          status |= TG_ST_BAD_ACTION;
+      }
       if (i > 0 && P.a_arrival && P.a_arrival[row + i - 1] > P.a_arrival[row + i]) status |= TG_ST_UNSORTED;
     }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(TG_FULL, status, o);
@@ -272,8 +297,9 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
     int rounds = 0;
     if (status == 0) {
       extern __shared__ __align__(16) unsigned char k2_smem[];
-      int* dem = (int*)(k2_smem + (KR_THREADS / 32) * WARP_SMEM_BYTES + 16) + (threadIdx.x >> 5) * 64;   // 4 ints per pool: demand, capacity
+      int* dem = (int*)(k2_smem + (KR_THREADS / 32) * WARP_SMEM_BYTES + 16) + (threadIdx.x >> 5) * 72;   // 4 ints per pool: demand, capacity
       int* cap = dem + 32;
+      int* aside = cap + 32;                              // 1 int per pool
       int next = 0, nw = 0, nr = 0, r = 0;
       bool drained = false;
       // units in use per core / GPU pool, kept up to date by what starts and what is released
@@ -307,6 +333,11 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
             const int fa = __shfl_sync(TG_FULL, a, b);
             const int j = P.a_pool[row + fa];
             const PoolDev& pd = P.pool[j];
+            if (P.n_side > 0 && lane == 0)                 // a concurrency pool held the action's further amounts until now
+              for (int e = 0; e < P.n_side; ++e) {
+                const int k = P.a_side_pool[e * P.side_plane + row + fa];
+                if (k != 0xff && P.pool[k].window_us == 0) R.pst[((size_t)sc * P.P + k) * 2 + 1] -= P.a_side_units[e * P.side_plane + row + fa];
+              }
             if (pd.type == TG_POOL_API) { if (pd.window_us == 0 && lane == 0) R.pst[((size_t)sc * P.P + j) * 2 + 1] -= P.o_alloc[row + fa]; }
             else {
               const int freed = P.o_alloc[row + fa];
@@ -348,17 +379,28 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
         __syncwarp();
         // 4. schedule
         if (nw > 0) {
-          const int n = replay_prefix(P, R, sc, wait, nw, dem, cap, lane);
+          const int n = replay_prefix(P, R, sc, wait, nw, dem, cap, aside, lane);
           const int nr0 = nr;
           bool ok = true;
           if (n > 0)
             for (int j = 0; j < P.P && ok; ++j) {
               int add = 0;
-              ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add);
+              ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add, aside[j]);
 #pragma unroll
               for (int jj = 0; jj < TG_MAX_POOLS; ++jj) if (jj == j) busy[jj] += add;
             }
           if (!ok) { if (lane == 0) P.o_status[sc] |= TG_ST_WORKSPACE; break; }
+          if (P.n_side > 0 && nr > nr0) {                   // the started actions consume their further amounts
+            __syncwarp();
+            for (int i = nr0 + lane; i < nr; i += 32)
+              for (int e = 0; e < P.n_side; ++e) {
+                const int k = P.a_side_pool[e * P.side_plane + row + run[i]];
+                if (k != 0xff)
+                  atomicAdd(&R.pst[((size_t)sc * P.P + k) * 2 + (P.pool[k].window_us > 0 ? 0 : 1)],
+                            (int)P.a_side_units[e * P.side_plane + row + run[i]]);
+              }
+            __syncwarp();
+          }
           if (nr > nr0) {                                   // drop the started actions from the queue
             int kw = 0;
             for (int i0 = 0; i0 < nw; i0 += 32) {

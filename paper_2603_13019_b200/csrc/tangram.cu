@@ -102,6 +102,7 @@ __device__ void make_task(const Params& P, int sc, int j, const PoolMeta& mt, co
   T.type = pd.type; T.group = pd.group;
   T.cap[0] = pd.capacity; T.cap[1] = T.cap[2] = T.cap[3] = 0;
   if (pd.type == TG_POOL_GPU) gpu_caps(pd, busy_row, lane, T.cap);
+  if (P.n_side > 0 && pd.type == TG_POOL_API) T.cap[0] -= P.side_res[(size_t)sc * P.P + j];   // set aside for the other pools' candidates
   T.m = mt.m; T.cs = C.cs; T.cp = C.cp; T.cmask = C.cmask; T.cg = C.cg;
   T.n_ac = with_waiting ? mt.count - mt.m : 0;
   T.ac_tmin = P.tmin + row + mt.base + mt.m;
@@ -451,7 +452,7 @@ struct tangram_round {
   int64_t launches;
   // workspace
   void* d_order; void* d_tmin; void* d_meta; void* d_slabs; void* d_arena; void* d_arena_top;
-  HeadState* hst; void* d_preq; void* d_keepn; int* d_fl; u32* d_ok_table;
+  HeadState* hst; void* d_preq; void* d_keepn; int* d_fl; u32* d_ok_table; int* d_side_bad; int* d_side_res;
   BatchWs W; int sim_blocks; SimLists L; int n_sm;
   ReplayWs R;
   // host-buffer mode: copy-in, kernels and copy-out of successive chunks on streams of their own
@@ -560,7 +561,8 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
       desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->max_rounds < 0 ||
       desc->round_us < 0 || desc->workspace_bytes < 0 || desc->slot_wait_us < 0 || desc->cache_slots < 0 ||
-      desc->cache_slots > 4 || (desc->cache_slots > 0 && desc->host_buffers))
+      desc->cache_slots > 4 || (desc->cache_slots > 0 && desc->host_buffers) || desc->side_costs < 0 ||
+      desc->side_costs > 2 || (desc->side_costs > 0 && desc->host_buffers))
     return TANGRAM_EINVAL;
   if ((int64_t)desc->n_scenarios * desc->max_actions > (int64_t)1 << 31) return TANGRAM_EINVAL;
   tangram_round* r = new (std::nothrow) tangram_round();
@@ -633,6 +635,10 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   bad |= cudaMalloc((void**)&r->d_preq, SC * sizeof(unsigned short)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->d_keepn, (size_t)P.S * P.P * sizeof(int)) != cudaSuccess;
   bad |= cudaMalloc((void**)&r->d_fl, ((size_t)P.S * P.P + 2) * sizeof(int)) != cudaSuccess;
+  if (desc->side_costs > 0) {                              // cost vectors: flags and set-aside amounts
+    bad |= cudaMalloc((void**)&r->d_side_bad, (size_t)P.S * sizeof(int)) != cudaSuccess;
+    bad |= cudaMalloc((void**)&r->d_side_res, (size_t)P.S * P.P * sizeof(int)) != cudaSuccess;
+  }
   const long long n_sims = (long long)P.P * P.S * 2;
   r->sim_blocks = (int)((n_sims + 31) / 32);
   r->n_sm = prop.multiProcessorCount;
@@ -732,6 +738,8 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   }
   P.order = (int*)r->d_order; P.tmin = (i64*)r->d_tmin; P.meta = (PoolMeta*)r->d_meta;
   P.preq = (unsigned short*)r->d_preq; P.keepn = (int*)r->d_keepn;
+  P.n_side = desc->side_costs; P.side_plane = (u64)P.S * P.N;
+  P.side_bad = r->d_side_bad; P.side_res = r->d_side_res;
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
@@ -799,7 +807,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
-  cudaFree(r->d_ok_table); cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl);
+  cudaFree(r->d_ok_table); cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl); cudaFree(r->d_side_bad); cudaFree(r->d_side_res);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
@@ -876,6 +884,8 @@ static void bind_device_io(Params& P, const tangram_actions* a, const tangram_re
   P.gpu_busy = P.n_nodes_total ? a->gpu_busy : nullptr;
   P.a_service = a->service; P.a_restore = (const i64*)a->restore_us;
   P.cache_tag = a->gpu_cache_tag; P.cache_use = (i64*)a->gpu_cache_use;
+  P.a_side_pool = a->side_pool; P.a_side_units = a->side_units;
+  if (!a->side_pool) P.n_side = 0;                         // no entries handed over: the key resource only
   P.o_alloc = res->alloc_units; P.o_node = res->place_node; P.o_off = res->place_off;
   P.o_act = (i64*)res->act_us; P.o_total = (i64*)res->total_act_us;
   P.o_nsel = res->n_selected; P.o_status = res->status;
@@ -888,6 +898,13 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
   const long long n_sims = (long long)P.P * P.S * 2;
   CK(cudaMemsetAsync(P.arena_top, 0, 256, st));          // arena top and the task counters
   if (ev) CK(cudaEventRecord(ev[0], st));
+  if (P.n_side > 0) {
+    CK(cudaMemsetAsync(P.side_bad, 0, (size_t)P.S * sizeof(int), st));
+    size_t blocks = ((size_t)P.S * P.N + 255) / 256;
+    if (blocks > (size_t)r->n_sm * 16) blocks = (size_t)r->n_sm * 16;
+    k_side_check<<<(unsigned)blocks, 256, 0, st>>>(P);
+    r->launches += 1;
+  }
   k_head<<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[1], st));
   const unsigned place_grid = ((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS;
@@ -953,6 +970,7 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
                                       tangram_result* res, void* cuda_stream) {
   if (!r || !check_io(a, res)) return TANGRAM_EINVAL;
   if (r->desc.cache_slots > 0 && r->P.n_nodes_total > 0 && (!a->gpu_cache_tag || !a->gpu_cache_use)) return TANGRAM_EINVAL;
+  if (r->desc.side_costs > 0 && (!a->side_pool) != (!a->side_units)) return TANGRAM_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   Params P = r->P;
   P.now = now_us;
@@ -1011,6 +1029,7 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
                                     void* cuda_stream) {
   if (!r || !check_io(a, res) || r->desc.max_rounds <= 0 || !a->arrival_us) return TANGRAM_EINVAL;
   if (r->desc.cache_slots > 0 && r->P.n_nodes_total > 0 && (!a->gpu_cache_tag || !a->gpu_cache_use)) return TANGRAM_EINVAL;
+  if (r->desc.side_costs > 0 && (!a->side_pool) != (!a->side_units)) return TANGRAM_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   Params P = r->P;
   P.now = 0;
@@ -1079,7 +1098,7 @@ extern "C" int tangram_schedule_batch_static(const tangram_round_desc* desc, con
   if (!desc || !desc->pools || !check_io(a, res)) return TANGRAM_EINVAL;
   if (desc->n_scenarios < 1 || desc->max_actions < 1 || desc->n_pools < 1 ||
       desc->n_pools > TANGRAM_MAX_POOLS || desc->depth < 1 || desc->depth > 32 || desc->host_buffers ||
-      desc->cache_slots != 0)
+      desc->cache_slots != 0 || desc->side_costs != 0)
     return TANGRAM_EINVAL;
   if ((int64_t)desc->n_scenarios * desc->max_actions > (int64_t)1 << 31) return TANGRAM_ETOOBIG;
   Params P;

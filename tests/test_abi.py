@@ -41,7 +41,7 @@ def _desc(binding, pools, **kw):
     d = binding._RoundDesc(kw.get("n_scenarios", 4), kw.get("max_actions", 16), kw.get("n_pools", len(pools)),
                            kw.get("depth", 2), kw.get("round_us", 10_000), kw.get("max_rounds", 0),
                            kw.get("host_buffers", 0), kw.get("workspace_bytes", 0), kw.get("slot_wait_us", 0),
-                           kw.get("cache_slots", 0), 0, arr)
+                           kw.get("cache_slots", 0), kw.get("side_costs", 0), arr)
     return d, arr
 
 
@@ -73,6 +73,8 @@ def test_round_create_rejects_bad_descriptions():
     assert create(good, slot_wait_us=-1) == EINVAL
     assert create(good, cache_slots=5) == EINVAL
     assert create(good, cache_slots=1, host_buffers=1) == EINVAL                    # no service cache through host buffers
+    assert create(good, side_costs=3) == EINVAL and create(good, side_costs=-1) == EINVAL
+    assert create(good, side_costs=1, host_buffers=1) == EINVAL                     # no cost vectors through host buffers
     assert create(good, n_scenarios=1 << 20, max_actions=1 << 12) == EINVAL         # more than 2^31 records
     assert create([(1, 24, 3, 0)]) == EINVAL                                        # nodes of 3 GPUs
     assert create([(1, 20, 8, 0)]) == EINVAL                                        # capacity not whole nodes

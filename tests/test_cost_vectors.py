@@ -166,3 +166,67 @@ def test_no_pool_is_overdrawn_and_elastic_actions_still_get_the_spare_units(orac
         side = sum(np.where(sel & (a["side_pool"][e] == j), a["side_units"][e], 0).sum(axis=1) for e in range(2))
         assert np.all(key + side <= POOLS[j].capacity)
     assert np.any(o["n_selected"] < plain["n_selected"])          # the amounts did bind somewhere
+
+
+# ------------------------------------------------------------------ CUDA path against the oracle
+KEYS = ("status", "n_selected", "total_act_us", "alloc_units", "place_node", "place_off", "act_us")
+
+
+def _gpu_round(pools, a, n_side, **kw):
+    import torch
+    from paper_2603_13019_b200 import binding
+    S, N = a["pool"].shape
+    rnd = binding.Round(S, N, pools, side_costs=n_side, **kw)
+    if kw.get("max_rounds", 0) > 0:
+        out = rnd.replay_trace(binding.to_device(a))
+    else:
+        out = rnd.schedule_batch(binding.to_device(a))
+    torch.cuda.synchronize()
+    g = {k: v.cpu().numpy() for k, v in out.items()}
+    rnd.destroy()
+    return g
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(8))
+def test_rounds_with_cost_vectors_match_oracle(oracle, seed):
+    n_side = 1 + seed % 2
+    pools = POOLS if seed < 6 else (Pool(POOL_API, 60, 0, 0), Pool(POOL_CPU, 64, 16), Pool(POOL_API, 30, 0, 50_000))
+    # un-narrowed masks: the quota / concurrency pools get elastic key actions, which share what the
+    # other pools' candidates leave
+    w, a = random_round(700 + seed, 64, [200, 90, 700, 150, 4200, 60, 300, 120][seed], pools, max_mult=4,
+                        narrow=seed % 3 == 0, busy_fraction=0.2 if seed % 2 else 0.0,
+                        small_durations=0.3 if seed == 3 else 0.0)
+    a = add_side_costs(seed, a, pools, n_side=n_side, fraction=0.5, max_share=[0.2, 0.05, 0.02, 0.3][seed % 4],
+                       invalid=0.002 if seed in (1, 5) else 0.0)
+    o = oracle.schedule_batch(pools, a)
+    g = _gpu_round(pools, a, n_side)
+    for k in KEYS:
+        assert np.array_equal(o[k], g[k]), k
+    assert (o["status"] == 0).sum() > 8 and (o["alloc_units"] > 0).sum() > 100
+    if seed in (1, 5):
+        assert (o["status"] == 1).sum() > 0
+
+
+@pytest.mark.gpu
+def test_a_round_created_with_cost_vectors_runs_without_them(oracle):
+    w, a = random_round(11, 16, 100, POOLS, max_mult=4)
+    g = _gpu_round(POOLS, a, 2)                                  # no side arrays handed over
+    o = oracle.schedule_batch(POOLS, a)
+    for k in KEYS:
+        assert np.array_equal(o[k], g[k]), k
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(4))
+def test_traces_with_cost_vectors_match_oracle(oracle, seed):
+    pools = (Pool(POOL_CPU, 32, 8), Pool(POOL_GPU, 32, 8), Pool(POOL_API, 40, 0, 0), Pool(POOL_API, 25, 0, 200_000))
+    w, a = random_round(800 + seed, 12, 160, pools, max_mult=4, narrow=seed % 2 == 0, small_durations=0.2)
+    rng = np.random.default_rng(seed)
+    a["arrival_us"] = np.cumsum(rng.integers(0, 5000, a["pool"].shape), axis=1).astype(np.int64)
+    a = add_side_costs(seed, a, pools, n_side=2, fraction=0.6, max_share=0.3)
+    o = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=1500)
+    g = _gpu_round(pools, a, 2, round_us=10_000, max_rounds=1500)
+    for k in KEYS + ("rounds_used", "occupancy"):
+        assert np.array_equal(o[k], g[k]), k
+    assert (o["alloc_units"] > 0).sum() > 300
