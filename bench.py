@@ -100,10 +100,11 @@ class ClockSampler:
 
 def _oracle_call(w, arrays, lo, hi):
     import oracle
+    K = int(w.params.get("cache_slots", 0))
     if w.replay:
         return oracle.replay_trace(w.pools, arrays, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds,
-                                   lo=lo, hi=hi, want_occupancy=False)
-    return oracle.schedule_batch(w.pools, arrays, depth=w.depth, lo=lo, hi=hi)
+                                   lo=lo, hi=hi, want_occupancy=False, cache_slots=K)
+    return oracle.schedule_batch(w.pools, arrays, depth=w.depth, lo=lo, hi=hi, cache_slots=K)
 
 
 def _oracle_throughput(w, arrays, target_s: float, threads: int):
@@ -165,7 +166,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     if args.steps <= 0:
-        args.steps = 100 if args.config in ("cfg0", "cfg1", "cfg4") and args.impl == "ours" else 5
+        args.steps = 100 if args.config in ("cfg0", "cfg1", "cfg4", "cfg4_vec", "cfg1_cache") and args.impl == "ours" else 5
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     rank = int(os.environ.get("RANK", "0"))
@@ -193,7 +194,9 @@ def main():
     lo = rank * S
     chunk = max(1, min(S, (64 << 20) // N))
     parts = [generate(w, lo + c, lo + min(S, c + chunk)) for c in range(0, S, chunk)]
-    arrays = {k: (None if parts[0][k] is None else np.concatenate([p[k] for p in parts])) for k in parts[0]}
+    # per-action and per-scenario arrays are scenario-major; the cost-vector planes are [entry][scenario][action]
+    arrays = {k: (None if parts[0][k] is None else np.concatenate([p[k] for p in parts], axis=1 if k.startswith("side_") else 0))
+              for k in parts[0]}
     del parts
 
     cpu = None
@@ -205,7 +208,8 @@ def main():
                "one_thread": {"value": v1, "unit": "actions/s", "cores": 1, "sample": sample1}}
 
     dev = binding.to_device(arrays)
-    rnd = binding.Round(S, N, w.pools, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds)
+    extras = dict(cache_slots=int(w.params.get("cache_slots", 0)), side_costs=int(w.params.get("side_costs", 0)))
+    rnd = binding.Round(S, N, w.pools, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds, **extras)
     res = rnd.new_result(replay=w.replay)
     stream = torch.cuda.current_stream()
     if w.replay:                                   # a step of a replay workload = the whole trace
@@ -244,7 +248,7 @@ def main():
 
     # end to end through host buffers (pinned), copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not any(extras.values()):          # cost vectors and the service cache take device buffers only
         hrnd = binding.Round(S, N, w.pools, depth=w.depth, host_buffers=True, round_us=w.round_us,
                              max_rounds=w.max_rounds)
         hin = binding.to_device(arrays, pin=True)

@@ -48,8 +48,39 @@ __device__ __forceinline__ int warp_incl_scan32(int x, int lane) {
 // than the action's key pool and an amount of 1 .. its capacity.  One thread per action; a scenario with
 // a bad entry is flagged for k_head, which then decides nothing of it.
 __global__ void __launch_bounds__(256) k_side_check(const __grid_constant__ Params P) {
-  const size_t total = (size_t)P.S * P.N;
-  for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (size_t)gridDim.x * blockDim.x) {
+  // sixteen consecutive actions of one scenario per thread (128-bit loads) where the rows allow it
+  const bool vec = (P.N % 16 == 0) && (P.side_plane % 16 == 0) &&
+                   ((((size_t)P.a_pool | (size_t)P.a_side_pool) & 15) == 0) && (((size_t)P.a_side_units & 15) == 0);
+  const size_t total = (size_t)P.S * P.N, step = (size_t)gridDim.x * blockDim.x;
+  if (vec) {
+    for (size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x; q < total / 16; q += step) {
+      const size_t o = q * 16;
+      const int sc = (int)(o / P.N), i0 = (int)(o - (size_t)sc * P.N);
+      const int n = min(max(P.n_actions[sc], 0), P.N) - i0;    // records of this group that exist
+      if (n <= 0) continue;
+      bool bad = false;
+      for (int e = 0; e < P.n_side; ++e) {
+        __align__(16) u8 k[16];
+        *(uint4*)k = *(const uint4*)(P.a_side_pool + e * P.side_plane + o);
+        const uint4 kk = *(const uint4*)k;
+        if ((kk.x & kk.y & kk.z & kk.w) == 0xffffffffu) continue;   // no entry in the whole group
+        __align__(16) unsigned short c[16];
+        __align__(16) u8 kp[16];
+        *(uint4*)c = *(const uint4*)(P.a_side_units + e * P.side_plane + o);
+        *(uint4*)(c + 8) = *(const uint4*)(P.a_side_units + e * P.side_plane + o + 8);
+        *(uint4*)kp = *(const uint4*)(P.a_pool + o);
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+          if (x >= n || k[x] == 0xff) continue;
+          const int kx = k[x] < P.P ? k[x] : 0;
+          bad |= k[x] >= P.P || P.pool[kx].type != TG_POOL_API || k[x] == kp[x] || c[x] < 1 || c[x] > P.pool[kx].capacity;
+        }
+      }
+      if (bad) P.side_bad[sc] = 1;
+    }
+    return;
+  }
+  for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += step) {
     const int sc = (int)(o / P.N), i = (int)(o - (size_t)sc * P.N);
     if (i >= min(max(P.n_actions[sc], 0), P.N)) continue;
     bool bad = false;
@@ -64,6 +95,8 @@ __global__ void __launch_bounds__(256) k_side_check(const __grid_constant__ Para
   }
 }
 
+// SIDE: the actions carry further cost-vector entries (Section 4.1); the plain instance keeps its registers.
+template <bool SIDE>
 __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, HeadState* hst) {
   const int lane = threadIdx.x & 31;
   const int sc = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
@@ -95,11 +128,26 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
   const u32 lt = (1u << lane) - 1u;
   // the records of the next chunk are loaded while this one is worked on
   int nj = 0; u32 nun = 0, nmk = 0; i64 ns = 0, np_ = 0;
+  int nk0 = 0xff, nu0 = 0, nk1 = 0xff, nu1 = 0;    // further entries of the cost vectors
+  if (SIDE && lane < n_act) {
+    nk0 = P.a_side_pool[row + lane]; nu0 = P.a_side_units[row + lane];
+    if (P.n_side > 1) { nk1 = P.a_side_pool[P.side_plane + row + lane]; nu1 = P.a_side_units[P.side_plane + row + lane]; }
+  }
   if (lane < n_act) { nj = P.a_pool[row + lane]; nun = P.a_unit[row + lane]; nmk = P.a_mask[row + lane]; ns = P.a_s[row + lane]; np_ = P.a_p[row + lane]; }
   for (int c0 = 0; c0 < n_act; c0 += 32) {
     const int i = c0 + lane;
     const bool present = i < n_act;
     const int j = nj; const u32 un = nun, mk = nmk; const i64 s = ns, p = np_;
+    const int k0 = nk0, k1 = nk1;
+    int su0 = nu0, su1 = nu1;
+    if (SIDE) {
+      const int i2 = i + 32;
+      nk0 = 0xff; nk1 = 0xff; nu0 = 0; nu1 = 0;
+      if (i2 < n_act) {
+        nk0 = P.a_side_pool[row + i2]; nu0 = P.a_side_units[row + i2];
+        if (P.n_side > 1) { nk1 = P.a_side_pool[P.side_plane + row + i2]; nu1 = P.a_side_units[P.side_plane + row + i2]; }
+      }
+    }
     {
       const int i2 = i + 32;
       nj = 0; nun = 0; nmk = 0; ns = 0; np_ = 0;
@@ -118,13 +166,8 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
     const int units = g * rmin, mxu = g * rmax;
     const int lz = gpu ? level_of(g, gang, rmin) : 0, lzx = gpu ? level_of(g, gang, rmax) : 0;
     // further entries of the cost vector: the slot they charge and the amount (slot -1: none)
-    int ss0 = -1, su0 = 0, ss1 = -1, su1 = 0;
-    if (P.n_side > 0) {
-      int k0 = 0xff, k1 = 0xff;
-      if (present) {
-        k0 = P.a_side_pool[row + i]; su0 = P.a_side_units[row + i];
-        if (P.n_side > 1) { k1 = P.a_side_pool[P.side_plane + row + i]; su1 = P.a_side_units[P.side_plane + row + i]; }
-      }
+    int ss0 = -1, ss1 = -1;
+    if (SIDE) {
       const u32 p0 = __shfl_sync(TG_FULL, pinfo, k0 < P.P ? k0 : 0), p1 = __shfl_sync(TG_FULL, pinfo, k1 < P.P ? k1 : 0);
       if (valid && k0 < P.P) ss0 = p0 >> 8;
       if (valid && k1 < P.P) ss1 = p1 >> 8;
@@ -168,7 +211,7 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
       const int c = ((cand && v >= slot0 && v <= slot0 + lzx) ? mxu : 0) + sd;
       const int tot = __reduce_add_sync(TG_FULL, c);
       if (lane == v) mxd += tot;
-      if (P.n_side > 0) { const int st = __reduce_add_sync(TG_FULL, sd); if (lane == v) sres += st; }
+      if (SIDE) { const int st = __reduce_add_sync(TG_FULL, sd); if (lane == v) sres += st; }
     }
     if (ob) {
       // The prefix is complete.  A pool may need its waiting list only if one of its candidates
@@ -200,8 +243,8 @@ __global__ void __launch_bounds__(256) k_head(const __grid_constant__ Params P, 
       if (((elw >> jj) & 1u) && (unfit & slots)) need |= 1u << jj;
     }
   }
-  const int anybad = (__any_sync(TG_FULL, bad) || (P.n_side > 0 && P.side_bad[sc])) ? 1 : 0;
-  if (P.n_side > 0) {
+  const int anybad = (__any_sync(TG_FULL, bad) || (SIDE && P.side_bad[sc])) ? 1 : 0;
+  if (SIDE) {
     const int sr = __shfl_sync(TG_FULL, sres, lane < P.P ? P.pool[lane].slot0 : 0);
     if (lane < P.P) P.side_res[(size_t)sc * P.P + lane] = sr;
   }

@@ -905,7 +905,8 @@ static int run_pipeline(tangram_round* r, const Params& P, const BatchWs& W, con
     k_side_check<<<(unsigned)blocks, 256, 0, st>>>(P);
     r->launches += 1;
   }
-  k_head<<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
+  if (P.n_side > 0) k_head<true><<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
+  else k_head<false><<<(P.S + 7) / 8, 256, 0, st>>>(P, r->hst);
   if (ev) CK(cudaEventRecord(ev[1], st));
   const unsigned place_grid = ((P.S + 31) / 32 * P.P + KPL_WARPS - 1) / KPL_WARPS;
   {                                                        // the output fill runs beside everything that follows

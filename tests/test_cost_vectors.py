@@ -230,3 +230,16 @@ def test_traces_with_cost_vectors_match_oracle(oracle, seed):
     for k in KEYS + ("rounds_used", "occupancy"):
         assert np.array_equal(o[k], g[k]), k
     assert (o["alloc_units"] > 0).sum() > 300
+
+
+@pytest.mark.gpu
+def test_cfg4_with_cost_vectors_matches_oracle(oracle):
+    from workloads import generate, make_workload
+    w = make_workload("cfg4_vec", n_scenarios=48)
+    a = generate(w)
+    o = oracle.schedule_batch(w.pools, a, depth=w.depth)
+    g = _gpu_round(w.pools, a, 2, depth=w.depth)
+    for k in KEYS:
+        assert np.array_equal(o[k], g[k]), k
+    plain = oracle.schedule_batch(w.pools, {k: v for k, v in a.items() if not k.startswith("side_")}, depth=w.depth)
+    assert (o["n_selected"] < plain["n_selected"]).sum() > 10      # the memory pool ends many prefixes early

@@ -184,3 +184,23 @@ def test_traces_with_a_service_cache_match_oracle(oracle, seed):
     for k in CACHE_KEYS + ("rounds_used", "occupancy"):
         assert np.array_equal(o[k], g[k]), k
     assert (o["alloc_units"] > 0).sum() > 800 and np.all(o["status"] == 0)
+
+
+@pytest.mark.gpu
+def test_cfg1_with_a_service_cache_matches_oracle(oracle):
+    import torch
+    from paper_2603_13019_b200 import binding
+    from workloads import generate, make_workload
+    w = make_workload("cfg1_cache", n_scenarios=96)
+    a = generate(w)
+    o = oracle.schedule_batch(w.pools, a, depth=w.depth, cache_slots=2)
+    rnd = binding.Round(96, w.max_actions, w.pools, depth=w.depth, cache_slots=2)
+    dev = binding.to_device(a)
+    out = rnd.schedule_batch(dev)
+    torch.cuda.synchronize()
+    g = {k: v.cpu().numpy() for k, v in out.items()}
+    g["cache_tag"] = dev["cache_tag"].cpu().numpy().view(np.uint32)
+    g["cache_use"] = dev["cache_use"].cpu().numpy()
+    rnd.destroy()
+    for k in CACHE_KEYS:
+        assert np.array_equal(o[k], g[k]), k

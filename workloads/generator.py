@@ -93,6 +93,7 @@ class _Draws:
 # fixed field ids (two consecutive ids are consumed by a normal draw)
 _F_POOL, _F_INEL, _F_LEVEL, _F_S, _F_P, _F_OUT, _F_SIZE, _F_ARR, _F_DUR, _F_BUSY = (
     1, 2, 3, 4, 6, 8, 9, 10, 11, 12)
+_F_MEM, _F_TOKEN, _F_SERVICE, _F_RESTORE, _F_CTAG, _F_CUSE = 40, 41, 42, 43, 44, 45
 
 
 def _pow2_mask(max_level: int) -> int:
@@ -256,6 +257,19 @@ CONFIGS: Dict[str, Workload] = {
 }
 
 
+# cfg4 with cost vectors (Section 4.1): a concurrency pool of 2048 memory units is added; every action of
+# the core pool asks 1 .. 32 units of it beside its cores, and three in ten GPU actions one token of the
+# second quota pool (a tool call made while the service runs)
+CONFIGS["cfg4_vec"] = Workload("cfg4_vec", 16384, 4096, CONFIGS["cfg4"].pools + (Pool(POOL_API, 2048, 0, 0),), "mixed",
+                               params=dict(CONFIGS["cfg4"].params, mix=(0.50, 0.25, 0.15, 0.10, 0.0), side_costs=2,
+                                           mem_pool=4, mem_max=32, token_pool=3, token_fraction=0.3))
+# cfg1 with the service cache of the GPU pool (Section 5.3): 6 services (24 instances with the four chunk sizes), every GPU remembers two instances,
+# restoration takes 0.5 .. 4 s, two thirds of the entries start filled
+CONFIGS["cfg1_cache"] = Workload("cfg1_cache", 4096, 1024, CONFIGS["cfg1"].pools, "mixed",
+                                 params=dict(CONFIGS["cfg1"].params, cache_slots=2, n_services=6,
+                                             restore_lo_us=500_000.0, restore_hi_us=4_000_000.0, cache_fill=0.67))
+
+
 def _ablation(dop: int, cores: int = 256, rate_per_s: float = 110.0, name: Optional[str] = None) -> Workload:
     return Workload(name or ("abl_dop%d" % dop if dop else "abl_elastic"), 64, 4000, (Pool(POOL_CPU, cores, _CPU_NUMA),),
                     "ablation", replay=True, max_rounds=12_000,
@@ -308,6 +322,29 @@ def generate(w: Workload, lo: int = 0, hi: Optional[int] = None) -> Dict[str, Op
     for k in ("pool", "unit", "level_mask", "s_us", "p_us", "arrival_us"):
         if a[k] is not None:
             a[k] = np.ascontiguousarray(a[k])
+    P = w.params
+    if P.get("side_costs", 0):                       # further entries of the cost vectors
+        ptype = np.array([p.type for p in w.pools], dtype=np.int64)[a["pool"]]
+        sp = np.full((int(P["side_costs"]), S, N), 0xFF, np.uint8)
+        su = np.zeros((int(P["side_costs"]), S, N), np.uint16)
+        cpu = ptype == POOL_CPU
+        sp[0] = np.where(cpu, P["mem_pool"], 0xFF)
+        su[0] = np.where(cpu, 1 + (d.uniform(_F_MEM) * P["mem_max"]).astype(np.int64), 0)
+        tok = (ptype == POOL_GPU) & (d.uniform(_F_TOKEN) < P["token_fraction"])
+        sp[1] = np.where(tok, P["token_pool"], 0xFF)
+        su[1] = np.where(tok, 1, 0)
+        a["side_pool"], a["side_units"] = sp, su
+    if P.get("cache_slots", 0):                      # services and the cache state of the GPU pools
+        K = int(P["cache_slots"])
+        a["service"] = (d.uniform(_F_SERVICE) * P["n_services"]).astype(np.uint16)
+        a["restore_us"] = (P["restore_lo_us"] + d.uniform(_F_RESTORE) * (P["restore_hi_us"] - P["restore_lo_us"])).astype(np.int64)
+        # a node's GPUs start with the same instances (what earlier whole-node or aligned runs left behind)
+        dc = _Draws(w.base_seed, lo, hi, w.n_nodes * K, salt=7)
+        inst = (dc.uniform(_F_CTAG) * P["n_services"]).astype(np.int64) * 8 + (dc.bits(_F_SERVICE) % _U(4)).astype(np.int64)
+        tag = np.where(dc.uniform(_F_CUSE) < P["cache_fill"], inst + 1, 0).astype(np.uint32)
+        use = -(dc.bits(_F_CUSE + 1) % _U(1_000_000)).astype(np.int64)
+        per_gpu = lambda x: np.ascontiguousarray(np.broadcast_to(x.reshape(S, w.n_nodes, 1, K), (S, w.n_nodes, 8, K))).reshape(S, -1)
+        a["cache_tag"], a["cache_use"] = per_gpu(tag), per_gpu(use)
     return a
 
 
