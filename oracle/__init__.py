@@ -162,6 +162,69 @@ def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, de
     return out
 
 
+def _record_args(arrays, sl):
+    return (_c(arrays["pool"][sl], np.uint8), _c(arrays["unit"][sl], np.uint8), _c(arrays["level_mask"][sl], np.uint32),
+            _c(arrays["s_us"][sl], np.int64), _c(arrays["p_us"][sl], np.int64),
+            _c(arrays["arrival_us"][sl], np.int64) if arrays.get("arrival_us") is not None else None,
+            _c(arrays["n_actions"][sl], np.int32))
+
+
+def order_queue(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], policy: int) -> np.ndarray:
+    """Permutation [scenario][position] -> action index that sorts every queue by the policy's key
+    (1: shortest least-level duration, 2: longest, 3: earliest arrival), equal keys in queue order."""
+    S, N = arrays["pool"].shape
+    pool, unit, mask, s, p, arr, n_act = _record_args(arrays, slice(0, S))
+    perm = np.empty((S, N), np.int32)
+    pf = _pools_flat(pools)
+    rc = lib().oracle_order_queue(C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), _p(n_act, C.c_int),
+                                  _p(pool, C.c_uint8), _p(unit, C.c_uint8), _p(mask, C.c_uint32), _p(s, C.c_longlong),
+                                  _p(p, C.c_longlong), _p(arr, C.c_longlong), C.c_int(policy), _p(perm, C.c_int))
+    assert rc == 0
+    return perm
+
+
+def schedule_batch_ordered(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], policy: int, *, depth: int = 2,
+                           now_us: int = 0) -> Dict[str, np.ndarray]:
+    """One round on every queue sorted by `policy`; results at the actions' own positions."""
+    S, N = arrays["pool"].shape
+    pool, unit, mask, s, p, arr, n_act = _record_args(arrays, slice(0, S))
+    busy = _c(arrays["gpu_busy"], np.uint8) if arrays.get("gpu_busy") is not None else None
+    out = dict(
+        alloc_units=np.empty((S, N), np.int32), place_node=np.empty((S, N), np.int32),
+        place_off=np.empty((S, N), np.int32), act_us=np.empty((S, N), np.int64),
+        total_act_us=np.empty(S, np.int64), n_selected=np.empty(S, np.int32), status=np.empty(S, np.int32))
+    pf = _pools_flat(pools)
+    rc = lib().oracle_schedule_batch_ordered(
+        C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), C.c_int(depth), C.c_int(_n_nodes(pools)),
+        _p(n_act, C.c_int), _p(pool, C.c_uint8), _p(unit, C.c_uint8), _p(mask, C.c_uint32), _p(s, C.c_longlong),
+        _p(p, C.c_longlong), _p(arr, C.c_longlong), _p(busy, C.c_uint8), C.c_longlong(now_us), C.c_int(policy),
+        _p(out["alloc_units"], C.c_int), _p(out["place_node"], C.c_int), _p(out["place_off"], C.c_int),
+        _p(out["act_us"], C.c_longlong), _p(out["total_act_us"], C.c_longlong), _p(out["n_selected"], C.c_int),
+        _p(out["status"], C.c_int))
+    assert rc == 0
+    return out
+
+
+def pin_trajectories(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], traj_node: np.ndarray,
+                     node_mem_free: np.ndarray) -> Dict[str, np.ndarray]:
+    """Pins the trajectories of every queue to CPU nodes (arrays "trajectory" int32, "traj_mem" uint32).
+    Returns pool (the rewritten column), n_admitted and the updated state (copies)."""
+    S, N = arrays["pool"].shape
+    pool, unit, mask, s, p, arr, n_act = _record_args(arrays, slice(0, S))
+    traj = _c(arrays["trajectory"], np.int32)
+    mem = _c(arrays["traj_mem"], np.uint32)
+    tn = np.array(traj_node, dtype=np.int32, order="C", copy=True)
+    mf = np.array(node_mem_free, dtype=np.int64, order="C", copy=True)
+    out = dict(pool=np.empty((S, N), np.uint8), n_admitted=np.empty(S, np.int32), traj_node=tn, node_mem_free=mf)
+    pf = _pools_flat(pools)
+    rc = lib().oracle_pin_trajectories(
+        C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), _p(n_act, C.c_int), _p(pool, C.c_uint8),
+        _p(unit, C.c_uint8), _p(mask, C.c_uint32), _p(traj, C.c_int), _p(mem, C.c_uint32), C.c_int(tn.shape[1]),
+        _p(tn, C.c_int), _p(mf, C.c_longlong), _p(out["pool"], C.c_uint8), _p(out["n_admitted"], C.c_int))
+    assert rc == 0
+    return out
+
+
 # ------------------------------------------------------------------ single pieces
 def duration(s: int, p: int, r: int) -> int:
     return int(lib().oracle_duration(int(s), int(p), int(r)))

@@ -78,6 +78,16 @@
 //       consumes nothing.  They are booked after all pools have placed their key grants, so
 //       a quota pool's place_off counts what was used before the round plus the key grants
 //       ahead in queue order.
+//   R27 Other queue orders (Section 4.2: the algorithm works with other ordering algorithms): the
+//       waiting queue is sorted by a key before the round -- shortest or longest duration at the
+//       least level (Eq. 1), or earliest arrival -- equal keys in queue order; everything after
+//       that is Algorithm 1 on the sorted queue.  An invalid record has key 0.
+//   R28 Per-node CPU scheduling (Section 5.2): every CPU pool is one node with a scheduler of its
+//       own.  In queue order, the first action of a trajectory pins it: among the nodes with at
+//       least as many cores as the action's least level and at least the trajectory's memory
+//       free, the one with the most free memory (lowest index on ties) takes the trajectory and
+//       sets its memory aside; all its actions run there.  An action whose trajectory finds no
+//       node ends the admitted queue (first come first served: what stands behind it waits).
 //
 // The paper prints no worked example of a schedule.  estimate() and the eviction loop are
 // heuristics; they are pinned by closed forms, by an independent list-scheduling statement
@@ -843,6 +853,122 @@ int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int
                                    n_actions, pool, unit, mask, s, p, arrival, gpu_busy, alloc_units, place_node,
                                    place_off, act_us, total_act_us, n_selected, status, occupancy, rounds_used,
                                    nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr);
+}
+
+// R27: permutation that sorts every scenario's queue by the policy's key (1: shortest least-level
+// duration first, 2: longest first, 3: earliest arrival first; anything else: queue order), equal keys
+// in queue order.  perm[sc][k] = index of the action at position k; positions >= n_actions: k itself.
+int oracle_order_queue(int n_scenarios, int max_actions, int n_pools, const int* pools_flat, const int* n_actions,
+                       const uint8_t* pool, const uint8_t* unit, const uint32_t* mask, const i64* s, const i64* p,
+                       const i64* arrival, int policy, int* perm) {
+  std::vector<PoolDesc> pd(n_pools);
+  for (int j = 0; j < n_pools; ++j)
+    pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
+  for (int sc = 0; sc < n_scenarios; ++sc) {
+    size_t base = (size_t)sc * max_actions;
+    int n = n_actions[sc];
+    std::vector<i64> key(n, 0);
+    for (int i = 0; i < n; ++i) {
+      Action a = decode_action(pool[base + i], unit[base + i], mask[base + i], s[base + i], p[base + i],
+                               arrival ? arrival[base + i] : 0, pd);
+      if (policy == 1 || policy == 2) key[i] = a.valid ? duration(a, a.r.front()) : 0;
+      if (policy == 2) key[i] = -key[i];
+      if (policy == 3) key[i] = a.arrival;
+    }
+    std::vector<int> idx(n);
+    for (int i = 0; i < n; ++i) idx[i] = i;
+    std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return key[x] < key[y]; });
+    for (int k = 0; k < max_actions; ++k) perm[base + k] = k < n ? idx[k] : k;
+  }
+  return 0;
+}
+
+// One round on the queue sorted by `policy` (R27); results are indexed by the actions' own positions.
+int oracle_schedule_batch_ordered(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+                                  int depth, int n_nodes, const int* n_actions, const uint8_t* pool,
+                                  const uint8_t* unit, const uint32_t* mask, const i64* s, const i64* p,
+                                  const i64* arrival, const uint8_t* gpu_busy, i64 now, int policy,
+                                  int* alloc_units, int* place_node, int* place_off, i64* act_us,
+                                  i64* total_act_us, int* n_selected, int* status) {
+  std::vector<PoolDesc> pd(n_pools);
+  for (int j = 0; j < n_pools; ++j)
+    pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
+  std::vector<int> perm((size_t)n_scenarios * max_actions);
+  oracle_order_queue(n_scenarios, max_actions, n_pools, pools_flat, n_actions, pool, unit, mask, s, p, arrival,
+                     policy, perm.data());
+  for (int sc = 0; sc < n_scenarios; ++sc) {
+    size_t base = (size_t)sc * max_actions;
+    int n = n_actions[sc];
+    for (int i = 0; i < max_actions; ++i) {
+      alloc_units[base + i] = 0; place_node[base + i] = -1; place_off[base + i] = -1; act_us[base + i] = -1;
+    }
+    total_act_us[sc] = 0; n_selected[sc] = 0; status[sc] = STATUS_OK;
+    std::vector<Action> acts;
+    if (!load_actions(acts, n, pd, pool + base, unit + base, mask + base, s + base, p + base,
+                      arrival ? arrival + base : nullptr)) {
+      status[sc] = STATUS_BAD_ACTION;
+      continue;
+    }
+    std::vector<PoolRuntime> pools = fresh_pools(pd, gpu_busy ? gpu_busy + (size_t)sc * n_nodes : nullptr);
+    std::vector<int> W(perm.begin() + base, perm.begin() + base + n);
+    std::vector<Running> E;
+    std::vector<Grant> grants = schedule_round(pools, acts, W, E, now, depth);
+    for (const Grant& g : grants) {
+      const Action& a = acts[g.action];
+      alloc_units[base + g.action] = g.units;
+      place_node[base + g.action] = g.node;
+      place_off[base + g.action] = g.off;
+      i64 act = (now - a.arrival) + duration(a, g.r);
+      act_us[base + g.action] = act;
+      total_act_us[sc] = sat_add(total_act_us[sc], act);
+      n_selected[sc]++;
+    }
+  }
+  return 0;
+}
+
+// R28: pins the trajectories of every scenario's queue to CPU nodes (= CPU pools).  trajectory: per
+// action, -1 = not tied to a trajectory (the action keeps its pool); traj_mem: memory of the whole
+// trajectory, read at the action that pins it.  traj_node [scenario][max_traj] (-1: not pinned) and
+// node_mem_free [scenario][pool] (entries of CPU pools) are state, in and out.  pool_out gets the
+// pool column with every trajectory action moved to its node; n_admitted the length of the queue
+// up to the first action whose trajectory found no node.
+int oracle_pin_trajectories(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+                            const int* n_actions, const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
+                            const int* trajectory, const uint32_t* traj_mem, int max_traj,
+                            int* traj_node, i64* node_mem_free, uint8_t* pool_out, int* n_admitted) {
+  std::vector<PoolDesc> pd(n_pools);
+  for (int j = 0; j < n_pools; ++j)
+    pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
+  for (int sc = 0; sc < n_scenarios; ++sc) {
+    size_t base = (size_t)sc * max_actions;
+    int* tn = traj_node + (size_t)sc * max_traj;
+    i64* mf = node_mem_free + (size_t)sc * n_pools;
+    int n = n_actions[sc], adm = n;
+    for (int i = 0; i < max_actions; ++i) pool_out[base + i] = pool[base + i];
+    for (int i = 0; i < n; ++i) {
+      int t = trajectory[base + i];
+      if (t < 0 || t >= max_traj) continue;
+      if (pool[base + i] >= n_pools || pd[pool[base + i]].type != POOL_CPU) continue;   // not an action of the CPU manager
+      if (tn[t] < 0) {
+        // least level of the action in cores: g times its smallest multiplicity
+        int g = unit[base + i] & 0x7F, rmin = 0;
+        for (int r = 1; r <= 32 && !rmin; ++r) if (mask[base + i] >> (r - 1) & 1u) rmin = r;
+        i64 need = (i64)g * rmin;
+        int best = -1;
+        for (int j = 0; j < n_pools; ++j) {
+          if (pd[j].type != POOL_CPU || pd[j].capacity < need || mf[j] < (i64)traj_mem[base + i]) continue;
+          if (best < 0 || mf[j] > mf[best]) best = j;
+        }
+        if (best < 0) { adm = i; break; }
+        tn[t] = best;
+        mf[best] -= traj_mem[base + i];
+      }
+      pool_out[base + i] = (uint8_t)tn[t];
+    }
+    n_admitted[sc] = adm;
+  }
+  return 0;
 }
 
 // ---- single pieces, exported so that tests can pin each of them on its own ----------

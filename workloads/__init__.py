@@ -23,5 +23,6 @@ from .generator import (  # noqa: F401
     random_round,
     contiguous_replica_round,
     add_side_costs,
+    add_trajectories,
     ablation_sweep,
 )

@@ -434,6 +434,26 @@ def add_side_costs(seed: int, arrays: Dict[str, Optional[np.ndarray]], pools: Tu
     return out
 
 
+def add_trajectories(seed: int, arrays: Dict[str, Optional[np.ndarray]], pools: Tuple[Pool, ...], max_traj: int,
+                     fraction: float = 0.9, mem_hi: int = 64, pinned: float = 0.3,
+                     mem_free_hi: int = 600) -> Dict[str, Optional[np.ndarray]]:
+    """Trajectories for the per-node CPU scheduling (Section 5.2): returns a copy of `arrays` with "trajectory"
+    (int32 per action, -1 = none), "traj_mem" (uint32, memory of the whole trajectory), and the state
+    "traj_node" ([scenario][max_traj], a fraction already pinned to a random CPU pool) and "node_mem_free"
+    ([scenario][pool])."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    S, N = arrays["pool"].shape
+    cpu = np.array([j for j, p in enumerate(pools) if p.type == POOL_CPU], dtype=np.int64)
+    traj = np.where(rng.random((S, N)) < fraction, rng.integers(0, max_traj, size=(S, N)), -1).astype(np.int32)
+    per_traj_mem = rng.integers(0, mem_hi + 1, size=(S, max_traj))
+    mem = np.take_along_axis(per_traj_mem, np.maximum(traj, 0).astype(np.int64), axis=1).astype(np.uint32)
+    node = np.where(rng.random((S, max_traj)) < pinned, cpu[rng.integers(0, len(cpu), size=(S, max_traj))], -1).astype(np.int32)
+    out = dict(arrays)
+    out["trajectory"], out["traj_mem"], out["traj_node"] = traj, mem, node
+    out["node_mem_free"] = rng.integers(0, mem_free_hi + 1, size=(S, len(pools))).astype(np.int64)
+    return out
+
+
 def contiguous_replica_round(seed: int, n_scenarios: int, max_actions: int, nodes: int, max_mult: int,
                              *, small_durations: float = 0.0, busy_fraction: float = 0.3
                              ) -> Tuple[Workload, Dict[str, Optional[np.ndarray]]]:
