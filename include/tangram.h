@@ -213,6 +213,50 @@ void tangram_round_destroy(tangram_round* round);
 /* Launches of this library's kernels since the round was created (for accounting). */
 int64_t tangram_kernel_launches(const tangram_round* round);
 
+/* Other queue orders (Section 4.2: first come first served is the paper's choice against starvation, and
+ * "the algorithm can work with other ordering algorithms").  policy: 1 = shortest duration at the least
+ * level first (Eq. 1), 2 = longest first, 3 = earliest arrival first; equal keys keep their queue order; a
+ * record that no pool can serve has key 0.
+ *
+ * tangram_order_queue writes the permutation: perm[sc * max_actions + k] = index of the action that
+ * stands at position k of the sorted queue (positions >= n_actions[sc]: k).  perm: device, caller-owned.
+ *
+ * tangram_schedule_batch_ordered runs one round (as tangram_schedule_batch) on every queue sorted that way;
+ * results are written at the actions' own positions.  policy 0 is tangram_schedule_batch itself.  Its first
+ * call allocates 54 B per action of device memory that the round keeps (cudaMalloc; TANGRAM_ENOMEM).
+ * Device buffers only; max_actions <= 16384 (TANGRAM_ETOOBIG beyond); not with cache_slots / side_costs
+ * (TANGRAM_EINVAL).  Asynchronous on the stream. */
+#define TANGRAM_ORDER_FCFS 0
+#define TANGRAM_ORDER_SHORTEST 1
+#define TANGRAM_ORDER_LONGEST 2
+#define TANGRAM_ORDER_ARRIVAL 3
+int tangram_order_queue(tangram_round* round, const tangram_actions* actions, int policy, int32_t* perm,
+                        void* cuda_stream);
+int tangram_schedule_batch_ordered(tangram_round* round, const tangram_actions* actions, int policy,
+                                   int64_t now_us, tangram_result* result, void* cuda_stream);
+
+/* Per-node CPU scheduling (Section 5.2, pool in CPU manager): every TANGRAM_POOL_CPU pool of the round is one
+ * node with a scheduler of its own (Algorithm 1 treats the pools independently).  In queue order, the first
+ * action of a trajectory pins it: among the nodes with at least as many cores as the action's least level
+ * (g times its smallest multiplicity) and at least traj_mem free memory, the one with the most free memory
+ * (lowest pool index on ties) takes it and sets the memory aside; every action of a pinned trajectory gets
+ * that node as its pool.  An action whose trajectory finds no node ends the admitted queue: n_admitted is
+ * what to pass as n_actions to the round (first come first served: what stands behind it waits).
+ * Actions with trajectory < 0 or >= max_trajectories, and actions whose pool is not a CPU pool, keep their
+ * pool.  All pointers device memory, caller-owned; traj_node and node_mem_free are state, in and out (the
+ * caller gives memory back when a trajectory ends).  Device buffers only.  Asynchronous on the stream. */
+typedef struct {
+  const int32_t* trajectory;   /* per action [scenario][action]                                          */
+  const uint32_t* traj_mem;    /* per action: memory of the action's whole trajectory                    */
+  int32_t max_trajectories;    /* row length of traj_node                                                */
+  int32_t* traj_node;          /* [scenario][max_trajectories] pool index of the node, -1 = not pinned   */
+  int64_t* node_mem_free;      /* [scenario][n_pools] free memory of every CPU pool (other entries unused) */
+  uint8_t* pool_out;           /* [scenario][action] the pool column with the trajectories' nodes        */
+  int32_t* n_admitted;         /* [scenario]                                                             */
+} tangram_pinning;
+int tangram_pin_trajectories(tangram_round* round, const tangram_actions* actions, const tangram_pinning* pin,
+                             void* cuda_stream);
+
 /* Measurement aid (no counterpart in the paper).  tangram_set_profiling(round, 1) creates CUDA
  * events once; from then on every call records events around each of its kernels on the
  * call's stream (up to 256 calls between two switches).  After the caller has synchronised,

@@ -42,6 +42,12 @@ class _Actions(C.Structure):
                 ("side_pool", C.c_void_p), ("side_units", C.c_void_p)]
 
 
+class _Pinning(C.Structure):
+    _fields_ = [("trajectory", C.c_void_p), ("traj_mem", C.c_void_p), ("max_trajectories", C.c_int32),
+                ("traj_node", C.c_void_p), ("node_mem_free", C.c_void_p), ("pool_out", C.c_void_p),
+                ("n_admitted", C.c_void_p)]
+
+
 class _Result(C.Structure):
     _fields_ = [("alloc_units", C.c_void_p), ("place_node", C.c_void_p), ("place_off", C.c_void_p),
                 ("act_us", C.c_void_p), ("total_act_us", C.c_void_p), ("n_selected", C.c_void_p),
@@ -51,7 +57,8 @@ class _Result(C.Structure):
 EXPORTS = ("tangram_round_create", "tangram_schedule_batch", "tangram_replay_trace",
            "tangram_round_destroy", "tangram_kernel_launches", "tangram_strerror",
            "tangram_last_cuda_error", "tangram_set_profiling", "tangram_kernel_time_ms",
-           "tangram_kernel_name", "tangram_schedule_batch_static")
+           "tangram_kernel_name", "tangram_schedule_batch_static", "tangram_order_queue",
+           "tangram_schedule_batch_ordered", "tangram_pin_trajectories")
 
 
 def load_library(path: Optional[str] = None):
@@ -84,6 +91,13 @@ def load_library(path: Optional[str] = None):
     lib.tangram_kernel_name.restype = C.c_char_p
     lib.tangram_kernel_name.argtypes = [C.c_int]
     lib.tangram_schedule_batch_static.restype = C.c_int
+    lib.tangram_order_queue.restype = C.c_int
+    lib.tangram_order_queue.argtypes = [C.c_void_p, C.POINTER(_Actions), C.c_int, C.c_void_p, C.c_void_p]
+    lib.tangram_schedule_batch_ordered.restype = C.c_int
+    lib.tangram_schedule_batch_ordered.argtypes = [C.c_void_p, C.POINTER(_Actions), C.c_int, C.c_int64,
+                                                   C.POINTER(_Result), C.c_void_p]
+    lib.tangram_pin_trajectories.restype = C.c_int
+    lib.tangram_pin_trajectories.argtypes = [C.c_void_p, C.POINTER(_Actions), C.POINTER(_Pinning), C.c_void_p]
     lib.tangram_schedule_batch_static.argtypes = [C.POINTER(_RoundDesc), C.POINTER(_Actions), C.c_int64,
                                                   C.POINTER(_Result), C.c_void_p]
     if path is None:
@@ -213,6 +227,42 @@ class Round:
         a, r = self._actions(actions), self._result(result)
         _check(self._lib.tangram_replay_trace(self._h, C.byref(a), C.byref(r), self._stream(stream)))
         return result
+
+    def order_queue(self, actions: Dict, policy: int, stream=None):
+        """tangram_order_queue: the permutation that sorts every queue by the policy's key (device int32 [S][N])."""
+        import torch
+        perm = torch.empty((self.n_scenarios, self.max_actions), dtype=torch.int32, device="cuda")
+        a = self._actions(actions)
+        _check(self._lib.tangram_order_queue(self._h, C.byref(a), int(policy), C.c_void_p(perm.data_ptr()),
+                                             self._stream(stream)))
+        return perm
+
+    def schedule_batch_ordered(self, actions: Dict, policy: int, now_us: int = 0, result: Optional[Dict] = None,
+                               stream=None) -> Dict:
+        """tangram_schedule_batch_ordered: one round on every queue sorted by `policy`."""
+        result = self.new_result() if result is None else result
+        a, r = self._actions(actions), self._result(result)
+        _check(self._lib.tangram_schedule_batch_ordered(self._h, C.byref(a), int(policy), int(now_us), C.byref(r),
+                                                        self._stream(stream)))
+        return result
+
+    def pin_trajectories(self, actions: Dict, stream=None) -> Dict:
+        """tangram_pin_trajectories: actions["trajectory"] (int32), ["traj_mem"] (int32 bit pattern of uint32),
+        state ["traj_node"] (int32 [S][T]) and ["node_mem_free"] (int64 [S][P]) are updated in place; returns
+        the rewritten pool column and n_admitted (device tensors)."""
+        import torch
+        S, N = self.n_scenarios, self.max_actions
+        T = actions["traj_node"].shape[1]
+        out = dict(pool=torch.empty((S, N), dtype=torch.uint8, device="cuda"),
+                   n_admitted=torch.empty((S,), dtype=torch.int32, device="cuda"))
+        pin = _Pinning(self._ptr("trajectory", actions["trajectory"], torch.int32, S * N),
+                       self._ptr("traj_mem", actions["traj_mem"], torch.int32, S * N), T,
+                       self._ptr("traj_node", actions["traj_node"], torch.int32, S * T),
+                       self._ptr("node_mem_free", actions["node_mem_free"], torch.int64, S * len(self.pools)),
+                       out["pool"].data_ptr(), out["n_admitted"].data_ptr())
+        a = self._actions(actions)
+        _check(self._lib.tangram_pin_trajectories(self._h, C.byref(a), C.byref(pin), self._stream(stream)))
+        return out
 
     def set_profiling(self, enable: bool):
         """tangram_set_profiling: record CUDA events around every kernel of the following calls."""

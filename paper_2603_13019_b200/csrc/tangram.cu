@@ -10,6 +10,7 @@
 #include "common.cuh"
 #include "prefix_kernel.cuh"
 #include "prefix_stream.cuh"
+#include "order_pin.cuh"
 #include "sims.cuh"
 #include "select.cuh"
 #include "place.cuh"
@@ -464,6 +465,8 @@ struct tangram_round {
   cudaEvent_t sim_fork, sim_join[TG_N_SIM_CLASSES + 1];
   // the certified pools (k_easy and their placement) run beside the kernels that follow k_solve
   cudaStream_t side; cudaEvent_t side_fork, side_join;
+  // sorted copy of the queue and of its results (tangram_schedule_batch_ordered), allocated at its first call
+  char* d_sorted; int* d_perm;
   // staging for host-buffer mode
   char* d_stage; size_t stage_bytes;
   size_t in_off[8], out_off[9];
@@ -807,7 +810,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
-  cudaFree(r->d_ok_table); cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl); cudaFree(r->d_side_bad); cudaFree(r->d_side_res);
+  cudaFree(r->d_ok_table); cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl); cudaFree(r->d_side_bad); cudaFree(r->d_side_res); cudaFree(r->d_sorted); cudaFree(r->d_perm);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
@@ -1062,6 +1065,107 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
     if (res->rounds_used)
       CK(cudaMemcpyAsync(res->rounds_used, r->d_stage + r->out_off[8], (size_t)P.S * sizeof(int), cudaMemcpyDeviceToHost, st));
   }
+  return TANGRAM_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Other queue orders (Section 4.2) and trajectories pinned to CPU nodes (Section 5.2)
+// ---------------------------------------------------------------------------------------
+#define TG_MAX_DEVICES_ORDER 64
+static int next_pow2(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+
+static int launch_order(tangram_round* r, const Params& P, int policy, int* perm, cudaStream_t st) {
+  OrderIo O;
+  O.policy = policy; O.n_pad = next_pow2(P.N); O.perm = perm;
+  const size_t smem = (size_t)O.n_pad * 12;
+  static size_t granted[TG_MAX_DEVICES_ORDER];          // largest dynamic shared memory asked for, per device
+  if (r->device >= 0 && r->device < TG_MAX_DEVICES_ORDER && smem > granted[r->device]) {
+    CK(cudaFuncSetAttribute(k_order, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    granted[r->device] = smem;
+  }
+  k_order<<<P.S, KO_THREADS, smem, st>>>(P, O);
+  r->launches += 1;
+  CK(cudaGetLastError());
+  return TANGRAM_OK;
+}
+
+static bool order_args_ok(const tangram_round* r, const tangram_actions* a, int policy) {
+  return r && a && a->pool && a->unit && a->level_mask && a->s_us && a->p_us && a->n_actions &&
+         policy >= 1 && policy <= 3 && !r->desc.host_buffers;
+}
+
+extern "C" int tangram_order_queue(tangram_round* r, const tangram_actions* a, int policy, int32_t* perm,
+                                   void* cuda_stream) {
+  if (!order_args_ok(r, a, policy) || !perm) return TANGRAM_EINVAL;
+  if (r->P.N > KO_MAX_N) return TANGRAM_ETOOBIG;
+  Params P = r->P;
+  P.a_pool = a->pool; P.a_unit = a->unit; P.a_mask = a->level_mask;
+  P.a_s = (const i64*)a->s_us; P.a_p = (const i64*)a->p_us; P.a_arrival = (const i64*)a->arrival_us;
+  P.n_actions = a->n_actions;
+  return launch_order(r, P, policy, perm, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int tangram_schedule_batch_ordered(tangram_round* r, const tangram_actions* a, int policy, int64_t now_us,
+                                              tangram_result* res, void* cuda_stream) {
+  if (!r || !check_io(a, res)) return TANGRAM_EINVAL;
+  if (policy == 0) return tangram_schedule_batch(r, a, now_us, res, cuda_stream);
+  if (!order_args_ok(r, a, policy) || r->desc.cache_slots > 0 || r->desc.side_costs > 0) return TANGRAM_EINVAL;
+  if (r->P.N > KO_MAX_N) return TANGRAM_ETOOBIG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  Params P = r->P;
+  P.now = now_us;
+  bind_device_io(P, a, res);
+  const size_t SN = (size_t)P.S * P.N;
+  // sorted records (pool, unit, mask, s, p, arrival) and sorted results (alloc, node, off, act): 50 B per action
+  const size_t off_unit = align_up(SN, 256), off_mask = off_unit + align_up(SN, 256), off_s = off_mask + align_up(SN * 4, 256),
+               off_p = off_s + SN * 8, off_arr = off_p + SN * 8, off_alloc = off_arr + SN * 8, off_node = off_alloc + SN * 4,
+               off_off = off_node + SN * 4, off_act = align_up(off_off + SN * 4, 256), total = off_act + SN * 8;
+  if (!r->d_sorted) {
+    if (cudaMalloc((void**)&r->d_sorted, total) != cudaSuccess || cudaMalloc((void**)&r->d_perm, SN * sizeof(int)) != cudaSuccess) {
+      cudaGetLastError();
+      cudaFree(r->d_sorted); cudaFree(r->d_perm); r->d_sorted = nullptr; r->d_perm = nullptr;
+      return TANGRAM_ENOMEM;
+    }
+  }
+  char* d = r->d_sorted;
+  int rc = launch_order(r, P, policy, r->d_perm, st);
+  if (rc) return rc;
+  GatherIo G;
+  G.perm = r->d_perm; G.pool = (u8*)d; G.unit = (u8*)(d + off_unit); G.mask = (u32*)(d + off_mask);
+  G.s = (i64*)(d + off_s); G.p = (i64*)(d + off_p); G.arrival = P.a_arrival ? (i64*)(d + off_arr) : nullptr;
+  size_t blocks = (SN + 255) / 256;
+  if (blocks > (size_t)r->n_sm * 32) blocks = (size_t)r->n_sm * 32;
+  k_gather<<<(unsigned)blocks, 256, 0, st>>>(P, G);
+  // the round itself, on the sorted copy; the per-scenario results go straight to the caller
+  Params Q = P;
+  Q.a_pool = G.pool; Q.a_unit = G.unit; Q.a_mask = G.mask; Q.a_s = G.s; Q.a_p = G.p; Q.a_arrival = G.arrival;
+  Q.o_alloc = (int*)(d + off_alloc); Q.o_node = (int*)(d + off_node); Q.o_off = (int*)(d + off_off); Q.o_act = (i64*)(d + off_act);
+  rc = run_pipeline(r, Q, r->W, r->L, st, nullptr);
+  if (rc) return rc;
+  ScatterIo X;
+  X.perm = r->d_perm; X.alloc = Q.o_alloc; X.node = Q.o_node; X.off = Q.o_off; X.act = Q.o_act;
+  X.o_alloc = P.o_alloc; X.o_node = P.o_node; X.o_off = P.o_off; X.o_act = P.o_act;
+  k_scatter<<<(unsigned)blocks, 256, 0, st>>>(P, X);
+  r->launches += 2;
+  CK(cudaGetLastError());
+  return TANGRAM_OK;
+}
+
+extern "C" int tangram_pin_trajectories(tangram_round* r, const tangram_actions* a, const tangram_pinning* pin,
+                                        void* cuda_stream) {
+  if (!r || !a || !pin || !a->pool || !a->unit || !a->level_mask || !a->n_actions || r->desc.host_buffers ||
+      !pin->trajectory || !pin->traj_mem || pin->max_trajectories < 1 || !pin->traj_node || !pin->node_mem_free ||
+      !pin->pool_out || !pin->n_admitted)
+    return TANGRAM_EINVAL;
+  Params P = r->P;
+  P.a_pool = a->pool; P.a_unit = a->unit; P.a_mask = a->level_mask; P.n_actions = a->n_actions;
+  PinIo X;
+  X.trajectory = pin->trajectory; X.traj_mem = pin->traj_mem; X.max_traj = pin->max_trajectories;
+  X.traj_node = pin->traj_node; X.mem_free = (i64*)pin->node_mem_free; X.pool_out = pin->pool_out;
+  X.n_admitted = pin->n_admitted;
+  k_pin<<<(P.S + 7) / 8, 256, 0, (cudaStream_t)cuda_stream>>>(P, X);
+  r->launches += 1;
+  CK(cudaGetLastError());
   return TANGRAM_OK;
 }
 

@@ -96,8 +96,9 @@ def test_a_trajectory_goes_to_the_node_with_the_most_free_memory_and_stays_there
 
 
 def test_nodes_without_the_cores_or_the_memory_are_filtered_out(oracle):
-    # the action needs at least 4 x 3 = 12 cores: node 0 (8 cores) is out although it has the most memory
-    a = _traj([(0, 4, 0b1100, 100, 0)], [0], [10], [-1], [90, 20, 999, 30])
+    # the action needs at least 4 x 3 = 12 cores (its least level; its largest, 20, fits no node and does not
+    # matter): node 0 (8 cores) is out although it has the most memory
+    a = _traj([(0, 4, 0b11100, 100, 0)], [0], [10], [-1], [90, 20, 999, 30])
     o = oracle.pin_trajectories(NODES, a, a["traj_node"], a["node_mem_free"])
     assert o["pool"][0, 0] == 3 and list(o["node_mem_free"][0]) == [90, 20, 999, 20]
     # the memory of the whole trajectory has to be free: 25 fits node 3 only
@@ -116,3 +117,67 @@ def test_a_trajectory_that_finds_no_node_ends_the_admitted_queue(oracle):
     # trajectory 0 -> node 3 (60 left); trajectory 1 needs 80: nowhere; what stands behind it waits as well
     assert o["n_admitted"][0] == 1 and list(o["traj_node"][0]) == [3, -1, -1]
     assert list(o["pool"][0]) == [3, 0, 0, 0] and list(o["node_mem_free"][0]) == [50, 60, 999, 60]
+
+
+# ------------------------------------------------------------------ CUDA path against the oracle
+KEYS = ("status", "n_selected", "total_act_us", "alloc_units", "place_node", "place_off", "act_us")
+POOLS = (Pool(POOL_CPU, 64, 16), Pool(POOL_GPU, 32, 8), Pool(POOL_API, 40, 0, 0), Pool(POOL_CPU, 32, 8))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed,policy", [(0, SJF), (1, LJF), (2, ARRIVAL), (3, SJF), (4, LJF), (5, SJF)])
+def test_ordered_rounds_match_oracle(oracle, seed, policy):
+    import torch
+    from paper_2603_13019_b200 import binding
+    # 4200 actions: a padded sort of 8192; 33: one of 64; tiny durations: many equal keys
+    N = [300, 4200, 33, 1000, 64, 2048][seed]
+    w, a = random_round(900 + seed, 24, N, POOLS, max_mult=4, narrow=seed != 3, small_durations=0.6 if seed in (0, 4) else 0.0,
+                        busy_fraction=0.2 if seed % 2 else 0.0)
+    a["arrival_us"] = np.random.default_rng(seed).integers(-50, 200, a["pool"].shape).astype(np.int64)
+    o = oracle.schedule_batch_ordered(POOLS, a, policy, now_us=300)
+    operm = oracle.order_queue(POOLS, a, policy)
+    rnd = binding.Round(24, N, POOLS)
+    dev = binding.to_device(a)
+    perm = rnd.order_queue(dev, policy)
+    out = rnd.schedule_batch_ordered(dev, policy, now_us=300)
+    out2 = rnd.schedule_batch_ordered(dev, policy, now_us=300)      # the kept staging is reused
+    torch.cuda.synchronize()
+    assert np.array_equal(operm, perm.cpu().numpy())
+    for res in (out, out2):
+        for k in KEYS:
+            assert np.array_equal(o[k], res[k].cpu().numpy()), k
+    plain = oracle.schedule_batch(POOLS, a, now_us=300)
+    assert not np.array_equal(plain["alloc_units"], o["alloc_units"])
+    rnd.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(5))
+def test_pinned_trajectories_match_oracle(oracle, seed):
+    import torch
+    from paper_2603_13019_b200 import binding
+    N = [200, 1500, 31, 700, 4096][seed]
+    w, a = random_round(950 + seed, 40, N, POOLS, max_mult=4, narrow=seed != 1)
+    a = add_trajectories(seed, a, POOLS, max_traj=[16, 300, 5, 64, 900][seed], mem_hi=[64, 8, 64, 30, 4][seed],
+                         pinned=0.3 if seed != 2 else 0.0)
+    o = oracle.pin_trajectories(POOLS, a, a["traj_node"], a["node_mem_free"])
+    rnd = binding.Round(40, N, POOLS)
+    dev = binding.to_device(a)
+    dev["traj_mem"] = dev["traj_mem"].view(torch.int32) if dev["traj_mem"].dtype != torch.int32 else dev["traj_mem"]
+    out = rnd.pin_trajectories(dev)
+    torch.cuda.synchronize()
+    assert np.array_equal(o["pool"], out["pool"].cpu().numpy())
+    assert np.array_equal(o["n_admitted"], out["n_admitted"].cpu().numpy())
+    assert np.array_equal(o["traj_node"], dev["traj_node"].cpu().numpy())
+    assert np.array_equal(o["node_mem_free"], dev["node_mem_free"].cpu().numpy())
+    if seed != 2:
+        assert (o["n_admitted"] < a["n_actions"]).sum() > 3 and (o["n_admitted"] == a["n_actions"]).sum() > 3
+    # the pinned queue goes through the round: pool column from the pin, queue cut at n_admitted
+    b = dict(a, pool=o["pool"], n_actions=o["n_admitted"])
+    ob = oracle.schedule_batch(POOLS, b)
+    devb = dict(dev, pool=out["pool"], n_actions=out["n_admitted"])
+    g = rnd.schedule_batch(devb)
+    torch.cuda.synchronize()
+    for k in KEYS:
+        assert np.array_equal(ob[k], g[k].cpu().numpy()), k
+    rnd.destroy()
