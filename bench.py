@@ -162,6 +162,8 @@ def main():
     ap.add_argument("--config", default="cfg4", choices=list(CONFIGS))
     ap.add_argument("--scenarios", type=int, default=0, help="override the number of scenarios (smaller runs)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--order", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="queue order of a single-round config: 0 first come first served, 1 shortest first, 2 longest first, 3 arrival")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -200,7 +202,7 @@ def main():
     del parts
 
     cpu = None
-    if rank == 0 and not args.no_cpu_baseline:
+    if rank == 0 and not args.no_cpu_baseline and not args.order:   # the oracle leg times the first-come-first-served round
         threads = os.cpu_count() or 1
         v, sample = _oracle_throughput(w, arrays, 15.0, threads)
         v1, sample1 = _oracle_throughput(w, arrays, 5.0, 1)
@@ -212,6 +214,9 @@ def main():
     rnd = binding.Round(S, N, w.pools, depth=w.depth, round_us=w.round_us, max_rounds=w.max_rounds, **extras)
     res = rnd.new_result(replay=w.replay)
     stream = torch.cuda.current_stream()
+    if args.order and not w.replay:                # the round on the sorted queue (sort, gather, round, scatter)
+        _plain = rnd.schedule_batch
+        rnd.schedule_batch = lambda a_, now_, res_, st_: rnd.schedule_batch_ordered(a_, args.order, now_, res_, st_)
     if w.replay:                                   # a step of a replay workload = the whole trace
         _sb = rnd.schedule_batch
         rnd.schedule_batch = lambda a_, now_, res_, st_: rnd.replay_trace(a_, res_, st_)
@@ -248,7 +253,7 @@ def main():
 
     # end to end through host buffers (pinned), copies inside the timed region
     e2e = None
-    if not args.no_e2e and not any(extras.values()):          # cost vectors and the service cache take device buffers only
+    if not args.no_e2e and not any(extras.values()) and not args.order:          # cost vectors and the service cache take device buffers only
         hrnd = binding.Round(S, N, w.pools, depth=w.depth, host_buffers=True, round_us=w.round_us,
                              max_rounds=w.max_rounds)
         hin = binding.to_device(arrays, pin=True)
@@ -300,6 +305,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
             "config": {"workload": w.name, "scenarios_per_gpu": S, "actions_per_scenario": N,
                        "pools": [[p.type, p.capacity, p.group, p.window_us] for p in w.pools], "depth": w.depth,
+                       "queue_order": args.order,
                        "l2": "inputs+outputs %.0f MB per step, larger than L2" % (ALGO_BYTES_PER_ACTION * S * N / 1e6)
                        if ALGO_BYTES_PER_ACTION * S * N > 126e6 else "working set below L2; no flush",
                        "parallelism": "independent replicas" if world > 1 else "single GPU",

@@ -3,7 +3,7 @@
 // k_order (Section 4.2: Algorithm 1 takes the queue in any order): one CTA per scenario sorts the
 // queue by a policy key -- least-level duration (Eq. 1) ascending or descending, or arrival time --
 // with the queue position as second key, so equal keys keep their order.  Keys and positions live
-// in shared memory (12 B per action, padded to a power of two); the sort is a bitonic network.
+// in shared memory (8 or 12 B per action, padded to a power of two); the sort is a bitonic network.
 // k_gather / k_scatter move the records into sorted order and the results back to the actions' own
 // positions, so the kernels of the round run unchanged on the sorted queue.
 //
@@ -34,17 +34,20 @@ __device__ __forceinline__ i64 warp_max64_from_m1(i64 v) {
 
 __device__ __forceinline__ bool ko_less(u64 ka, u32 ia, u64 kb, u32 ib) { return ka < kb || (ka == kb && ia < ib); }
 
+// WIDE = false: duration keys stay below 2^42 and positions below 2^14, so key and position are one 64-bit
+// word (8 B per action); WIDE = true (arrival times, any 64-bit value): key and position side by side (12 B).
+template <bool WIDE>
 __global__ void __launch_bounds__(KO_THREADS) k_order(const __grid_constant__ Params P, const OrderIo O) {
   extern __shared__ __align__(16) unsigned char ko_smem[];
   u64* key = (u64*)ko_smem;
-  u32* idx = (u32*)(key + O.n_pad);
+  u32* idx = (u32*)(key + O.n_pad);                    // WIDE only
   const int sc = blockIdx.x, t = threadIdx.x;
   const size_t row = (size_t)sc * P.N;
   const int n = min(max(P.n_actions[sc], 0), P.N);
   for (int i = t; i < O.n_pad; i += KO_THREADS) {
     u64 k = ~0ull;                                     // padding and the positions behind the queue stay where they are
     if (i < n) {
-      if (O.policy == 3) k = (u64)(P.a_arrival ? P.a_arrival[row + i] : 0) ^ 0x8000000000000000ull;
+      if (WIDE) k = (u64)(P.a_arrival ? P.a_arrival[row + i] : 0) ^ 0x8000000000000000ull;
       else {
         const int j = P.a_pool[row + i];
         int g, gang; u32 eff;
@@ -54,7 +57,8 @@ __global__ void __launch_bounds__(KO_THREADS) k_order(const __grid_constant__ Pa
         k = O.policy == 2 ? (u64)((1ll << 42) - T) : (u64)T;
       }
     }
-    key[i] = k; idx[i] = (u32)i;
+    if (WIDE) { key[i] = k; idx[i] = (u32)i; }
+    else key[i] = i < n ? (k << 14) | (u64)i : (~0ull << 14) | (u64)i;
   }
   __syncthreads();
   for (int size = 2; size <= O.n_pad; size <<= 1) {
@@ -63,14 +67,16 @@ __global__ void __launch_bounds__(KO_THREADS) k_order(const __grid_constant__ Pa
         // pair (lo, lo + stride); ascending where bit `size` of lo is clear
         const int lo = ((x & ~(stride - 1)) << 1) | (x & (stride - 1)), hi = lo + stride;
         const u64 ka = key[lo], kb = key[hi];
-        const u32 ia = idx[lo], ib = idx[hi];
         const bool up = (lo & size) == 0;
-        if (ko_less(kb, ib, ka, ia) == up) { key[lo] = kb; key[hi] = ka; idx[lo] = ib; idx[hi] = ia; }
+        if (WIDE) {
+          const u32 ia = idx[lo], ib = idx[hi];
+          if (ko_less(kb, ib, ka, ia) == up) { key[lo] = kb; key[hi] = ka; idx[lo] = ib; idx[hi] = ia; }
+        } else if ((kb < ka) == up) { key[lo] = kb; key[hi] = ka; }
       }
       __syncthreads();
     }
   }
-  for (int i = t; i < P.N; i += KO_THREADS) O.perm[row + i] = (int)idx[i];
+  for (int i = t; i < P.N; i += KO_THREADS) O.perm[row + i] = WIDE ? (int)idx[i] : (int)(key[i] & 0x3fffu);
 }
 
 // the record columns in sorted order

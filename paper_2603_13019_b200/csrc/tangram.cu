@@ -1071,19 +1071,16 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
 // ---------------------------------------------------------------------------------------
 // Other queue orders (Section 4.2) and trajectories pinned to CPU nodes (Section 5.2)
 // ---------------------------------------------------------------------------------------
-#define TG_MAX_DEVICES_ORDER 64
 static int next_pow2(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
 static int launch_order(tangram_round* r, const Params& P, int policy, int* perm, cudaStream_t st) {
   OrderIo O;
   O.policy = policy; O.n_pad = next_pow2(P.N); O.perm = perm;
-  const size_t smem = (size_t)O.n_pad * 12;
-  static size_t granted[TG_MAX_DEVICES_ORDER];          // largest dynamic shared memory asked for, per device
-  if (r->device >= 0 && r->device < TG_MAX_DEVICES_ORDER && smem > granted[r->device]) {
-    CK(cudaFuncSetAttribute(k_order, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    granted[r->device] = smem;
-  }
-  k_order<<<P.S, KO_THREADS, smem, st>>>(P, O);
+  const bool wide = policy == 3;
+  const size_t smem = (size_t)O.n_pad * (wide ? 12 : 8);
+  CK(cudaFuncSetAttribute(wide ? k_order<true> : k_order<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  if (wide) k_order<true><<<P.S, KO_THREADS, smem, st>>>(P, O);
+  else k_order<false><<<P.S, KO_THREADS, smem, st>>>(P, O);
   r->launches += 1;
   CK(cudaGetLastError());
   return TANGRAM_OK;
