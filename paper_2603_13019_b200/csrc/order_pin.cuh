@@ -79,6 +79,82 @@ __global__ void __launch_bounds__(KO_THREADS) k_order(const __grid_constant__ Pa
   for (int i = t; i < P.N; i += KO_THREADS) O.perm[row + i] = WIDE ? (int)idx[i] : (int)(key[i] & 0x3fffu);
 }
 
+// The same sort for the duration keys when the padded queue gives every thread EPT >= 1 whole elements
+// (thread t holds positions t * EPT .. t * EPT + EPT - 1 in registers): compare-exchanges at strides below EPT
+// stay inside a thread, strides below 32 * EPT go through warp shuffles, and only the strides beyond that
+// through shared memory (one conflict-free store / load of every element per such stage).
+template <int EPT>
+__global__ void __launch_bounds__(KO_THREADS) k_order_regs(const __grid_constant__ Params P, const OrderIo O) {
+  extern __shared__ __align__(16) unsigned char ko_smem[];
+  u64* sm = (u64*)ko_smem;                             // [EPT][KO_THREADS]
+  const int sc = blockIdx.x, t = threadIdx.x, lane = t & 31;
+  const size_t row = (size_t)sc * P.N;
+  const int n = min(max(P.n_actions[sc], 0), P.N);
+  u64 v[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    const int i = t * EPT + e;
+    u64 k = ~0ull << 14;                               // padding and the positions behind the queue stay where they are
+    if (i < n) {
+      const int j = P.a_pool[row + i];
+      int g, gang; u32 eff;
+      i64 T = 0;                                       // a record no pool can serve has key 0
+      if (j < P.P && decode_levels(P.pool[j], P.a_unit[row + i], P.a_mask[row + i], g, gang, eff))
+        T = duration(clamp_param(P.a_s[row + i]), clamp_param(P.a_p[row + i]), __ffs(eff));
+      k = (O.policy == 2 ? (u64)((1ll << 42) - T) : (u64)T) << 14;
+    }
+    v[e] = k | (u64)i;
+  }
+  for (int size = 2; size <= O.n_pad; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      if (stride < EPT) {
+        // cs is a compile-time copy of the stride, so that v[] stays in registers
+#pragma unroll
+        for (int cs = 1; cs < EPT; cs <<= 1) {
+          if (cs != stride) continue;
+#pragma unroll
+          for (int e = 0; e < EPT; ++e) {
+            if (e & cs) continue;
+            const bool up = ((t * EPT + e) & size) == 0;
+            const u64 a = v[e], b = v[e | cs];
+            if ((b < a) == up) { v[e] = b; v[e | cs] = a; }
+          }
+        }
+      } else if (stride < 32 * EPT) {
+        const int m = stride / EPT;                    // partner lane = lane ^ m
+        const bool lower = (lane & m) == 0;
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) {
+          const u64 o = __shfl_xor_sync(TG_FULL, v[e], m);
+          const bool up = ((t * EPT + e) & size) == 0;
+          const u64 lo_v = o < v[e] ? o : v[e], hi_v = o < v[e] ? v[e] : o;
+          v[e] = (lower == up) ? lo_v : hi_v;
+        }
+      } else {
+        const int m = stride / EPT;                    // partner thread = t ^ m
+        const bool lower = (t & m) == 0;
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) sm[e * KO_THREADS + t] = v[e];
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) {
+          const u64 o = sm[e * KO_THREADS + (t ^ m)];
+          const bool up = ((t * EPT + e) & size) == 0;
+          const u64 lo_v = o < v[e] ? o : v[e], hi_v = o < v[e] ? v[e] : o;
+          v[e] = (lower == up) ? lo_v : hi_v;
+        }
+      }
+    }
+  }
+  // through shared memory once more, so that a warp writes consecutive positions
+  __syncthreads();
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) ((u32*)sm)[t * EPT + e] = (u32)(v[e] & 0x3fffu);
+  __syncthreads();
+  for (int i = t; i < P.N; i += KO_THREADS) O.perm[row + i] = (int)((u32*)sm)[i];
+}
+
 // the record columns in sorted order
 struct GatherIo {
   const int* perm;

@@ -1077,6 +1077,17 @@ static int launch_order(tangram_round* r, const Params& P, int policy, int* perm
   OrderIo O;
   O.policy = policy; O.n_pad = next_pow2(P.N); O.perm = perm;
   const bool wide = policy == 3;
+  if (!wide && O.n_pad >= KO_THREADS) {                  // whole elements per thread: the register version
+    const int ept = O.n_pad / KO_THREADS;
+    const size_t sm = (size_t)O.n_pad * 8;
+    void (*kern)(Params, OrderIo) = ept == 1 ? k_order_regs<1> : ept == 2 ? k_order_regs<2> : ept == 4 ? k_order_regs<4> :
+                                    ept == 8 ? k_order_regs<8> : ept == 16 ? k_order_regs<16> : k_order_regs<32>;
+    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+    kern<<<P.S, KO_THREADS, sm, st>>>(P, O);
+    r->launches += 1;
+    CK(cudaGetLastError());
+    return TANGRAM_OK;
+  }
   const size_t smem = (size_t)O.n_pad * (wide ? 12 : 8);
   CK(cudaFuncSetAttribute(wide ? k_order<true> : k_order<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   if (wide) k_order<true><<<P.S, KO_THREADS, smem, st>>>(P, O);

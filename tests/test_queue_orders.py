@@ -125,12 +125,13 @@ POOLS = (Pool(POOL_CPU, 64, 16), Pool(POOL_GPU, 32, 8), Pool(POOL_API, 40, 0, 0)
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("seed,policy", [(0, SJF), (1, LJF), (2, ARRIVAL), (3, SJF), (4, LJF), (5, SJF)])
+@pytest.mark.parametrize("seed,policy", [(0, SJF), (1, LJF), (2, ARRIVAL), (3, SJF), (4, LJF), (5, SJF), (6, SJF), (7, LJF), (8, ARRIVAL)])
 def test_ordered_rounds_match_oracle(oracle, seed, policy):
     import torch
     from paper_2603_13019_b200 import binding
-    # 4200 actions: a padded sort of 8192; 33: one of 64; tiny durations: many equal keys
-    N = [300, 4200, 33, 1000, 64, 2048][seed]
+    # every tile size of the register sort (1 .. 32 elements per thread), queues below one element per thread,
+    # the wide keys of the arrival order; tiny durations: many equal keys
+    N = [300, 4200, 33, 1000, 64, 2048, 4096, 9000, 5000][seed]
     w, a = random_round(900 + seed, 24, N, POOLS, max_mult=4, narrow=seed != 3, small_durations=0.6 if seed in (0, 4) else 0.0,
                         busy_fraction=0.2 if seed % 2 else 0.0)
     a["arrival_us"] = np.random.default_rng(seed).integers(-50, 200, a["pool"].shape).astype(np.int64)
