@@ -39,8 +39,8 @@ METRIC = "actions scheduled/sec (1xB200)"
 # scenarios); traffic grows in proportion to the actions, so a launch's traffic is this times its actions.
 # The k_stream interval of the per-kernel timing holds k_fill as well (it runs beside it), the k_finish interval
 # k_easy and the certified pools' k_place (beside it), the k_place interval the solver-side pools' placement.
-NCU_BYTES_PER_ACTION = {"cfg4": {"k_head": 1.72, "k_stream": 34.1, "k_solve": 1.54, "k_sims": 2.40,
-                                 "k_finish": 1.88 + 1.91 + 0.53, "k_place": 0.05 + 0.22}}
+NCU_BYTES_PER_ACTION = {"cfg4": {"k_head": 1.72, "k_stream": 11.70 + 22.48, "k_solve": 1.54, "k_sims": 2.46,
+                                 "k_finish": 1.88 + 1.90 + 0.55, "k_place": 0.02 + 0.23}}
 NCU_TRAFFIC_SOURCE = "ncu on 2048 scenarios of the same shape, scaled by actions (profiles/)"
 
 
