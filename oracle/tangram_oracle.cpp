@@ -94,7 +94,12 @@
 // and by cases worked by hand in the tests (two accepted evictions and a refused third,
 // evicted candidates ahead of the waiting list, a running action of the same pool in the
 // heap, saturating sums), DPArrange by exhaustive enumeration, the chunk test by brute-force
-// packing, placement by worked examples.
+// packing, placement by worked examples; the service cache, the cost vectors, the queue orders
+// and the trajectory pinning by hand-worked cases of their own (same-level preference, LRU order,
+// restoration once per action; an amount that ends the prefix, a later candidate's amount set
+// aside, an evicted candidate that consumes nothing, concurrency and quota bookkeeping over
+// rounds; keys and ties of the three orders, the ordered round against the plain round on the
+// permuted records; most-free-memory node, the core and memory filters, the admitted queue).
 #include <algorithm>
 #include <climits>
 #include <cstdint>
