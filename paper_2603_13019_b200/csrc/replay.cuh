@@ -378,8 +378,10 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
         }
         __syncwarp();
         // 4. schedule
+        int blocked_pool = -1;                              // pool of a head-of-line action that does not fit
         if (nw > 0) {
           const int n = replay_prefix(P, R, sc, wait, nw, dem, cap, aside, lane);
+          if (n == 0 && P.n_side == 0) blocked_pool = P.a_pool[row + wait[0]];
           const int nr0 = nr;
           bool ok = true;
           if (n > 0)
@@ -440,6 +442,46 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
               if (occ) occ[(size_t)rr * P.P + j] = v;
             }
           if (r_next > r) r = (int)r_next;
+        } else if (blocked_pool >= 0) {
+          // The action at the head of the queue does not fit its pool, so nothing can start (the prefix is
+          // empty) until that pool changes: an action running on it ends, or its quota window turns.  The
+          // rounds up to then only admit arrivals behind the head and release what ends on other pools;
+          // their occupancy rows follow from the completion times.
+          const PoolDev& hp = P.pool[blocked_pool];
+          i64 t_next = TG_INF;
+          if (hp.type == TG_POOL_API && hp.window_us > 0) t_next = (R.win[(size_t)sc * P.P + blocked_pool] + 1) * (i64)hp.window_us;
+          for (int i = lane; i < nr; i += 32) {
+            const int a = run[i];
+            if (P.a_pool[row + a] == blocked_pool) t_next = min(t_next, (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a]);
+          }
+          t_next = warp_min64(t_next);
+          i64 r_next = t_next == TG_INF ? (i64)R.max_rounds : (t_next + R.round_us - 1) / R.round_us;
+          if (r_next > R.max_rounds) r_next = R.max_rounds;
+          if (r_next > r) {
+            if (occ) {
+              for (i64 rr = r + lane; rr < r_next; rr += 32)
+                for (int j = 0; j < P.P; ++j) {
+                  const PoolDev& pd = P.pool[j];
+                  int v = busy[j];
+                  if (pd.type == TG_POOL_API && pd.window_us > 0 && (rr * R.round_us) / pd.window_us != R.win[(size_t)sc * P.P + j]) v = 0;
+                  occ[(size_t)rr * P.P + j] = v;
+                }
+              __syncwarp();
+              // what ends on the other pools inside the jump leaves the rows from its round on
+              for (int i = lane; i < nr; i += 32) {
+                const int a = run[i];
+                const int j = P.a_pool[row + a];
+                const PoolDev& pd = P.pool[j];
+                if (pd.type == TG_POOL_API && pd.window_us > 0) continue;      // used quota is not given back
+                const i64 fin = (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a];
+                i64 fr = (fin + R.round_us - 1) / R.round_us;
+                if (fr < r) fr = r;
+                for (i64 rr = fr; rr < r_next; ++rr) atomicSub(&occ[(size_t)rr * P.P + j], P.o_alloc[row + a]);
+              }
+              __syncwarp();
+            }
+            r = (int)r_next;
+          }
         }
       }
       rounds = drained ? r : R.max_rounds;

@@ -188,18 +188,22 @@ __device__ int dp_small(const PoolTask& T, int nrows, int ncell, const int ext[4
                      "r"(pa[k]), "r"(pb[k]), "r"((u32)du[k]), "r"((u32)((u64)du[k] >> 32)) : "memory");
       __syncwarp();
       for (int b = 0; b < nb; ++b) {
+        // all level entries of the row are loaded before any is used, and the first four are applied without
+        // a branch: their loads and shuffles do not depend on one another, only the running minimum does
+        u32 va[DPS_LEVELS], vb[DPS_LEVELS], dlo[DPS_LEVELS], dhi[DPS_LEVELS];
+#pragma unroll
+        for (int k = 0; k < DPS_LEVELS; ++k)
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(va[k]), "=r"(vb[k]), "=r"(dlo[k]), "=r"(dhi[k])
+                       : "r"(lists + (u32)(b * DPS_LEVELS + k) * 16u) : "memory");
         i64 best = TG_INF; u32 bestv = 0;
 #pragma unroll
         for (int k = 0; k < DPS_LEVELS; ++k) {
-          u32 va, vb, dlo, dhi;
-          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(va), "=r"(vb), "=r"(dlo), "=r"(dhi)
-                       : "r"(lists + (u32)(b * DPS_LEVELS + k) * 16u) : "memory");
-          if (va == 0) break;                            // the row has no further level (a multiplicity is never 0)
-          const i64 dd = (i64)(((u64)dhi << 32) | dlo);
-          const i64 pv = __shfl_up_sync(TG_FULL, prev, va >> 8);
-          const bool ok = ((pe - vb) & GUARD) == GUARD && pv != TG_INF;
+          if (k >= 4 && va[k] == 0) break;               // the row has no further level (a multiplicity is never 0)
+          const i64 dd = (i64)(((u64)dhi[k] << 32) | dlo[k]);
+          const i64 pv = __shfl_up_sync(TG_FULL, prev, va[k] >> 8);
+          const bool ok = va[k] != 0 && ((pe - vb[k]) & GUARD) == GUARD && pv != TG_INF;
           const i64 cand = pv + dd;
-          if (ok && cand < best) { best = cand; bestv = va; }
+          if (ok && cand < best) { best = cand; bestv = va[k]; }
         }
         prev = lane < ncell ? best : TG_INF;
         asm volatile("st.shared.u16 [%0], %1;" :: "r"(scratch + (u32)(t0 + b) * 64u + (u32)lane * 2u), "h"((unsigned short)bestv) : "memory");
