@@ -42,9 +42,10 @@ __device__ __forceinline__ int pool_busy_units(const Params& P, const ReplayWs& 
 
 // Candidate prefix of the waiting queue (Algorithm 1, line 2) against the pools' current state.
 // dem / cap: 4 ints per pool in the warp's scratch.  Warp-uniform result.
-// aside: per pool, what the candidates ask of it beside their key resource (cost vectors).
+// aside: per pool, what the candidates ask of it beside their key resource (cost vectors);
+// ncand: per pool, how many of the candidates have it as their key pool.
 __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const int* wait, int nw,
-                             int* dem, int* cap, int* aside, int lane) {
+                             int* dem, int* cap, int* aside, int* ncand, int lane) {
   const size_t row = (size_t)sc * P.N;
   for (int j = 0; j < P.P; ++j) {
     const PoolDev& pd = P.pool[j];
@@ -60,7 +61,7 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
     }
     if (lane < 4) { cap[j * 4 + lane] = c[lane]; dem[j * 4 + lane] = 0; }
   }
-  if (lane < TG_MAX_POOLS) aside[lane] = 0;
+  if (lane < TG_MAX_POOLS) { aside[lane] = 0; ncand[lane] = 0; }
   __syncwarp();
   int n = 0;
   bool stop = false;
@@ -97,6 +98,7 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
       __syncwarp();
       if (lane <= bl) dem[bj * 4 + lane] += bu;
       if (lane == 0) {
+        ncand[bj] += 1;
         if (a0 != 0xff) { dem[a0 * 4] += c0; aside[a0] += c0; }
         if (a1 != 0xff) { dem[a1 * 4] += c1; aside[a1] += c1; }
       }
@@ -141,7 +143,7 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
     int a = -1; bool mine = false;
     if (i < nw) { a = wait[i]; mine = P.a_pool[row + a] == j; }
     const u32 bc = __ballot_sync(TG_FULL, mine && i < n), ba = __ballot_sync(TG_FULL, mine && i >= n);
-    if (mine) {
+    if (mine && (i < n || m >= 2)) {                    // (the waiting actions' durations feed the estimate only)
       int g, gang; u32 eff;
       decode_levels(pd, P.a_unit[row + a], P.a_mask[row + a], g, gang, eff);
       const i64 s = clamp_param(P.a_s[row + a]), p = clamp_param(P.a_p[row + a]);
@@ -159,8 +161,9 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
   }
   elastic = __any_sync(TG_FULL, elastic);
   // completion times (relative to now) of what runs on this pool seed the heap
+  // (only an eviction step looks at the heap: with one candidate, or none that is elastic, nobody reads it)
   int ns = 0;
-  for (int i0 = 0; i0 < nr; i0 += 32) {
+  for (int i0 = 0; i0 < nr && elastic && m >= 2; i0 += 32) {
     const int i = i0 + lane;
     int a = -1; bool mine = false;
     if (i < nr) { a = run[i]; mine = P.a_pool[row + a] == j; }
@@ -246,7 +249,7 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
 // Blocks of KR_THREADS threads: a scenario is a long chain of dependent steps on one warp, so the warps
 // are spread over as many SMs (and schedulers) as possible instead of sharing one.
 #define KR_THREADS 64
-#define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 288) + 16)
+#define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 320) + 16)
 __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * KR_THREADS + threadIdx.x) >> 5;
@@ -297,9 +300,10 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
     int rounds = 0;
     if (status == 0) {
       extern __shared__ __align__(16) unsigned char k2_smem[];
-      int* dem = (int*)(k2_smem + (KR_THREADS / 32) * WARP_SMEM_BYTES + 16) + (threadIdx.x >> 5) * 72;   // 4 ints per pool: demand, capacity
+      int* dem = (int*)(k2_smem + (KR_THREADS / 32) * WARP_SMEM_BYTES + 16) + (threadIdx.x >> 5) * 80;   // 4 ints per pool: demand, capacity
       int* cap = dem + 32;
       int* aside = cap + 32;                              // 1 int per pool
+      int* ncand = aside + 8;                             // 1 int per pool
       int next = 0, nw = 0, nr = 0, r = 0;
       bool drained = false;
       // units in use per core / GPU pool, kept up to date by what starts and what is released
@@ -319,10 +323,16 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
         // 2. release what has finished; the running list is compacted in place
         int kept = 0;
         bool gpu_released = false;
+        i64 min_fin = TG_INF;                               // earliest completion among what keeps running
         for (int i0 = 0; i0 < nr; i0 += 32) {
           const int i = i0 + lane;
           int a = -1; bool done = false;
-          if (i < nr) { a = run[i]; done = (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a] <= now; }
+          if (i < nr) {
+            a = run[i];
+            const i64 fin = (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a];
+            done = fin <= now;
+            if (!done) min_fin = min(min_fin, fin);
+          }
           const u32 bd = __ballot_sync(TG_FULL, done), bk = __ballot_sync(TG_FULL, i < nr && !done);
           __syncwarp();
           if (i < nr && !done) run[kept + __popc(bk & ((1u << lane) - 1u))] = a;
@@ -354,6 +364,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
           }
         }
         nr = kept;
+        const int nr_before = nr;
         if (__any_sync(TG_FULL, gpu_released)) {            // node masks follow the owner map
           for (int j = 0; j < P.P; ++j) {
             const PoolDev& pd = P.pool[j];
@@ -380,12 +391,13 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
         // 4. schedule
         int blocked_pool = -1;                              // pool of a head-of-line action that does not fit
         if (nw > 0) {
-          const int n = replay_prefix(P, R, sc, wait, nw, dem, cap, aside, lane);
+          const int n = replay_prefix(P, R, sc, wait, nw, dem, cap, aside, ncand, lane);
           if (n == 0 && P.n_side == 0) blocked_pool = P.a_pool[row + wait[0]];
           const int nr0 = nr;
           bool ok = true;
           if (n > 0)
             for (int j = 0; j < P.P && ok; ++j) {
+              if (ncand[j] == 0) continue;                  // no candidate has this pool as its key pool
               int add = 0;
               ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add, aside[j]);
 #pragma unroll
@@ -425,8 +437,10 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
         if (next == n_act && nw == 0 && nr == 0) { drained = true; break; }
         // with an empty queue nothing happens before the next arrival or completion: jump there
         if (nw == 0) {
+          // (what was running before this round: the release scan's minimum; what started in it: the tail of the list)
           i64 t_next = next < n_act ? (P.a_arrival ? P.a_arrival[row + next] : 0) : TG_INF;
-          for (int i = lane; i < nr; i += 32) {
+          t_next = min(t_next, min_fin);
+          for (int i = nr_before + lane; i < nr; i += 32) {
             const int a = run[i];
             t_next = min(t_next, (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a]);
           }
