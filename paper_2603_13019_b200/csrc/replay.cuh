@@ -113,16 +113,16 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
 // actions that sit on pool j), placement on the pool's live state, start of what was selected.
 // Appends the started actions to run[] (nr updated).  Returns false if the scratch ran out.
 __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, const int* wait, int nw, int n,
-                            int* run, int& nr, i64 now, Slab slab, int lane, int& busy_units, int aside_j) {
+                            int* run, int& nr, i64 now, Slab slab, int lane, int& busy_units, int aside_j, int m) {
   const size_t row = (size_t)sc * P.N;
   const PoolDev& pd = P.pool[j];
-  // members of the pool among the candidates (m) and behind them (n_ac)
-  int m = 0, n_ac = 0;
-  for (int i0 = 0; i0 < nw; i0 += 32) {
+  // m: members of the pool among the candidates (counted by the prefix); n_ac: members behind them, which
+  // only an eviction step's estimate looks at (a single candidate is never evicted)
+  int n_ac = 0;
+  for (int i0 = n & ~31; i0 < nw && m >= 2; i0 += 32) {
     const int i = i0 + lane;
-    const bool mine = i < nw && P.a_pool[row + wait[i]] == j;
-    m += __popc(__ballot_sync(TG_FULL, mine && i < n));
-    n_ac += __popc(__ballot_sync(TG_FULL, mine && i >= n));
+    const bool mine = i < nw && i >= n && P.a_pool[row + wait[i]] == j;
+    n_ac += __popc(__ballot_sync(TG_FULL, mine));
   }
   if (m == 0) return true;
   CandArrays C;
@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
             for (int j = 0; j < P.P && ok; ++j) {
               if (ncand[j] == 0) continue;                  // no candidate has this pool as its key pool
               int add = 0;
-              ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add, aside[j]);
+              ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add, aside[j], ncand[j]);
 #pragma unroll
               for (int jj = 0; jj < TG_MAX_POOLS; ++jj) if (jj == j) busy[jj] += add;
             }

@@ -1424,8 +1424,29 @@ __device__ int evict_resume(const Params& P, const PoolTask& T, Slab slab, int l
   return keep;
 }
 
+// A single candidate: nothing can be evicted (the head stays), and DPArrange for one task is the feasible
+// level of least duration, the smallest one among equals (value, then units).  Lane r-1 tries multiplicity r.
+__device__ __forceinline__ void solve_single(const PoolTask& T, int lane) {
+  const int g = T.cg[0] & 0x7f, gang = T.cg[0] >> 7, r = lane + 1;
+  const u32 mk = T.cmask[0];
+  bool ok = (mk >> lane) & 1u;
+  if (ok) {
+    const int lz = T.type == TG_POOL_GPU ? level_of(g, gang, r) : 0;
+    int cap = T.cap[0];
+#pragma unroll
+    for (int l = 1; l < 4; ++l) if (l == lz) cap = T.cap[l];
+    ok = g * r <= cap;
+  }
+  const i64 key = ok ? ((duration(T.cs[0], T.cp[0], r) << 6) | (i64)r) : TG_INF;
+  const i64 best = warp_min64(key);
+  // (the least level fits: the prefix admitted the action)
+  if (lane == 0) { const u8 rr = best == TG_INF ? (u8)__ffs(mk) : (u8)(best & 63); T.rsel[0] = rr; T.rkeep[0] = rr; }
+  __syncwarp();
+}
+
 // The whole loop, starting from the full candidate list.
 __device__ int evict_loop(const Params& P, const PoolTask& T, Slab slab, int lane) {
+  if (T.m == 1) { solve_single(T, lane); return 1; }
   i64 opt;
   if (!solve_prefix(P, T, T.m, slab, lane, &opt)) return -1;
   for (int i = lane; i < T.m; i += 32) T.rkeep[i] = T.rsel[i];
