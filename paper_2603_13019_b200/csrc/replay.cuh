@@ -26,14 +26,20 @@ struct ReplayWs {
   int U, Dtot;
   i64 round_us; int max_rounds;
   int* occupancy; int* rounds_used;
+  int state_bytes;  // > 0: a scenario's live state (owner .. win) fits that many bytes of shared memory per warp
 };
 
-__device__ __forceinline__ int pool_busy_units(const Params& P, const ReplayWs& R, int sc, int j, int lane) {
+// Where the live state of the scenario at hand is: the arrays of ReplayWs, or the warp's shared memory (the
+// bases are moved back by the scenario's offset, so that the same indexing reaches either).
+__host__ __device__ __forceinline__ size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
+struct ReplayState { int* owner; u8* nm; int* dfree; int* pst; i64* win; };
+
+__device__ __forceinline__ int pool_busy_units(const Params& P, const ReplayWs& R, const ReplayState& Z, int sc, int j, int lane) {
   const PoolDev& pd = P.pool[j];
   int b = 0;
-  if (pd.type == TG_POOL_API) b = pd.window_us > 0 ? R.pst[((size_t)sc * P.P + j) * 2] : R.pst[((size_t)sc * P.P + j) * 2 + 1];
+  if (pd.type == TG_POOL_API) b = pd.window_us > 0 ? Z.pst[((size_t)sc * P.P + j) * 2] : Z.pst[((size_t)sc * P.P + j) * 2 + 1];
   else {
-    const int* ow = R.owner + (size_t)sc * R.U + R.unit0[j];
+    const int* ow = Z.owner + (size_t)sc * R.U + R.unit0[j];
     for (int c = lane; c < pd.capacity; c += 32) b += ow[c] != -1;
     b = warp_sum32(b);
   }
@@ -44,19 +50,19 @@ __device__ __forceinline__ int pool_busy_units(const Params& P, const ReplayWs& 
 // dem / cap: 4 ints per pool in the warp's scratch.  Warp-uniform result.
 // aside: per pool, what the candidates ask of it beside their key resource (cost vectors);
 // ncand: per pool, how many of the candidates have it as their key pool.
-__device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const int* wait, int nw,
+__device__ int replay_prefix(const Params& P, const ReplayWs& R, const ReplayState& Z, int sc, const int* wait, int nw,
                              int* dem, int* cap, int* aside, int* ncand, int lane) {
   const size_t row = (size_t)sc * P.N;
   for (int j = 0; j < P.P; ++j) {
     const PoolDev& pd = P.pool[j];
     int c[4] = {0, 0, 0, 0};
-    if (pd.type == TG_POOL_GPU) gpu_caps(pd, R.nm + (size_t)sc * P.n_nodes_total, lane, c);
+    if (pd.type == TG_POOL_GPU) gpu_caps(pd, Z.nm + (size_t)sc * P.n_nodes_total, lane, c);
     else if (pd.type == TG_POOL_CPU) {
       int f = 0;
-      for (int d = lane; d < pd.capacity / pd.group; d += 32) f += R.dfree[(size_t)sc * R.Dtot + R.dom0[j] + d];
+      for (int d = lane; d < pd.capacity / pd.group; d += 32) f += Z.dfree[(size_t)sc * R.Dtot + R.dom0[j] + d];
       c[0] = warp_sum32(f);
     } else {
-      const int* ps = R.pst + ((size_t)sc * P.P + j) * 2;
+      const int* ps = Z.pst + ((size_t)sc * P.P + j) * 2;
       c[0] = pd.capacity - (pd.window_us > 0 ? ps[0] : ps[1]);
     }
     if (lane < 4) { cap[j * 4 + lane] = c[lane]; dem[j * 4 + lane] = 0; }
@@ -112,7 +118,7 @@ __device__ int replay_prefix(const Params& P, const ReplayWs& R, int sc, const i
 // One pool of one replay round: selection among the pool's candidates (the first n waiting
 // actions that sit on pool j), placement on the pool's live state, start of what was selected.
 // Appends the started actions to run[] (nr updated).  Returns false if the scratch ran out.
-__device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, const int* wait, int nw, int n,
+__device__ bool replay_pool(const Params& P, const ReplayWs& R, const ReplayState& Z, int sc, int j, const int* wait, int nw, int n,
                             int* run, int& nr, i64 now, Slab slab, int lane, int& busy_units, int aside_j, int m) {
   const size_t row = (size_t)sc * P.N;
   const PoolDev& pd = P.pool[j];
@@ -180,13 +186,13 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
     PoolTask T;
     T.type = pd.type; T.group = pd.group;
     T.cap[0] = T.cap[1] = T.cap[2] = T.cap[3] = 0;
-    if (pd.type == TG_POOL_GPU) gpu_caps(pd, R.nm + (size_t)sc * P.n_nodes_total, lane, T.cap);
+    if (pd.type == TG_POOL_GPU) gpu_caps(pd, Z.nm + (size_t)sc * P.n_nodes_total, lane, T.cap);
     else if (pd.type == TG_POOL_CPU) {
       int f = 0;
-      for (int d = lane; d < pd.capacity / pd.group; d += 32) f += R.dfree[(size_t)sc * R.Dtot + R.dom0[j] + d];
+      for (int d = lane; d < pd.capacity / pd.group; d += 32) f += Z.dfree[(size_t)sc * R.Dtot + R.dom0[j] + d];
       T.cap[0] = warp_sum32(f);
     } else {
-      const int* ps = R.pst + ((size_t)sc * P.P + j) * 2;
+      const int* ps = Z.pst + ((size_t)sc * P.P + j) * 2;
       T.cap[0] = pd.capacity - (pd.window_us > 0 ? ps[0] : ps[1]) - aside_j;   // set aside for the other pools' candidates
     }
     T.m = m; T.cs = C.cs; T.cp = C.cp; T.cmask = C.cmask; T.cg = C.cg;
@@ -208,19 +214,19 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
   const u8* missed = nullptr;                            // candidates whose chunk did not cache their service
   if (pd.type == TG_POOL_GPU && P.cache_slots > 0) {
     const size_t cbase = ((size_t)sc * P.n_nodes_total + pd.node0) * 8 * P.cache_slots;
-    place_gpu_cache(pd, R.nm + (size_t)sc * P.n_nodes_total + pd.node0, keep, C.cg, C.rkeep, C.cidx, C.pnode, C.poff,
+    place_gpu_cache(pd, Z.nm + (size_t)sc * P.n_nodes_total + pd.node0, keep, C.cg, C.rkeep, C.cidx, C.pnode, C.poff,
                     C.rsel, P.a_service ? P.a_service + row : nullptr, P.cache_tag + cbase, P.cache_use + cbase,
-                    P.cache_slots, now, lane, R.owner + (size_t)sc * R.U + R.unit0[j]);
+                    P.cache_slots, now, lane, Z.owner + (size_t)sc * R.U + R.unit0[j]);
     missed = C.rsel;
   } else if (pd.type == TG_POOL_GPU) {
-    place_gpu(pd, R.nm + (size_t)sc * P.n_nodes_total + pd.node0, keep, C.cg, C.rkeep, C.pnode, C.poff, lane,
-              R.owner + (size_t)sc * R.U + R.unit0[j], C.cidx);
+    place_gpu(pd, Z.nm + (size_t)sc * P.n_nodes_total + pd.node0, keep, C.cg, C.rkeep, C.pnode, C.poff, lane,
+              Z.owner + (size_t)sc * R.U + R.unit0[j], C.cidx);
   } else if (pd.type == TG_POOL_CPU) {
-    place_cpu_owner(pd, R.owner + (size_t)sc * R.U + R.unit0[j], R.dfree + (size_t)sc * R.Dtot + R.dom0[j],
+    place_cpu_owner(pd, Z.owner + (size_t)sc * R.U + R.unit0[j], Z.dfree + (size_t)sc * R.Dtot + R.dom0[j],
                     keep, C.cg, C.rkeep, C.cidx, C.pnode, C.poff, lane);
   } else {
     if (lane == 0) {
-      int* ps = R.pst + ((size_t)sc * P.P + j) * 2 + (pd.window_us > 0 ? 0 : 1);
+      int* ps = Z.pst + ((size_t)sc * P.P + j) * 2 + (pd.window_us > 0 ? 0 : 1);
       for (int i = 0; i < keep; ++i) { C.pnode[i] = 0; C.poff[i] = *ps; *ps += (C.cg[i] & 0x7f) * C.rkeep[i]; }
     }
   }
@@ -250,6 +256,7 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, int sc, int j, c
 // are spread over as many SMs (and schedulers) as possible instead of sharing one.
 #define KR_THREADS 64
 #define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 320) + 16)
+#define KR_STATE_MAX 16384
 __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * KR_THREADS + threadIdx.x) >> 5;
@@ -258,9 +265,23 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
     const size_t row = (size_t)sc * P.N;
     const int n_act = min(max(P.n_actions[sc], 0), P.N);
     int* wait = R.wait + row; int* run = R.run + row;
-    int* owner = R.owner + (size_t)sc * R.U;
-    u8* nm = R.nm + (size_t)sc * P.n_nodes_total;
-    int* dfree = R.dfree + (size_t)sc * R.Dtot;
+    ReplayState Z;
+    Z.owner = R.owner; Z.nm = R.nm; Z.dfree = R.dfree; Z.pst = R.pst; Z.win = R.win;
+    if (R.state_bytes > 0) {
+      // the state is small: it lives in this warp's shared memory for the whole trace
+      extern __shared__ __align__(16) unsigned char k2_smem[];
+      unsigned char* base = k2_smem + (KR_THREADS / 32) * (WARP_SMEM_BYTES + 320) + 16 + (size_t)(threadIdx.x >> 5) * R.state_bytes;
+      const size_t o_nm = align16((size_t)R.U * 4), o_df = o_nm + align16((size_t)P.n_nodes_total + 1),
+                   o_ps = o_df + align16((size_t)R.Dtot * 4), o_wn = o_ps + align16((size_t)P.P * 8);
+      Z.owner = (int*)((size_t)base - (size_t)sc * R.U * 4);
+      Z.nm = (u8*)((size_t)(base + o_nm) - (size_t)sc * P.n_nodes_total);
+      Z.dfree = (int*)((size_t)(base + o_df) - (size_t)sc * R.Dtot * 4);
+      Z.pst = (int*)((size_t)(base + o_ps) - (size_t)sc * P.P * 8);
+      Z.win = (i64*)((size_t)(base + o_wn) - (size_t)sc * P.P * 8);
+    }
+    int* owner = Z.owner + (size_t)sc * R.U;
+    u8* nm = Z.nm + (size_t)sc * P.n_nodes_total;
+    int* dfree = Z.dfree + (size_t)sc * R.Dtot;
     int* occ = R.occupancy ? R.occupancy + (size_t)sc * R.max_rounds * P.P : nullptr;
     // outputs and state start empty
     for (int i = lane; i < P.N; i += 32) { P.o_alloc[row + i] = 0; P.o_node[row + i] = -1; P.o_off[row + i] = -1; P.o_act[row + i] = -1; }
@@ -282,7 +303,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
     if (status & TG_ST_BAD_ACTION) status = TG_ST_BAD_ACTION;
     for (int j = 0; j < P.P; ++j) {
       const PoolDev& pd = P.pool[j];
-      if (pd.type == TG_POOL_API) { if (lane < 2) R.pst[((size_t)sc * P.P + j) * 2 + lane] = 0; if (lane == 0) R.win[(size_t)sc * P.P + j] = 0; continue; }
+      if (pd.type == TG_POOL_API) { if (lane < 2) Z.pst[((size_t)sc * P.P + j) * 2 + lane] = 0; if (lane == 0) Z.win[(size_t)sc * P.P + j] = 0; continue; }
       for (int c = lane; c < pd.capacity; c += 32) {
         int v = -1;
         if (pd.type == TG_POOL_GPU && P.gpu_busy && (P.gpu_busy[(size_t)sc * P.n_nodes_total + pd.node0 + c / pd.group] >> (c % pd.group) & 1)) v = -2;
@@ -308,15 +329,15 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
       bool drained = false;
       // units in use per core / GPU pool, kept up to date by what starts and what is released
       int busy[TG_MAX_POOLS];
-      for (int j = 0; j < P.P; ++j) busy[j] = P.pool[j].type == TG_POOL_API ? 0 : pool_busy_units(P, R, sc, j, lane);
+      for (int j = 0; j < P.P; ++j) busy[j] = P.pool[j].type == TG_POOL_API ? 0 : pool_busy_units(P, R, Z, sc, j, lane);
       while (r < R.max_rounds) {
         const i64 now = (i64)r * R.round_us;
         // 1. quota refill
         for (int j = 0; j < P.P; ++j) {
           const PoolDev& pd = P.pool[j];
-          if (pd.type == TG_POOL_API && pd.window_us > 0 && now / pd.window_us != R.win[(size_t)sc * P.P + j]) {
+          if (pd.type == TG_POOL_API && pd.window_us > 0 && now / pd.window_us != Z.win[(size_t)sc * P.P + j]) {
             __syncwarp();
-            if (lane == 0) { R.win[(size_t)sc * P.P + j] = now / pd.window_us; R.pst[((size_t)sc * P.P + j) * 2] = 0; }
+            if (lane == 0) { Z.win[(size_t)sc * P.P + j] = now / pd.window_us; Z.pst[((size_t)sc * P.P + j) * 2] = 0; }
             __syncwarp();
           }
         }
@@ -346,9 +367,9 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
             if (P.n_side > 0 && lane == 0)                 // a concurrency pool held the action's further amounts until now
               for (int e = 0; e < P.n_side; ++e) {
                 const int k = P.a_side_pool[e * P.side_plane + row + fa];
-                if (k != 0xff && P.pool[k].window_us == 0) R.pst[((size_t)sc * P.P + k) * 2 + 1] -= P.a_side_units[e * P.side_plane + row + fa];
+                if (k != 0xff && P.pool[k].window_us == 0) Z.pst[((size_t)sc * P.P + k) * 2 + 1] -= P.a_side_units[e * P.side_plane + row + fa];
               }
-            if (pd.type == TG_POOL_API) { if (pd.window_us == 0 && lane == 0) R.pst[((size_t)sc * P.P + j) * 2 + 1] -= P.o_alloc[row + fa]; }
+            if (pd.type == TG_POOL_API) { if (pd.window_us == 0 && lane == 0) Z.pst[((size_t)sc * P.P + j) * 2 + 1] -= P.o_alloc[row + fa]; }
             else {
               const int freed = P.o_alloc[row + fa];
 #pragma unroll
@@ -391,7 +412,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
         // 4. schedule
         int blocked_pool = -1;                              // pool of a head-of-line action that does not fit
         if (nw > 0) {
-          const int n = replay_prefix(P, R, sc, wait, nw, dem, cap, aside, ncand, lane);
+          const int n = replay_prefix(P, R, Z, sc, wait, nw, dem, cap, aside, ncand, lane);
           if (n == 0 && P.n_side == 0) blocked_pool = P.a_pool[row + wait[0]];
           const int nr0 = nr;
           bool ok = true;
@@ -399,7 +420,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
             for (int j = 0; j < P.P && ok; ++j) {
               if (ncand[j] == 0) continue;                  // no candidate has this pool as its key pool
               int add = 0;
-              ok = replay_pool(P, R, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add, aside[j], ncand[j]);
+              ok = replay_pool(P, R, Z, sc, j, wait, nw, n, run, nr, now, warp_slab(P, gw), lane, add, aside[j], ncand[j]);
 #pragma unroll
               for (int jj = 0; jj < TG_MAX_POOLS; ++jj) if (jj == j) busy[jj] += add;
             }
@@ -410,7 +431,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
               for (int e = 0; e < P.n_side; ++e) {
                 const int k = P.a_side_pool[e * P.side_plane + row + run[i]];
                 if (k != 0xff)
-                  atomicAdd(&R.pst[((size_t)sc * P.P + k) * 2 + (P.pool[k].window_us > 0 ? 0 : 1)],
+                  atomicAdd(&Z.pst[((size_t)sc * P.P + k) * 2 + (P.pool[k].window_us > 0 ? 0 : 1)],
                             (int)P.a_side_units[e * P.side_plane + row + run[i]]);
               }
             __syncwarp();
@@ -431,7 +452,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
           }
         }
         // 5. occupancy of this round
-        for (int j = 0; j < P.P; ++j) if (P.pool[j].type == TG_POOL_API) busy[j] = pool_busy_units(P, R, sc, j, lane);
+        for (int j = 0; j < P.P; ++j) if (P.pool[j].type == TG_POOL_API) busy[j] = pool_busy_units(P, R, Z, sc, j, lane);
         if (occ && lane == 0) for (int j = 0; j < P.P; ++j) occ[(size_t)r * P.P + j] = busy[j];
         ++r;
         if (next == n_act && nw == 0 && nr == 0) { drained = true; break; }
@@ -452,7 +473,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
             for (int j = 0; j < P.P; ++j) {
               const PoolDev& pd = P.pool[j];
               int v = busy[j];
-              if (pd.type == TG_POOL_API && pd.window_us > 0 && (rr * R.round_us) / pd.window_us != R.win[(size_t)sc * P.P + j]) v = 0;
+              if (pd.type == TG_POOL_API && pd.window_us > 0 && (rr * R.round_us) / pd.window_us != Z.win[(size_t)sc * P.P + j]) v = 0;
               if (occ) occ[(size_t)rr * P.P + j] = v;
             }
           if (r_next > r) r = (int)r_next;
@@ -463,7 +484,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
           // their occupancy rows follow from the completion times.
           const PoolDev& hp = P.pool[blocked_pool];
           i64 t_next = TG_INF;
-          if (hp.type == TG_POOL_API && hp.window_us > 0) t_next = (R.win[(size_t)sc * P.P + blocked_pool] + 1) * (i64)hp.window_us;
+          if (hp.type == TG_POOL_API && hp.window_us > 0) t_next = (Z.win[(size_t)sc * P.P + blocked_pool] + 1) * (i64)hp.window_us;
           for (int i = lane; i < nr; i += 32) {
             const int a = run[i];
             if (P.a_pool[row + a] == blocked_pool) t_next = min(t_next, (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a]);
@@ -477,7 +498,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
                 for (int j = 0; j < P.P; ++j) {
                   const PoolDev& pd = P.pool[j];
                   int v = busy[j];
-                  if (pd.type == TG_POOL_API && pd.window_us > 0 && (rr * R.round_us) / pd.window_us != R.win[(size_t)sc * P.P + j]) v = 0;
+                  if (pd.type == TG_POOL_API && pd.window_us > 0 && (rr * R.round_us) / pd.window_us != Z.win[(size_t)sc * P.P + j]) v = 0;
                   occ[(size_t)rr * P.P + j] = v;
                 }
               __syncwarp();

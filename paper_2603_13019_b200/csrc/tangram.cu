@@ -746,7 +746,7 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay, cudaFuncAttributeMaxDynamicSharedMemorySize, KR_DYN_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay, cudaFuncAttributeMaxDynamicSharedMemorySize, KR_DYN_SMEM + (KR_THREADS / 32) * KR_STATE_MAX);
   for (int c = 0; c < TG_N_SIM_CLASSES && e == cudaSuccess; ++c)
     e = cudaFuncSetAttribute(sim_kernel(g_sim_caps[c]), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TG_SMEM_PER_BLOCK - 1024);
@@ -1052,7 +1052,14 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
   int warps = P.n_workers < P.S ? P.n_workers : (int)align_up((size_t)P.S, K2_THREADS / 32);
   cudaEvent_t* ev = prof_begin(r, 2, -1, -1, -1);
   if (ev) CK(cudaEventRecord(ev[0], st));
-  k_replay<<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM, st>>>(P, R);
+  {
+    // a scenario's live state (owner of every unit, node masks, free cores per domain, quota counters) goes to
+    // shared memory when it is small
+    const size_t need = align16((size_t)R.U * 4) + align16((size_t)P.n_nodes_total + 1) + align16((size_t)R.Dtot * 4) +
+                        2 * align16((size_t)P.P * 8);
+    R.state_bytes = need <= KR_STATE_MAX ? (int)need : 0;
+  }
+  k_replay<<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM + (KR_THREADS / 32) * R.state_bytes, st>>>(P, R);
   if (ev) CK(cudaEventRecord(ev[1], st));
   r->launches += 1;
   CK(cudaGetLastError());
