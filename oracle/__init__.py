@@ -122,8 +122,9 @@ def schedule_batch(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, 
 
 def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, depth: int = 2,
                  round_us: int = 10_000, max_rounds: int, lo: int = 0, hi: Optional[int] = None,
-                 want_occupancy: bool = True, cache_slots: int = 0) -> Dict[str, np.ndarray]:
-    """Trace replay of scenarios [lo, hi)."""
+                 want_occupancy: bool = True, cache_slots: int = 0, policy: int = 0) -> Dict[str, np.ndarray]:
+    """Trace replay of scenarios [lo, hi).  policy 1 / 2: the waiting queue is kept in shortest / longest
+    least-level duration order (equal keys in arrival order) instead of first come first served."""
     S_all, N = arrays["pool"].shape
     hi = S_all if hi is None else hi
     S = hi - lo
@@ -155,7 +156,7 @@ def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, de
         _p(out["n_selected"], C.c_int), _p(out["status"], C.c_int), _p(out["occupancy"], C.c_int),
         _p(out["rounds_used"], C.c_int),
         _p(service, C.c_uint16), _p(restore, C.c_longlong), C.c_int(cache_slots), _p(tag, C.c_uint32),
-        _p(use, C.c_longlong), C.c_int(n_side), _p(side_pool, C.c_uint8), _p(side_units, C.c_uint16))
+        _p(use, C.c_longlong), C.c_int(n_side), _p(side_pool, C.c_uint8), _p(side_units, C.c_uint16), C.c_int(policy))
     assert rc == 0
     if cache_slots > 0:
         out["cache_tag"], out["cache_use"] = tag, use

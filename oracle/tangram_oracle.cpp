@@ -772,7 +772,7 @@ int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const
                         int* rounds_used,
                         const uint16_t* service, const i64* restore, int cache_slots,
                         unsigned* cache_tag, i64* cache_use,
-                        int n_side, const uint8_t* side_pool, const uint16_t* side_units) {
+                        int n_side, const uint8_t* side_pool, const uint16_t* side_units, int policy) {
   std::vector<PoolDesc> pd(n_pools);
   for (int j = 0; j < n_pools; ++j)
     pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
@@ -821,6 +821,11 @@ int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const
         E.erase(E.begin() + e);
       }
       while (next < n && acts[next].arrival <= now) W.push_back(next++);   // admit arrivals
+      if (policy == 1 || policy == 2)                               // R27: the queue in the policy's order
+        std::stable_sort(W.begin(), W.end(), [&](int x, int y) {
+          i64 kx = duration(acts[x], acts[x].r.front()), ky = duration(acts[y], acts[y].r.front());
+          return policy == 1 ? kx < ky : kx > ky;
+        });
       std::vector<Grant> grants = schedule_round(pools, acts, W, E, now, depth);
       for (const Grant& g : grants) {                               // start selected actions
         const Action& a = acts[g.action];
@@ -857,7 +862,7 @@ int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int
   return oracle_replay_trace_ext(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, round_us, max_rounds,
                                    n_actions, pool, unit, mask, s, p, arrival, gpu_busy, alloc_units, place_node,
                                    place_off, act_us, total_act_us, n_selected, status, occupancy, rounds_used,
-                                   nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr);
+                                   nullptr, nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr, 0);
 }
 
 // R27: permutation that sorts every scenario's queue by the policy's key (1: shortest least-level

@@ -73,6 +73,32 @@ def test_order_is_a_stable_sort_and_the_round_is_the_plain_round_on_the_sorted_q
         assert plain["n_selected"][0] == o["n_selected"][sc] and plain["total_act_us"][0] == o["total_act_us"][sc]
 
 
+def test_replay_keeps_the_queue_in_the_policys_order(oracle):
+    # one core, rounds of 10 ms.  a (30 ms) arrives at 0, b (50 ms) at 5 ms, c (10 ms) at 6 ms, d (10 ms) at 7 ms.
+    # a runs until 30 ms.  First come first served: b at 30 (ends 80), c at 80, d at 90.
+    # Shortest first: at 30 the queue is c, d, b (c before d: equal keys keep their arrival order): c 30-40,
+    # d 40-50, b 50-100.  Longest first: b, c, d as they came.
+    pools = [Pool(POOL_CPU, 1, 1)]
+    a = _arrays([(0, 1, 1, 30_000, 0), (0, 1, 1, 50_000, 0), (0, 1, 1, 10_000, 0), (0, 1, 1, 10_000, 0)],
+                arrival=[0, 5_000, 6_000, 7_000])
+    fcfs = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=40)
+    assert list(fcfs["act_us"][0]) == [30_000, 25_000 + 50_000, 74_000 + 10_000, 83_000 + 10_000]
+    sjf = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=40, policy=SJF)
+    assert list(sjf["act_us"][0]) == [30_000, 45_000 + 50_000, 24_000 + 10_000, 33_000 + 10_000]
+    assert sjf["rounds_used"][0] == 11 and sjf["total_act_us"][0] < fcfs["total_act_us"][0]
+    ljf = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=40, policy=LJF)
+    assert list(ljf["act_us"][0]) == list(fcfs["act_us"][0])
+    # a shorter action that arrives while the head does not fit becomes the head: 2 cores, x takes both for 30 ms,
+    # y (2 cores, 20 ms) waits; z (1 core, 5 ms) arrives at 12 ms: shortest first puts it ahead of y, but it does
+    # not fit either; at 30 ms z runs (ends 35), y has to wait for it (needs both cores): starts at 40
+    pools = [Pool(POOL_CPU, 2, 2)]
+    a = _arrays([(0, 2, 1, 30_000, 0), (0, 2, 1, 20_000, 0), (0, 1, 1, 5_000, 0)], arrival=[0, 1_000, 12_000])
+    sjf = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=40, policy=SJF)
+    assert list(sjf["act_us"][0]) == [30_000, 39_000 + 20_000, 18_000 + 5_000]
+    fcfs = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=40)
+    assert list(fcfs["act_us"][0]) == [30_000, 29_000 + 20_000, 38_000 + 5_000]
+
+
 # ------------------------------------------------------------------ trajectories pinned to CPU nodes
 def _traj(rows, traj, mem, node, free):
     a = _arrays(rows)
