@@ -232,6 +232,12 @@ int64_t tangram_kernel_launches(const tangram_round* round);
 #define TANGRAM_ORDER_ARRIVAL 3
 int tangram_order_queue(tangram_round* round, const tangram_actions* actions, int policy, int32_t* perm,
                         void* cuda_stream);
+/* tangram_replay_trace with the waiting queue kept in the policy's order: an arrival goes behind the last
+ * waiting action whose key is not larger than its own, every round runs Algorithm 1 on the queue as it stands.
+ * policy 0 and 3 are tangram_replay_trace itself (a trace is sorted by arrival).  The first call with
+ * policy 1 or 2 allocates 8 B per action that the round keeps (TANGRAM_ENOMEM). */
+int tangram_replay_trace_ordered(tangram_round* round, const tangram_actions* actions, int policy,
+                                 tangram_result* result, void* cuda_stream);
 int tangram_schedule_batch_ordered(tangram_round* round, const tangram_actions* actions, int policy,
                                    int64_t now_us, tangram_result* result, void* cuda_stream);
 

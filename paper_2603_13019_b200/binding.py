@@ -58,7 +58,7 @@ EXPORTS = ("tangram_round_create", "tangram_schedule_batch", "tangram_replay_tra
            "tangram_round_destroy", "tangram_kernel_launches", "tangram_strerror",
            "tangram_last_cuda_error", "tangram_set_profiling", "tangram_kernel_time_ms",
            "tangram_kernel_name", "tangram_schedule_batch_static", "tangram_order_queue",
-           "tangram_schedule_batch_ordered", "tangram_pin_trajectories")
+           "tangram_schedule_batch_ordered", "tangram_pin_trajectories", "tangram_replay_trace_ordered")
 
 
 def load_library(path: Optional[str] = None):
@@ -96,6 +96,8 @@ def load_library(path: Optional[str] = None):
     lib.tangram_schedule_batch_ordered.restype = C.c_int
     lib.tangram_schedule_batch_ordered.argtypes = [C.c_void_p, C.POINTER(_Actions), C.c_int, C.c_int64,
                                                    C.POINTER(_Result), C.c_void_p]
+    lib.tangram_replay_trace_ordered.restype = C.c_int
+    lib.tangram_replay_trace_ordered.argtypes = [C.c_void_p, C.POINTER(_Actions), C.c_int, C.POINTER(_Result), C.c_void_p]
     lib.tangram_pin_trajectories.restype = C.c_int
     lib.tangram_pin_trajectories.argtypes = [C.c_void_p, C.POINTER(_Actions), C.POINTER(_Pinning), C.c_void_p]
     lib.tangram_schedule_batch_static.argtypes = [C.POINTER(_RoundDesc), C.POINTER(_Actions), C.c_int64,
@@ -221,11 +223,15 @@ class Round:
         _check(self._lib.tangram_schedule_batch(self._h, C.byref(a), int(now_us), C.byref(r), self._stream(stream)))
         return result
 
-    def replay_trace(self, actions: Dict, result: Optional[Dict] = None, stream=None) -> Dict:
-        """tangram_replay_trace: device-resident replay of every scenario's arrival trace."""
+    def replay_trace(self, actions: Dict, result: Optional[Dict] = None, stream=None, policy: int = 0) -> Dict:
+        """tangram_replay_trace (policy 0) / tangram_replay_trace_ordered: device-resident replay of every
+        scenario's arrival trace."""
         result = self.new_result(replay=True) if result is None else result
         a, r = self._actions(actions), self._result(result)
-        _check(self._lib.tangram_replay_trace(self._h, C.byref(a), C.byref(r), self._stream(stream)))
+        if policy:
+            _check(self._lib.tangram_replay_trace_ordered(self._h, C.byref(a), int(policy), C.byref(r), self._stream(stream)))
+        else:
+            _check(self._lib.tangram_replay_trace(self._h, C.byref(a), C.byref(r), self._stream(stream)))
         return result
 
     def order_queue(self, actions: Dict, policy: int, stream=None):

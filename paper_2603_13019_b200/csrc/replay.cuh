@@ -26,6 +26,8 @@ struct ReplayWs {
   int U, Dtot;
   i64 round_us; int max_rounds;
   int* occupancy; int* rounds_used;
+  int policy;       // 0: first come first served; 1 / 2: the queue is kept in shortest / longest least-level duration order
+  u64* wkey;        // [S][N] sort keys of the waiting actions (policy 1 / 2 only)
   int state_bytes;  // > 0: a scenario's live state (owner .. win) fits that many bytes of shared memory per warp
 };
 
@@ -257,6 +259,8 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, const ReplayStat
 #define KR_THREADS 64
 #define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 320) + 16)
 #define KR_STATE_MAX 16384
+// ORDERED: the waiting queue is kept sorted by R.policy's key (the plain instance keeps its registers).
+template <bool ORDERED>
 __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
   const int lane = threadIdx.x & 31;
   const int gw = (blockIdx.x * KR_THREADS + threadIdx.x) >> 5;
@@ -399,6 +403,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
           __syncwarp();
         }
         // 3. admit arrivals
+        const int nw_admitted = nw;
         while (next < n_act) {
           const int i = next + lane;
           const bool in = i < n_act && (P.a_arrival ? P.a_arrival[row + i] : 0) <= now;
@@ -409,6 +414,34 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
           if (cnt < 32) break;
         }
         __syncwarp();
+        if (ORDERED && nw > nw_admitted) {
+          // Other queue orders (Section 4.2): the queue stays sorted by the policy's key, equal keys in arrival
+          // order.  Each new arrival goes behind the last entry whose key is not larger; the tail moves up by one.
+          u64* wkey = R.wkey + row;
+          for (int x = nw_admitted; x < nw; ++x) {
+            const int a = wait[x];
+            int g, gang; u32 eff;
+            decode_levels(P.pool[P.a_pool[row + a]], P.a_unit[row + a], P.a_mask[row + a], g, gang, eff);
+            const i64 T = duration(clamp_param(P.a_s[row + a]), clamp_param(P.a_p[row + a]), __ffs(eff));
+            const u64 k = R.policy == 2 ? (u64)((1ll << 42) - T) : (u64)T;
+            int p = 0;
+            for (int i0 = 0; i0 < x; i0 += 32) {
+              const int i = i0 + lane;
+              p += __popc(__ballot_sync(TG_FULL, i < x && wkey[i] <= k));
+            }
+            for (int hi = x; hi > p;) {
+              const int lo = max(p, hi - 32), i = lo + lane;
+              int va = 0; u64 vk = 0;
+              if (i < hi) { va = wait[i]; vk = wkey[i]; }
+              __syncwarp();
+              if (i < hi) { wait[i + 1] = va; wkey[i + 1] = vk; }
+              __syncwarp();
+              hi = lo;
+            }
+            if (lane == 0) { wait[p] = a; wkey[p] = k; }
+            __syncwarp();
+          }
+        }
         // 4. schedule
         int blocked_pool = -1;                              // pool of a head-of-line action that does not fit
         if (nw > 0) {
@@ -441,10 +474,11 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
             for (int i0 = 0; i0 < nw; i0 += 32) {
               const int i = i0 + lane;
               int a = -1; bool stay = false;
-              if (i < nw) { a = wait[i]; stay = P.o_act[row + a] < 0; }
+              u64 kk = 0;
+              if (i < nw) { a = wait[i]; stay = P.o_act[row + a] < 0; if (ORDERED) kk = R.wkey[row + i]; }
               const u32 b = __ballot_sync(TG_FULL, stay);
               __syncwarp();
-              if (stay) wait[kw + __popc(b & ((1u << lane) - 1u))] = a;
+              if (stay) { wait[kw + __popc(b & ((1u << lane) - 1u))] = a; if (ORDERED) R.wkey[row + kw + __popc(b & ((1u << lane) - 1u))] = kk; }
               kw += __popc(b);
             }
             nw = kw;
@@ -485,6 +519,8 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
           const PoolDev& hp = P.pool[blocked_pool];
           i64 t_next = TG_INF;
           if (hp.type == TG_POOL_API && hp.window_us > 0) t_next = (Z.win[(size_t)sc * P.P + blocked_pool] + 1) * (i64)hp.window_us;
+          // (in a sorted queue an arrival with a smaller key becomes the head)
+          if (ORDERED && next < n_act) t_next = min(t_next, P.a_arrival ? P.a_arrival[row + next] : 0);
           for (int i = lane; i < nr; i += 32) {
             const int a = run[i];
             if (P.a_pool[row + a] == blocked_pool) t_next = min(t_next, (P.a_arrival ? P.a_arrival[row + a] : 0) + P.o_act[row + a]);

@@ -466,7 +466,7 @@ struct tangram_round {
   // the certified pools (k_easy and their placement) run beside the kernels that follow k_solve
   cudaStream_t side; cudaEvent_t side_fork, side_join;
   // sorted copy of the queue and of its results (tangram_schedule_batch_ordered), allocated at its first call
-  char* d_sorted; int* d_perm;
+  char* d_sorted; int* d_perm; u64* d_wkey;
   // staging for host-buffer mode
   char* d_stage; size_t stage_bytes;
   size_t in_off[8], out_off[9];
@@ -746,7 +746,8 @@ extern "C" int tangram_round_create(const tangram_round_desc* desc, tangram_roun
   P.slabs = (char*)r->d_slabs; P.arena = (char*)r->d_arena; P.arena_top = (u64*)r->d_arena_top;
   e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_solve, cudaFuncAttributeMaxDynamicSharedMemorySize, K2_DYN_SMEM);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay, cudaFuncAttributeMaxDynamicSharedMemorySize, KR_DYN_SMEM + (KR_THREADS / 32) * KR_STATE_MAX);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, KR_DYN_SMEM + (KR_THREADS / 32) * KR_STATE_MAX);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_replay<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, KR_DYN_SMEM + (KR_THREADS / 32) * KR_STATE_MAX);
   for (int c = 0; c < TG_N_SIM_CLASSES && e == cudaSuccess; ++c)
     e = cudaFuncSetAttribute(sim_kernel(g_sim_caps[c]), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TG_SMEM_PER_BLOCK - 1024);
@@ -810,7 +811,7 @@ extern "C" void tangram_round_destroy(tangram_round* r) {
   if (!r) return;
   if (r->ev) tangram_set_profiling(r, 0);
   cudaFree(r->d_order); cudaFree(r->d_tmin); cudaFree(r->d_meta); cudaFree(r->d_slabs);
-  cudaFree(r->d_ok_table); cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl); cudaFree(r->d_side_bad); cudaFree(r->d_side_res); cudaFree(r->d_sorted); cudaFree(r->d_perm);
+  cudaFree(r->d_ok_table); cudaFree(r->d_arena); cudaFree(r->d_arena_top); cudaFree(r->d_stage); cudaFree(r->hst); cudaFree(r->d_preq); cudaFree(r->d_keepn); cudaFree(r->d_fl); cudaFree(r->d_side_bad); cudaFree(r->d_side_res); cudaFree(r->d_sorted); cudaFree(r->d_perm); cudaFree(r->d_wkey);
   cudaFree(r->W.ts); cudaFree(r->W.seed2); cudaFree(r->W.rs1); cudaFree(r->W.rs2);
   cudaFree(r->L.count); cudaFree(r->L.list);
   cudaFree(r->R.wait); cudaFree(r->R.run); cudaFree(r->R.owner); cudaFree(r->R.nm); cudaFree(r->R.dfree);
@@ -1029,15 +1030,34 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   return TANGRAM_OK;
 }
 
+static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_result* res, void* cuda_stream, int policy);
+
 extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, tangram_result* res,
                                     void* cuda_stream) {
+  return replay_impl(r, a, res, cuda_stream, 0);
+}
+
+extern "C" int tangram_replay_trace_ordered(tangram_round* r, const tangram_actions* a, int policy, tangram_result* res,
+                                            void* cuda_stream) {
+  if (policy < 0 || policy > 3) return TANGRAM_EINVAL;
+  return replay_impl(r, a, res, cuda_stream, policy == 3 ? 0 : policy);   // a trace is sorted by arrival already
+}
+
+static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_result* res, void* cuda_stream, int policy) {
   if (!r || !check_io(a, res) || r->desc.max_rounds <= 0 || !a->arrival_us) return TANGRAM_EINVAL;
+  if (policy && !r->d_wkey) {                              // sort keys of the waiting actions, kept by the round
+    if (cudaMalloc((void**)&r->d_wkey, (size_t)r->P.S * r->P.N * sizeof(u64)) != cudaSuccess) {
+      cudaGetLastError(); r->d_wkey = nullptr;
+      return TANGRAM_ENOMEM;
+    }
+  }
   if (r->desc.cache_slots > 0 && r->P.n_nodes_total > 0 && (!a->gpu_cache_tag || !a->gpu_cache_use)) return TANGRAM_EINVAL;
   if (r->desc.side_costs > 0 && (!a->side_pool) != (!a->side_units)) return TANGRAM_EINVAL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   Params P = r->P;
   P.now = 0;
   ReplayWs R = r->R;
+  R.policy = policy; R.wkey = policy ? r->d_wkey : nullptr;
   if (r->desc.host_buffers) {
     bind_stage(r, a, P);
     int rc = copy_in(r, a, P, 0, P.S, st);
@@ -1059,7 +1079,8 @@ extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, 
                         2 * align16((size_t)P.P * 8);
     R.state_bytes = need <= KR_STATE_MAX ? (int)need : 0;
   }
-  k_replay<<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM + (KR_THREADS / 32) * R.state_bytes, st>>>(P, R);
+  if (policy) k_replay<true><<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM + (KR_THREADS / 32) * R.state_bytes, st>>>(P, R);
+  else k_replay<false><<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM + (KR_THREADS / 32) * R.state_bytes, st>>>(P, R);
   if (ev) CK(cudaEventRecord(ev[1], st));
   r->launches += 1;
   CK(cudaGetLastError());
@@ -1138,7 +1159,7 @@ extern "C" int tangram_schedule_batch_ordered(tangram_round* r, const tangram_ac
   if (!r->d_sorted) {
     if (cudaMalloc((void**)&r->d_sorted, total) != cudaSuccess || cudaMalloc((void**)&r->d_perm, SN * sizeof(int)) != cudaSuccess) {
       cudaGetLastError();
-      cudaFree(r->d_sorted); cudaFree(r->d_perm); r->d_sorted = nullptr; r->d_perm = nullptr;
+      cudaFree(r->d_sorted); cudaFree(r->d_perm); cudaFree(r->d_wkey); r->d_sorted = nullptr; r->d_perm = nullptr;
       return TANGRAM_ENOMEM;
     }
   }

@@ -208,3 +208,34 @@ def test_pinned_trajectories_match_oracle(oracle, seed):
     for k in KEYS:
         assert np.array_equal(ob[k], g[k].cpu().numpy()), k
     rnd.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed,policy", [(0, SJF), (1, LJF), (2, SJF), (3, SJF), (4, LJF)])
+def test_ordered_traces_match_oracle(oracle, seed, policy):
+    import torch
+    from paper_2603_13019_b200 import binding
+    pools = [(Pool(POOL_CPU, 16, 4), Pool(POOL_GPU, 16, 8), Pool(POOL_API, 5, 0, 200_000)),
+             (Pool(POOL_GPU, 40, 8),), (Pool(POOL_CPU, 40, 8), Pool(POOL_GPU, 8, 4), Pool(POOL_API, 3, 0, 0)),
+             (Pool(POOL_CPU, 6, 3),), (Pool(POOL_CPU, 16, 4), Pool(POOL_GPU, 32, 8))][seed]
+    N = [150, 200, 120, 400, 300][seed]
+    w, a = random_round(970 + seed, 14, N, pools, max_mult=4, small_durations=0.3 if seed != 3 else 0.8,
+                        replicas=0.5 if seed in (1, 4) else 0.0)
+    rng = np.random.default_rng(seed)
+    # bursts: many arrivals per round while actions last up to 0.5 s, so the queue is long and its order matters
+    a["arrival_us"] = np.cumsum(rng.integers(0, [3000, 4000, 2500, 300, 3000][seed], a["pool"].shape), axis=1).astype(np.int64)
+    o = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=5000, policy=policy)
+    rnd = binding.Round(14, N, pools, round_us=10_000, max_rounds=5000)
+    dev = binding.to_device(a)
+    g = rnd.replay_trace(dev, policy=policy)
+    g2 = rnd.replay_trace(dev, policy=policy)
+    plain = rnd.replay_trace(dev)                                   # first come first served is untouched by the kept keys
+    torch.cuda.synchronize()
+    for res in (g, g2):
+        for k in KEYS + ("rounds_used", "occupancy"):
+            assert np.array_equal(o[k], res[k].cpu().numpy()), k
+    of = oracle.replay_trace(pools, a, round_us=10_000, max_rounds=5000)
+    for k in KEYS + ("rounds_used", "occupancy"):
+        assert np.array_equal(of[k], plain[k].cpu().numpy()), k
+    assert not np.array_equal(of["act_us"], o["act_us"])
+    rnd.destroy()
