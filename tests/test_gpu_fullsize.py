@@ -18,25 +18,32 @@ def _run_full(name):
     S, N = w.n_scenarios, w.max_actions
     chunk = max(1, (64 << 20) // N)
     parts = [generate(w, c, min(S, c + chunk)) for c in range(0, S, chunk)]
-    a = {k: (None if parts[0][k] is None else np.concatenate([p[k] for p in parts])) for k in parts[0]}
-    rnd = binding.Round(S, N, w.pools, depth=w.depth)
-    out = rnd.schedule_batch(binding.to_device(a))
+    a = {k: (None if parts[0][k] is None else np.concatenate([p[k] for p in parts], axis=1 if k.startswith("side_") else 0))
+         for k in parts[0]}
+    rnd = binding.Round(S, N, w.pools, depth=w.depth, cache_slots=int(w.params.get("cache_slots", 0)),
+                        side_costs=int(w.params.get("side_costs", 0)))
+    dev = binding.to_device(a)
+    out = rnd.schedule_batch(dev)
     torch.cuda.synchronize()
     g = {k: v.cpu().numpy() for k, v in out.items()}
+    if "cache_tag" in a:                                         # the cache state is updated in place
+        g["cache_tag"] = dev["cache_tag"].cpu().numpy().view(np.uint32)
+        g["cache_use"] = dev["cache_use"].cpu().numpy()
     rnd.destroy()
     return w, a, g
 
 
-@pytest.mark.parametrize("name,n_sample", [("cfg4", 96), ("cfg1", 128), ("cfg3", 24)])
+@pytest.mark.parametrize("name,n_sample", [("cfg4", 96), ("cfg1", 128), ("cfg3", 24), ("cfg4_vec", 64), ("cfg1_cache", 96)])
 def test_full_size_sampled_scenarios_match_oracle(oracle, name, n_sample):
     w, a, g = _run_full(name)
     S = w.n_scenarios
+    K = int(w.params.get("cache_slots", 0))
     assert np.all(g["status"] == 0)
     rng = np.random.default_rng(11)
     sample = np.unique(np.concatenate([[0, S - 1], rng.integers(0, S, n_sample)]))
     for sc in sample:
-        o = oracle.schedule_batch(w.pools, a, depth=w.depth, lo=int(sc), hi=int(sc) + 1)
-        for k in KEYS:
+        o = oracle.schedule_batch(w.pools, a, depth=w.depth, lo=int(sc), hi=int(sc) + 1, cache_slots=K)
+        for k in KEYS + (("cache_tag", "cache_use") if K else ()):
             assert np.array_equal(o[k][0], g[k][sc]), f"{name}: scenario {sc}: {k} differs"
     # invariants on every scenario: capacity per pool, totals, sentinels
     sel = g["alloc_units"] > 0
@@ -45,6 +52,9 @@ def test_full_size_sampled_scenarios_match_oracle(oracle, name, n_sample):
     assert np.all(g["act_us"][~sel] == -1) and np.all(g["place_node"][~sel] == -1)
     for j, p in enumerate(w.pools):
         used = np.where(a["pool"] == j, g["alloc_units"], 0).sum(1)
+        if "side_pool" in a:                                     # the further amounts of what was scheduled
+            for e in range(a["side_pool"].shape[0]):
+                used = used + np.where(sel & (a["side_pool"][e] == j), a["side_units"][e], 0).sum(1)
         busy = 0
         if p.type == POOL_GPU and a["gpu_busy"] is not None:
             busy = np.unpackbits(a["gpu_busy"], axis=1).sum(1)
