@@ -163,6 +163,40 @@ def replay_trace(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, de
     return out
 
 
+def replay_trace_pinned(pools: Sequence, arrays: Dict[str, Optional[np.ndarray]], *, depth: int = 2,
+                        round_us: int = 10_000, max_rounds: int, policy: int = 0) -> Dict[str, np.ndarray]:
+    """Trace replay with the trajectories pinned to CPU nodes as their actions arrive (arrays "trajectory",
+    "traj_mem", "traj_last", state "traj_node", "node_mem_free").  Returns the replay's outputs plus "pool"
+    (the pool every action ran on) and the final state "traj_node" / "node_mem_free" (copies)."""
+    S, N = arrays["pool"].shape
+    pool, unit, mask, s, p, arr, n_act = _record_args(arrays, slice(0, S))
+    busy = _c(arrays["gpu_busy"], np.uint8) if arrays.get("gpu_busy") is not None else None
+    out = dict(
+        alloc_units=np.empty((S, N), np.int32), place_node=np.empty((S, N), np.int32),
+        place_off=np.empty((S, N), np.int32), act_us=np.empty((S, N), np.int64),
+        total_act_us=np.empty(S, np.int64), n_selected=np.empty(S, np.int32),
+        status=np.empty(S, np.int32), rounds_used=np.empty(S, np.int32),
+        occupancy=np.empty((S, max_rounds, len(pools)), np.int32), pool=np.empty((S, N), np.uint8),
+        traj_node=np.array(arrays["traj_node"], dtype=np.int32, order="C", copy=True),
+        node_mem_free=np.array(arrays["node_mem_free"], dtype=np.int64, order="C", copy=True))
+    traj, mem, last = _c(arrays["trajectory"], np.int32), _c(arrays["traj_mem"], np.uint32), _c(arrays["traj_last"], np.uint8)
+    pf = _pools_flat(pools)
+    rc = lib().oracle_replay_trace_pin(
+        C.c_int(S), C.c_int(N), C.c_int(len(pools)), _p(pf, C.c_int), C.c_int(depth),
+        C.c_int(_n_nodes(pools)), C.c_longlong(round_us), C.c_int(max_rounds),
+        _p(n_act, C.c_int), _p(pool, C.c_uint8), _p(unit, C.c_uint8), _p(mask, C.c_uint32),
+        _p(s, C.c_longlong), _p(p, C.c_longlong), _p(arr, C.c_longlong), _p(busy, C.c_uint8),
+        _p(out["alloc_units"], C.c_int), _p(out["place_node"], C.c_int), _p(out["place_off"], C.c_int),
+        _p(out["act_us"], C.c_longlong), _p(out["total_act_us"], C.c_longlong),
+        _p(out["n_selected"], C.c_int), _p(out["status"], C.c_int), _p(out["occupancy"], C.c_int),
+        _p(out["rounds_used"], C.c_int),
+        None, None, C.c_int(0), None, None, C.c_int(0), None, None, C.c_int(policy),
+        _p(traj, C.c_int), _p(mem, C.c_uint32), _p(last, C.c_uint8), C.c_int(out["traj_node"].shape[1]),
+        _p(out["traj_node"], C.c_int), _p(out["node_mem_free"], C.c_longlong), _p(out["pool"], C.c_uint8))
+    assert rc == 0
+    return out
+
+
 def _record_args(arrays, sl):
     return (_c(arrays["pool"][sl], np.uint8), _c(arrays["unit"][sl], np.uint8), _c(arrays["level_mask"][sl], np.uint32),
             _c(arrays["s_us"][sl], np.int64), _c(arrays["p_us"][sl], np.int64),

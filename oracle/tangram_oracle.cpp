@@ -88,6 +88,10 @@
 //       free, the one with the most free memory (lowest index on ties) takes the trajectory and
 //       sets its memory aside; all its actions run there.  An action whose trajectory finds no
 //       node ends the admitted queue (first come first served: what stands behind it waits).
+//   R29 In a replay the trajectories are pinned as their actions arrive: an arrival whose trajectory
+//       finds no node waits outside the queue, and so does everything that arrives after it; it
+//       is tried again every round.  When the action marked as its trajectory's last one ends,
+//       the trajectory's memory goes back to its node and the trajectory is no longer pinned.
 //
 // The paper prints no worked example of a schedule.  estimate() and the eviction loop are
 // heuristics; they are pinned by closed forms, by an independent list-scheduling statement
@@ -685,6 +689,29 @@ void store_cache(const std::vector<PoolRuntime>& pools, const CacheIo* cache) {
   }
 }
 
+// Trajectories pinned on arrival during a replay (R28, R29): null trajectory = none of it.
+struct PinIo { const int* trajectory; const uint32_t* traj_mem; const uint8_t* traj_last; int max_traj;
+               int* traj_node; i64* mem_free; uint8_t* pool_out; };
+
+// R28 for one arriving action: true if it may join the queue (its trajectory has, or just got, a node).
+bool pin_on_arrival(const PinIo& io, const std::vector<PoolDesc>& pd, Action& a, int* tn, i64* mf, size_t at) {
+  int t = io.trajectory[at];
+  if (t < 0 || t >= io.max_traj || pd[a.pool].type != POOL_CPU) return true;
+  if (tn[t] < 0) {
+    i64 need = (i64)a.g * a.r.front();
+    int best = -1;
+    for (int j = 0; j < (int)pd.size(); ++j) {
+      if (pd[j].type != POOL_CPU || pd[j].capacity < need || mf[j] < (i64)io.traj_mem[at]) continue;
+      if (best < 0 || mf[j] > mf[best]) best = j;
+    }
+    if (best < 0) return false;
+    tn[t] = best;
+    mf[best] -= io.traj_mem[at];
+  }
+  a.pool = tn[t];
+  return true;
+}
+
 }  // namespace
 
 // =============================================================== C entry points
@@ -763,7 +790,7 @@ int oracle_schedule_batch(int n_scenarios, int max_actions, int n_pools, const i
 // what has finished, admits what has arrived, runs the scheduler, starts what it selects.
 // occupancy: [scenario][round][pool] units in use after the round's scheduling (zero after
 // the scenario has drained); rounds_used: rounds until drained (max_rounds if never).
-int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+int oracle_replay_trace_pin(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
                         int depth, int n_nodes, i64 round_us, int max_rounds, const int* n_actions,
                         const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
                         const i64* s, const i64* p, const i64* arrival, const uint8_t* gpu_busy,
@@ -772,7 +799,10 @@ int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const
                         int* rounds_used,
                         const uint16_t* service, const i64* restore, int cache_slots,
                         unsigned* cache_tag, i64* cache_use,
-                        int n_side, const uint8_t* side_pool, const uint16_t* side_units, int policy) {
+                        int n_side, const uint8_t* side_pool, const uint16_t* side_units, int policy,
+                        const int* trajectory, const uint32_t* traj_mem, const uint8_t* traj_last, int max_traj,
+                        int* traj_node, i64* node_mem_free, uint8_t* pool_out) {
+  const PinIo pin{trajectory, traj_mem, traj_last, max_traj, traj_node, node_mem_free, pool_out};
   std::vector<PoolDesc> pd(n_pools);
   for (int j = 0; j < n_pools; ++j)
     pd[j] = PoolDesc{pools_flat[4 * j], pools_flat[4 * j + 1], pools_flat[4 * j + 2], pools_flat[4 * j + 3]};
@@ -783,6 +813,7 @@ int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const
       alloc_units[base + i] = 0; place_node[base + i] = -1; place_off[base + i] = -1; act_us[base + i] = -1;
     }
     total_act_us[sc] = 0; n_selected[sc] = 0; status[sc] = STATUS_OK; rounds_used[sc] = 0;
+    if (pin.trajectory && pin.pool_out) for (int i = 0; i < max_actions; ++i) pin.pool_out[base + i] = pool[base + i];
     if (occupancy)
       std::memset(occupancy + (size_t)sc * max_rounds * n_pools, 0, sizeof(int) * (size_t)max_rounds * n_pools);
     std::vector<Action> acts;
@@ -818,9 +849,23 @@ int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const
         } else if (pr.d.window_us == 0) pr.in_use -= E[e].units;
         for (const std::pair<int, int>& c : acts[E[e].action].side)  // R26: held until the action ends
           if (pools[c.first].d.window_us == 0) pools[c.first].in_use -= c.second;
+        if (pin.trajectory && pin.traj_last && pin.traj_last[base + E[e].action]) {   // R29: the trajectory is over
+          const int t = pin.trajectory[base + E[e].action];
+          int* tn = pin.traj_node + (size_t)sc * pin.max_traj;
+          if (t >= 0 && t < pin.max_traj && tn[t] >= 0 && pd[acts[E[e].action].pool].type == POOL_CPU) {
+            pin.mem_free[(size_t)sc * n_pools + tn[t]] += pin.traj_mem[base + E[e].action];
+            tn[t] = -1;
+          }
+        }
         E.erase(E.begin() + e);
       }
-      while (next < n && acts[next].arrival <= now) W.push_back(next++);   // admit arrivals
+      while (next < n && acts[next].arrival <= now) {               // admit arrivals
+        if (pin.trajectory &&
+            !pin_on_arrival(pin, pd, acts[next], pin.traj_node + (size_t)sc * pin.max_traj,
+                            pin.mem_free + (size_t)sc * n_pools, base + next)) break;   // R29: waits outside the queue
+        if (pin.trajectory && pin.pool_out) pin.pool_out[base + next] = (uint8_t)acts[next].pool;
+        W.push_back(next++);
+      }
       if (policy == 1 || policy == 2)                               // R27: the queue in the policy's order
         std::stable_sort(W.begin(), W.end(), [&](int x, int y) {
           i64 kx = duration(acts[x], acts[x].r.front()), ky = duration(acts[y], acts[y].r.front());
@@ -850,6 +895,23 @@ int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const
     store_cache(pools, cache);
   }
   return 0;
+}
+
+int oracle_replay_trace_ext(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,
+                        int depth, int n_nodes, i64 round_us, int max_rounds, const int* n_actions,
+                        const uint8_t* pool, const uint8_t* unit, const uint32_t* mask,
+                        const i64* s, const i64* p, const i64* arrival, const uint8_t* gpu_busy,
+                        int* alloc_units, int* place_node, int* place_off, i64* act_us,
+                        i64* total_act_us, int* n_selected, int* status, int* occupancy,
+                        int* rounds_used,
+                        const uint16_t* service, const i64* restore, int cache_slots,
+                        unsigned* cache_tag, i64* cache_use,
+                        int n_side, const uint8_t* side_pool, const uint16_t* side_units, int policy) {
+  return oracle_replay_trace_pin(n_scenarios, max_actions, n_pools, pools_flat, depth, n_nodes, round_us, max_rounds,
+                                 n_actions, pool, unit, mask, s, p, arrival, gpu_busy, alloc_units, place_node,
+                                 place_off, act_us, total_act_us, n_selected, status, occupancy, rounds_used,
+                                 service, restore, cache_slots, cache_tag, cache_use, n_side, side_pool, side_units,
+                                 policy, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr);
 }
 
 int oracle_replay_trace(int n_scenarios, int max_actions, int n_pools, const int* pools_flat,

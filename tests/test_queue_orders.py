@@ -145,6 +145,31 @@ def test_a_trajectory_that_finds_no_node_ends_the_admitted_queue(oracle):
     assert list(o["pool"][0]) == [3, 0, 0, 0] and list(o["node_mem_free"][0]) == [50, 60, 999, 60]
 
 
+def test_replay_pins_trajectories_as_their_actions_arrive(oracle):
+    # two nodes of 4 cores with 10 and 6 units of memory free, rounds of 10 ms, one-core actions.
+    # a0 (trajectory 0, 8 units, 25 ms) arrives at 0: node 0 (most free), 2 left.  a1 (trajectory 1, 5 units, 12 ms,
+    # its last action) at 1 ms: only node 1 has 5: 1 left.  a2 (trajectory 2, 4 units, 10 ms) at 2 ms finds no node
+    # and waits outside the queue; a3 (trajectory 0 again, 5 ms, its last action) at 3 ms waits behind it although
+    # its trajectory has a node.  a1 runs 10 .. 22; the round at 30 gives its 5 units back to node 1, a2 goes there
+    # (6 >= 4), a3 to node 0; a3 ends at 35 and the round at 40 gives trajectory 0's 8 units back to node 0.
+    pools = [Pool(POOL_CPU, 4, 4), Pool(POOL_CPU, 4, 4)]
+    one = lambda t: (0, 1, 1, t, 0)
+    a = _arrays([one(25_000), one(12_000), one(10_000), one(5_000)], arrival=[0, 1_000, 2_000, 3_000])
+    a["trajectory"], a["traj_mem"] = np.array([[0, 1, 2, 0]], np.int32), np.array([[8, 5, 4, 8]], np.uint32)
+    a["traj_last"] = np.array([[0, 1, 0, 1]], np.uint8)
+    a["traj_node"], a["node_mem_free"] = np.full((1, 3), -1, np.int32), np.array([[10, 6]], np.int64)
+    o = oracle.replay_trace_pinned(pools, a, round_us=10_000, max_rounds=30)
+    assert list(o["pool"][0]) == [0, 1, 1, 0]
+    assert list(o["act_us"][0]) == [25_000, 9_000 + 12_000, 28_000 + 10_000, 27_000 + 5_000]
+    assert list(o["traj_node"][0]) == [-1, -1, 1] and list(o["node_mem_free"][0]) == [10, 2]
+    assert o["rounds_used"][0] == 5 and o["occupancy"][0, :5].tolist() == [[1, 0], [1, 1], [1, 1], [1, 1], [0, 0]]
+    # without the marks nothing is given back: a2 never finds a node, a3 never gets past it
+    a["traj_last"][:] = 0
+    o = oracle.replay_trace_pinned(pools, a, round_us=10_000, max_rounds=30)
+    assert list(o["alloc_units"][0]) == [1, 1, 0, 0] and o["rounds_used"][0] == 30
+    assert list(o["traj_node"][0]) == [0, 1, -1] and list(o["node_mem_free"][0]) == [2, 1]
+
+
 # ------------------------------------------------------------------ CUDA path against the oracle
 KEYS = ("status", "n_selected", "total_act_us", "alloc_units", "place_node", "place_off", "act_us")
 POOLS = (Pool(POOL_CPU, 64, 16), Pool(POOL_GPU, 32, 8), Pool(POOL_API, 40, 0, 0), Pool(POOL_CPU, 32, 8))
