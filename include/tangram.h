@@ -258,10 +258,21 @@ typedef struct {
   int32_t* traj_node;          /* [scenario][max_trajectories] pool index of the node, -1 = not pinned   */
   int64_t* node_mem_free;      /* [scenario][n_pools] free memory of every CPU pool (other entries unused) */
   uint8_t* pool_out;           /* [scenario][action] the pool column with the trajectories' nodes        */
-  int32_t* n_admitted;         /* [scenario]                                                             */
+  int32_t* n_admitted;         /* [scenario]; not used by tangram_replay_trace_pinned (may be null there) */
+  const uint8_t* traj_last;    /* per action, may be null; tangram_replay_trace_pinned only: non-zero marks the
+                                  last action of its trajectory                                          */
 } tangram_pinning;
 int tangram_pin_trajectories(tangram_round* round, const tangram_actions* actions, const tangram_pinning* pin,
                              void* cuda_stream);
+/* tangram_replay_trace (policy 0 or 3) / tangram_replay_trace_ordered (policy 1, 2) with the trajectories pinned
+ * as their actions arrive: in a round, after the releases, every arrival is pinned by the rule above against the
+ * memory free at that moment; the first arrival whose trajectory finds no node waits outside the queue, with
+ * everything that arrived after it, and is tried again every round.  When an action marked in traj_last ends,
+ * its traj_mem goes back to its trajectory's node and the trajectory is no longer pinned.  pool_out (written
+ * by the call) is the pool every action ran or waits on; traj_node / node_mem_free hold the final state.
+ * Device buffers only. */
+int tangram_replay_trace_pinned(tangram_round* round, const tangram_actions* actions, int policy,
+                                const tangram_pinning* pin, tangram_result* result, void* cuda_stream);
 
 /* Measurement aid (no counterpart in the paper).  tangram_set_profiling(round, 1) creates CUDA
  * events once; from then on every call records events around each of its kernels on the

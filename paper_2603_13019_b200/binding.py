@@ -45,7 +45,7 @@ class _Actions(C.Structure):
 class _Pinning(C.Structure):
     _fields_ = [("trajectory", C.c_void_p), ("traj_mem", C.c_void_p), ("max_trajectories", C.c_int32),
                 ("traj_node", C.c_void_p), ("node_mem_free", C.c_void_p), ("pool_out", C.c_void_p),
-                ("n_admitted", C.c_void_p)]
+                ("n_admitted", C.c_void_p), ("traj_last", C.c_void_p)]
 
 
 class _Result(C.Structure):
@@ -58,7 +58,7 @@ EXPORTS = ("tangram_round_create", "tangram_schedule_batch", "tangram_replay_tra
            "tangram_round_destroy", "tangram_kernel_launches", "tangram_strerror",
            "tangram_last_cuda_error", "tangram_set_profiling", "tangram_kernel_time_ms",
            "tangram_kernel_name", "tangram_schedule_batch_static", "tangram_order_queue",
-           "tangram_schedule_batch_ordered", "tangram_pin_trajectories", "tangram_replay_trace_ordered")
+           "tangram_schedule_batch_ordered", "tangram_pin_trajectories", "tangram_replay_trace_ordered", "tangram_replay_trace_pinned")
 
 
 def load_library(path: Optional[str] = None):
@@ -98,6 +98,9 @@ def load_library(path: Optional[str] = None):
                                                    C.POINTER(_Result), C.c_void_p]
     lib.tangram_replay_trace_ordered.restype = C.c_int
     lib.tangram_replay_trace_ordered.argtypes = [C.c_void_p, C.POINTER(_Actions), C.c_int, C.POINTER(_Result), C.c_void_p]
+    lib.tangram_replay_trace_pinned.restype = C.c_int
+    lib.tangram_replay_trace_pinned.argtypes = [C.c_void_p, C.POINTER(_Actions), C.c_int, C.POINTER(_Pinning),
+                                                C.POINTER(_Result), C.c_void_p]
     lib.tangram_pin_trajectories.restype = C.c_int
     lib.tangram_pin_trajectories.argtypes = [C.c_void_p, C.POINTER(_Actions), C.POINTER(_Pinning), C.c_void_p]
     lib.tangram_schedule_batch_static.argtypes = [C.POINTER(_RoundDesc), C.POINTER(_Actions), C.c_int64,
@@ -265,10 +268,30 @@ class Round:
                        self._ptr("traj_mem", actions["traj_mem"], torch.int32, S * N), T,
                        self._ptr("traj_node", actions["traj_node"], torch.int32, S * T),
                        self._ptr("node_mem_free", actions["node_mem_free"], torch.int64, S * len(self.pools)),
-                       out["pool"].data_ptr(), out["n_admitted"].data_ptr())
+                       out["pool"].data_ptr(), out["n_admitted"].data_ptr(), None)
         a = self._actions(actions)
         _check(self._lib.tangram_pin_trajectories(self._h, C.byref(a), C.byref(pin), self._stream(stream)))
         return out
+
+    def replay_trace_pinned(self, actions: Dict, policy: int = 0, result: Optional[Dict] = None, stream=None) -> Dict:
+        """tangram_replay_trace_pinned: the replay with trajectories pinned as their actions arrive
+        (actions["trajectory"], ["traj_mem"], ["traj_last"] uint8; state ["traj_node"], ["node_mem_free"] updated
+        in place).  The result gets "pool": the pool every action ran or waits on."""
+        import torch
+        S, N = self.n_scenarios, self.max_actions
+        T = actions["traj_node"].shape[1]
+        result = self.new_result(replay=True) if result is None else result
+        result["pool"] = torch.empty((S, N), dtype=torch.uint8, device="cuda")
+        pin = _Pinning(self._ptr("trajectory", actions["trajectory"], torch.int32, S * N),
+                       self._ptr("traj_mem", actions["traj_mem"], torch.int32, S * N), T,
+                       self._ptr("traj_node", actions["traj_node"], torch.int32, S * T),
+                       self._ptr("node_mem_free", actions["node_mem_free"], torch.int64, S * len(self.pools)),
+                       result["pool"].data_ptr(), None,
+                       self._ptr("traj_last", actions.get("traj_last"), torch.uint8, S * N))
+        a, r = self._actions(actions), self._result(result)
+        _check(self._lib.tangram_replay_trace_pinned(self._h, C.byref(a), int(policy), C.byref(pin), C.byref(r),
+                                                     self._stream(stream)))
+        return result
 
     def set_profiling(self, enable: bool):
         """tangram_set_profiling: record CUDA events around every kernel of the following calls."""

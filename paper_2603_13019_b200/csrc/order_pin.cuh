@@ -192,6 +192,53 @@ struct PinIo {
   int* traj_node; i64* mem_free; u8* pool_out; int* n_admitted;
 };
 
+// One chunk of up to 32 consecutive queue actions, one per lane (`have`: the lane holds one; rec = its record
+// index).  Lane j < P keeps node j's free memory (mf) and cores (-1: not a CPU node).  The actions whose
+// trajectory has no node yet are taken one after the other, lowest lane first.  Returns the lane of the first
+// action whose trajectory finds no node (32 if none); pool_of = the lane's pool afterwards (its trajectory's
+// node, or its own pool; untouched for a lane without an action); the actions from the returned lane on keep
+// their pools.
+__device__ __forceinline__ int pin_chunk(const Params& P, const u8* a_pool, size_t rec, bool have, const int* trajectory,
+                                         const u32* traj_mem, int max_traj, int* tn, i64& mf, int cores, int lane,
+                                         int& pool_of) {
+  int pj = 0xff, t = -1, node = -1, need = 0; u32 mem = 0;
+  bool mine = false;                                    // an action of the CPU manager with a trajectory
+  if (have) {
+    pj = a_pool[rec];
+    t = trajectory[rec];
+    mine = t >= 0 && t < max_traj && pj < P.P && P.pool[pj].type == TG_POOL_CPU;
+    if (mine) {
+      node = tn[t]; mem = traj_mem[rec];
+      const u32 mk = P.a_mask[rec];
+      need = (int)(P.a_unit[rec] & 0x7f) * (mk ? __ffs(mk) : 0);   // cores of the least level
+    }
+  }
+  int first_out = 32;
+  u32 open = __ballot_sync(TG_FULL, mine && node < 0);
+  while (open) {
+    const int b = __ffs(open) - 1;
+    const int bt = __shfl_sync(TG_FULL, t, b), bneed = __shfl_sync(TG_FULL, need, b);
+    const u32 bmem = __shfl_sync(TG_FULL, mem, b);
+    // the eligible node with the most free memory, lowest index on ties
+    const bool ok = cores >= 0 && cores >= bneed && mf >= (i64)bmem;
+    const i64 best = warp_max64_from_m1(ok ? mf : -1);
+    const u32 who = __ballot_sync(TG_FULL, ok && mf == best);
+    if (!who) {                                         // no node: the admitted queue ends before this action
+      first_out = b;
+      if (lane >= b) mine = false;                      // nothing from it on is touched
+      break;
+    }
+    const int bn = __ffs(who) - 1;
+    if (lane == bn) mf -= (i64)bmem;
+    if (lane == 0) tn[bt] = bn;
+    if (mine && t == bt) node = bn;                     // later actions of the trajectory in this chunk follow
+    open = __ballot_sync(TG_FULL, mine && node < 0) & ~((2u << b) - 1u);
+  }
+  if (have) pool_of = (mine && node >= 0) ? node : pj;
+  __syncwarp();
+  return first_out;
+}
+
 __global__ void __launch_bounds__(256) k_pin(const __grid_constant__ Params P, const PinIo X) {
   const int lane = threadIdx.x & 31;
   const int sc = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
@@ -203,44 +250,14 @@ __global__ void __launch_bounds__(256) k_pin(const __grid_constant__ Params P, c
   i64 mf = 0; int cores = -1;
   if (lane < P.P && P.pool[lane].type == TG_POOL_CPU) { mf = X.mem_free[(size_t)sc * P.P + lane]; cores = P.pool[lane].capacity; }
   int admitted = n;
-  bool stop = false;
   for (int c0 = 0; c0 < P.N; c0 += 32) {
     const int i = c0 + lane;
-    int pj = 0xff, t = -1, node = -1, need = 0; u32 mem = 0;
-    bool mine = false;                                  // an action of the CPU manager with a trajectory
-    if (i < P.N) pj = P.a_pool[row + i];
-    if (i < n && !stop) {
-      t = X.trajectory[row + i];
-      mine = t >= 0 && t < X.max_traj && pj < P.P && P.pool[pj].type == TG_POOL_CPU;
-      if (mine) {
-        node = tn[t]; mem = X.traj_mem[row + i];
-        const u32 mk = P.a_mask[row + i];
-        need = (int)(P.a_unit[row + i] & 0x7f) * (mk ? __ffs(mk) : 0);   // cores of the least level
-      }
+    int pool_of = i < P.N ? P.a_pool[row + i] : 0xff;
+    if (admitted == n && c0 < n) {                      // (behind the admitted queue the pool column is copied)
+      const int out = pin_chunk(P, P.a_pool, row + i, i < n, X.trajectory, X.traj_mem, X.max_traj, tn, mf, cores, lane, pool_of);
+      if (out < 32) admitted = c0 + out;
     }
-    // trajectories that are not pinned yet, one after the other in queue order
-    u32 open = __ballot_sync(TG_FULL, mine && node < 0);
-    while (open) {
-      const int b = __ffs(open) - 1;
-      const int bt = __shfl_sync(TG_FULL, t, b), bneed = __shfl_sync(TG_FULL, need, b);
-      const u32 bmem = __shfl_sync(TG_FULL, mem, b);
-      // the eligible node with the most free memory, lowest index on ties
-      const bool ok = cores >= 0 && cores >= bneed && mf >= (i64)bmem;
-      const i64 best = warp_max64_from_m1(ok ? mf : -1);
-      const u32 who = __ballot_sync(TG_FULL, ok && mf == best);
-      if (!who) {                                       // no node: the admitted queue ends before this action
-        admitted = c0 + b; stop = true;
-        if (lane >= b) mine = false;                    // nothing behind it is touched
-        break;
-      }
-      const int bn = __ffs(who) - 1;
-      if (lane == bn) mf -= (i64)bmem;
-      if (lane == 0) tn[bt] = bn;
-      if (mine && t == bt) node = bn;                   // later actions of the trajectory in this chunk follow
-      open = __ballot_sync(TG_FULL, mine && node < 0) & ~((2u << b) - 1u);
-    }
-    if (i < P.N) X.pool_out[row + i] = (u8)((mine && node >= 0) ? node : pj);
-    __syncwarp();
+    if (i < P.N) X.pool_out[row + i] = (u8)pool_of;
   }
   if (lane < P.P && cores >= 0) X.mem_free[(size_t)sc * P.P + lane] = mf;
   if (lane == 0) X.n_admitted[sc] = admitted;

@@ -13,6 +13,7 @@
 #include "sims.cuh"
 #include "select.cuh"
 #include "place.cuh"
+#include "order_pin.cuh"
 
 struct ReplayWs {
   int* wait;        // [S][N] waiting actions in queue order
@@ -28,6 +29,9 @@ struct ReplayWs {
   int* occupancy; int* rounds_used;
   int policy;       // 0: first come first served; 1 / 2: the queue is kept in shortest / longest least-level duration order
   u64* wkey;        // [S][N] sort keys of the waiting actions (policy 1 / 2 only)
+  // trajectories pinned to CPU nodes as their actions arrive (Section 5.2); trajectory == nullptr: none of it
+  const int* trajectory; const u32* traj_mem; const u8* traj_last; int max_traj;
+  int* traj_node; i64* mem_free; u8* pool_rw;   // pool_rw: the pool column the kernel reads (P.a_pool) and rewrites
   int state_bytes;  // > 0: a scenario's live state (owner .. win) fits that many bytes of shared memory per warp
 };
 
@@ -259,7 +263,8 @@ __device__ bool replay_pool(const Params& P, const ReplayWs& R, const ReplayStat
 #define KR_THREADS 64
 #define KR_DYN_SMEM ((KR_THREADS / 32) * (WARP_SMEM_BYTES + 320) + 16)
 #define KR_STATE_MAX 16384
-// ORDERED: the waiting queue is kept sorted by R.policy's key (the plain instance keeps its registers).
+// ORDERED: the extended instance: the waiting queue may be kept sorted by R.policy's key and the trajectories
+// pinned on arrival (R.trajectory); the plain instance keeps its registers.
 template <bool ORDERED>
 __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant__ Params P, const ReplayWs R) {
   const int lane = threadIdx.x & 31;
@@ -368,6 +373,14 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
             const int fa = __shfl_sync(TG_FULL, a, b);
             const int j = P.a_pool[row + fa];
             const PoolDev& pd = P.pool[j];
+            if (ORDERED && R.trajectory && R.traj_last && lane == 0 && R.traj_last[row + fa] && pd.type == TG_POOL_CPU) {
+              // the trajectory's last action has ended: its memory goes back to its node
+              const int t = R.trajectory[row + fa];
+              if (t >= 0 && t < R.max_traj) {
+                int* tn = R.traj_node + (size_t)sc * R.max_traj;
+                if (tn[t] >= 0) { R.mem_free[(size_t)sc * P.P + tn[t]] += (i64)R.traj_mem[row + fa]; tn[t] = -1; }
+              }
+            }
             if (P.n_side > 0 && lane == 0)                 // a concurrency pool held the action's further amounts until now
               for (int e = 0; e < P.n_side; ++e) {
                 const int k = P.a_side_pool[e * P.side_plane + row + fa];
@@ -408,13 +421,33 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
           const int i = next + lane;
           const bool in = i < n_act && (P.a_arrival ? P.a_arrival[row + i] : 0) <= now;
           const u32 b = __ballot_sync(TG_FULL, in);
-          const int cnt = (b == TG_FULL) ? 32 : __ffs(~b) - 1;        // arrivals are sorted: a prefix of the lanes
+          int cnt = (b == TG_FULL) ? 32 : __ffs(~b) - 1;              // arrivals are sorted: a prefix of the lanes
+          if (ORDERED && R.trajectory && cnt > 0) {
+            // per-node CPU scheduling: an arrival joins the queue once its trajectory has a node; the first one
+            // that finds none waits outside, with everything that arrived after it
+            __syncwarp();
+            i64 mf = 0; int cores = -1;
+            if (lane < P.P && P.pool[lane].type == TG_POOL_CPU) { mf = R.mem_free[(size_t)sc * P.P + lane]; cores = P.pool[lane].capacity; }
+            int pool_of = 0xff;
+            const int out = pin_chunk(P, R.pool_rw, row + i, lane < cnt, R.trajectory, R.traj_mem, R.max_traj,
+                                      R.traj_node + (size_t)sc * R.max_traj, mf, cores, lane, pool_of);
+            if (lane < P.P && cores >= 0) R.mem_free[(size_t)sc * P.P + lane] = mf;
+            const int adm = min(cnt, out);
+            if (lane < adm) R.pool_rw[row + i] = (u8)pool_of;
+            __syncwarp();
+            if (adm < cnt) {                                  // the gate: nothing behind the action without a node gets in
+              if (lane < adm) wait[nw + lane] = i;
+              nw += adm; next += adm;
+              break;
+            }
+            cnt = adm;
+          }
           if (lane < cnt) wait[nw + lane] = i;
           nw += cnt; next += cnt;
           if (cnt < 32) break;
         }
         __syncwarp();
-        if (ORDERED && nw > nw_admitted) {
+        if (ORDERED && R.policy && nw > nw_admitted) {
           // Other queue orders (Section 4.2): the queue stays sorted by the policy's key, equal keys in arrival
           // order.  Each new arrival goes behind the last entry whose key is not larger; the tail moves up by one.
           u64* wkey = R.wkey + row;
@@ -446,7 +479,7 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
         int blocked_pool = -1;                              // pool of a head-of-line action that does not fit
         if (nw > 0) {
           const int n = replay_prefix(P, R, Z, sc, wait, nw, dem, cap, aside, ncand, lane);
-          if (n == 0 && P.n_side == 0) blocked_pool = P.a_pool[row + wait[0]];
+          if (n == 0 && P.n_side == 0 && !(ORDERED && R.trajectory)) blocked_pool = P.a_pool[row + wait[0]];   // (a pin made later would see other free memory)
           const int nr0 = nr;
           bool ok = true;
           if (n > 0)
@@ -475,10 +508,10 @@ __global__ void __launch_bounds__(KR_THREADS, 1) k_replay(const __grid_constant_
               const int i = i0 + lane;
               int a = -1; bool stay = false;
               u64 kk = 0;
-              if (i < nw) { a = wait[i]; stay = P.o_act[row + a] < 0; if (ORDERED) kk = R.wkey[row + i]; }
+              if (i < nw) { a = wait[i]; stay = P.o_act[row + a] < 0; if (ORDERED && R.policy) kk = R.wkey[row + i]; }
               const u32 b = __ballot_sync(TG_FULL, stay);
               __syncwarp();
-              if (stay) { wait[kw + __popc(b & ((1u << lane) - 1u))] = a; if (ORDERED) R.wkey[row + kw + __popc(b & ((1u << lane) - 1u))] = kk; }
+              if (stay) { wait[kw + __popc(b & ((1u << lane) - 1u))] = a; if (ORDERED && R.policy) R.wkey[row + kw + __popc(b & ((1u << lane) - 1u))] = kk; }
               kw += __popc(b);
             }
             nw = kw;

@@ -1030,7 +1030,8 @@ extern "C" int tangram_schedule_batch(tangram_round* r, const tangram_actions* a
   return TANGRAM_OK;
 }
 
-static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_result* res, void* cuda_stream, int policy);
+static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_result* res, void* cuda_stream, int policy,
+                       const tangram_pinning* pin = nullptr);
 
 extern "C" int tangram_replay_trace(tangram_round* r, const tangram_actions* a, tangram_result* res,
                                     void* cuda_stream) {
@@ -1043,7 +1044,16 @@ extern "C" int tangram_replay_trace_ordered(tangram_round* r, const tangram_acti
   return replay_impl(r, a, res, cuda_stream, policy == 3 ? 0 : policy);   // a trace is sorted by arrival already
 }
 
-static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_result* res, void* cuda_stream, int policy) {
+extern "C" int tangram_replay_trace_pinned(tangram_round* r, const tangram_actions* a, int policy,
+                                           const tangram_pinning* pin, tangram_result* res, void* cuda_stream) {
+  if (policy < 0 || policy > 3 || !r || !pin || r->desc.host_buffers || !pin->trajectory || !pin->traj_mem ||
+      pin->max_trajectories < 1 || !pin->traj_node || !pin->node_mem_free || !pin->pool_out)
+    return TANGRAM_EINVAL;
+  return replay_impl(r, a, res, cuda_stream, policy == 3 ? 0 : policy, pin);
+}
+
+static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_result* res, void* cuda_stream, int policy,
+                       const tangram_pinning* pin) {
   if (!r || !check_io(a, res) || r->desc.max_rounds <= 0 || !a->arrival_us) return TANGRAM_EINVAL;
   if (policy && !r->d_wkey) {                              // sort keys of the waiting actions, kept by the round
     if (cudaMalloc((void**)&r->d_wkey, (size_t)r->P.S * r->P.N * sizeof(u64)) != cudaSuccess) {
@@ -1058,6 +1068,8 @@ static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_resul
   P.now = 0;
   ReplayWs R = r->R;
   R.policy = policy; R.wkey = policy ? r->d_wkey : nullptr;
+  R.trajectory = nullptr; R.traj_mem = nullptr; R.traj_last = nullptr; R.max_traj = 0;
+  R.traj_node = nullptr; R.mem_free = nullptr; R.pool_rw = nullptr;
   if (r->desc.host_buffers) {
     bind_stage(r, a, P);
     int rc = copy_in(r, a, P, 0, P.S, st);
@@ -1079,7 +1091,15 @@ static int replay_impl(tangram_round* r, const tangram_actions* a, tangram_resul
                         2 * align16((size_t)P.P * 8);
     R.state_bytes = need <= KR_STATE_MAX ? (int)need : 0;
   }
-  if (policy) k_replay<true><<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM + (KR_THREADS / 32) * R.state_bytes, st>>>(P, R);
+  if (pin) {
+    // the kernel reads and rewrites the caller's pool_out: it starts as a copy of the pool column
+    CK(cudaMemcpyAsync(pin->pool_out, a->pool, (size_t)P.S * P.N, cudaMemcpyDeviceToDevice, st));
+    P.a_pool = pin->pool_out;
+    R.trajectory = pin->trajectory; R.traj_mem = pin->traj_mem; R.traj_last = pin->traj_last;
+    R.max_traj = pin->max_trajectories; R.traj_node = pin->traj_node; R.mem_free = (i64*)pin->node_mem_free;
+    R.pool_rw = pin->pool_out;
+  }
+  if (policy || pin) k_replay<true><<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM + (KR_THREADS / 32) * R.state_bytes, st>>>(P, R);
   else k_replay<false><<<warps / (KR_THREADS / 32), KR_THREADS, KR_DYN_SMEM + (KR_THREADS / 32) * R.state_bytes, st>>>(P, R);
   if (ev) CK(cudaEventRecord(ev[1], st));
   r->launches += 1;

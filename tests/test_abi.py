@@ -103,6 +103,7 @@ def test_calls_reject_null_handles_and_buffers():
     assert lib.tangram_schedule_batch_ordered(None, ctypes.byref(a), 1, 0, ctypes.byref(r), None) == EINVAL
     assert lib.tangram_pin_trajectories(None, ctypes.byref(a), ctypes.byref(pin), None) == EINVAL
     assert lib.tangram_replay_trace_ordered(None, ctypes.byref(a), 1, ctypes.byref(r), None) == EINVAL
+    assert lib.tangram_replay_trace_pinned(None, ctypes.byref(a), 0, ctypes.byref(pin), ctypes.byref(r), None) == EINVAL
     # the allocation-free entry point validates its description and buffers the same way
     d, keep = _desc(binding, [(0, 64, 8, 0)])
     assert lib.tangram_schedule_batch_static(None, ctypes.byref(a), 0, ctypes.byref(r), None) == EINVAL

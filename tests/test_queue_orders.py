@@ -264,3 +264,33 @@ def test_ordered_traces_match_oracle(oracle, seed, policy):
         assert np.array_equal(of[k], plain[k].cpu().numpy()), k
     assert not np.array_equal(of["act_us"], o["act_us"])
     rnd.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed,policy", [(0, 0), (1, 0), (2, SJF), (3, 0), (4, LJF)])
+def test_traces_with_trajectories_pinned_on_arrival_match_oracle(oracle, seed, policy):
+    import torch
+    from paper_2603_13019_b200 import binding
+    pools = [(Pool(POOL_CPU, 16, 4), Pool(POOL_CPU, 8, 4), Pool(POOL_GPU, 16, 8)),
+             (Pool(POOL_CPU, 6, 3), Pool(POOL_CPU, 6, 3), Pool(POOL_CPU, 12, 4)),
+             (Pool(POOL_CPU, 16, 4), Pool(POOL_API, 6, 0, 0), Pool(POOL_CPU, 16, 8)),
+             (Pool(POOL_CPU, 4, 4), Pool(POOL_CPU, 4, 4)),
+             (Pool(POOL_CPU, 24, 8), Pool(POOL_GPU, 8, 8), Pool(POOL_CPU, 8, 8))][seed]
+    N = [200, 300, 150, 400, 250][seed]
+    w, a = random_round(990 + seed, 12, N, pools, max_mult=4, small_durations=0.3, replicas=0.0)
+    rng = np.random.default_rng(seed)
+    a["arrival_us"] = np.cumsum(rng.integers(0, [3000, 2000, 3000, 1500, 3000][seed], a["pool"].shape), axis=1).astype(np.int64)
+    # memory is tight enough for arrivals to wait at the gate, in some scenarios for good
+    a = add_trajectories(seed, a, pools, max_traj=[40, 25, 30, 60, 35][seed], mem_hi=40, pinned=0.0, mem_free_hi=700)
+    o = oracle.replay_trace_pinned(pools, a, round_us=10_000, max_rounds=4000, policy=policy)
+    rnd = binding.Round(12, N, pools, round_us=10_000, max_rounds=4000)
+    dev = binding.to_device(a)
+    dev["traj_mem"] = dev["traj_mem"].view(torch.int32)
+    g = rnd.replay_trace_pinned(dev, policy=policy)
+    torch.cuda.synchronize()
+    for k in KEYS + ("rounds_used", "occupancy", "pool"):
+        assert np.array_equal(o[k], g[k].cpu().numpy()), k
+    assert np.array_equal(o["traj_node"], dev["traj_node"].cpu().numpy())
+    assert np.array_equal(o["node_mem_free"], dev["node_mem_free"].cpu().numpy())
+    assert (o["alloc_units"] > 0).sum() > 500 and (o["pool"] != a["pool"]).sum() > 30
+    rnd.destroy()

@@ -438,7 +438,8 @@ def add_trajectories(seed: int, arrays: Dict[str, Optional[np.ndarray]], pools: 
                      fraction: float = 0.9, mem_hi: int = 64, pinned: float = 0.3,
                      mem_free_hi: int = 600) -> Dict[str, Optional[np.ndarray]]:
     """Trajectories for the per-node CPU scheduling (Section 5.2): returns a copy of `arrays` with "trajectory"
-    (int32 per action, -1 = none), "traj_mem" (uint32, memory of the whole trajectory), and the state
+    (int32 per action, -1 = none), "traj_mem" (uint32, memory of the whole trajectory), "traj_last" (uint8, marks
+    the last action of nine in ten trajectories), and the state
     "traj_node" ([scenario][max_traj], a fraction already pinned to a random CPU pool) and "node_mem_free"
     ([scenario][pool])."""
     rng = np.random.Generator(np.random.PCG64(seed))
@@ -451,6 +452,17 @@ def add_trajectories(seed: int, arrays: Dict[str, Optional[np.ndarray]], pools: 
     out = dict(arrays)
     out["trajectory"], out["traj_mem"], out["traj_node"] = traj, mem, node
     out["node_mem_free"] = rng.integers(0, mem_free_hi + 1, size=(S, len(pools))).astype(np.int64)
+    # the last action of most trajectories is marked (a trace gives the memory back when it ends)
+    last = np.zeros((S, N), np.uint8)
+    n_act = arrays["n_actions"]
+    for sc in range(S):
+        seen = set()
+        for i in range(int(n_act[sc]) - 1, -1, -1):
+            t = int(traj[sc, i])
+            if t >= 0 and t not in seen:
+                seen.add(t)
+                last[sc, i] = 1
+    out["traj_last"] = np.where(rng.random((S, N)) < 0.9, last, 0).astype(np.uint8)
     return out
 
 
