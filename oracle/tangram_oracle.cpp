@@ -103,7 +103,9 @@
 // restoration once per action; an amount that ends the prefix, a later candidate's amount set
 // aside, an evicted candidate that consumes nothing, concurrency and quota bookkeeping over
 // rounds; keys and ties of the three orders, the ordered round against the plain round on the
-// permuted records; most-free-memory node, the core and memory filters, the admitted queue).
+// permuted records, a one-core trace whose three orders differ; most-free-memory node, the core and
+// memory filters, the admitted queue, a replay in which an arrival waits at the gate until a
+// trajectory's last action gives its memory back).
 #include <algorithm>
 #include <climits>
 #include <cstdint>
